@@ -1,0 +1,194 @@
+/*
+ * CPU oracle for per-example gradient statistics of a linear layer.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain restatement of what the
+ * method computes; it exists so that the CUDA library can be checked against
+ * something written independently from the paper.  It shares no code with the
+ * CUDA path and nothing in the product may call it.
+ *
+ * Conventions: X is [B, T, d_in], dY is [B, T, d_out], both row-major.  Outputs
+ * are [d_out, d_in] row-major (the transpose of the paper's D x F layout, same
+ * numbers).  All arithmetic is fp64; inputs are either fp32 or bf16 bit patterns
+ * and are widened exactly.
+ *
+ * Every function here follows the "one example at a time" route of Section 2.1
+ * (the compute-intensive implementation): form the gradient of example b, apply
+ * phi to it, add it to the running sum over b.  That is the definition of the
+ * statistic in Eq. (2) with the 1/B left to the caller.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* bf16 -> double: a bf16 is the upper half of an IEEE binary32. */
+static double widen_bf16(uint16_t h) {
+  uint32_t u = ((uint32_t)h) << 16;
+  float f;
+  memcpy(&f, &u, sizeof f);
+  return (double)f;
+}
+
+/* Copy rows [row0, row0+rows) of a [*, width] matrix into doubles. */
+static void widen_rows(const void* src, int is_bf16, long long row0, long long rows, long long width,
+                       double* dst) {
+  long long n = rows * width, off = row0 * width;
+  if (is_bf16) {
+    const uint16_t* p = (const uint16_t*)src + off;
+    for (long long k = 0; k < n; ++k) dst[k] = widen_bf16(p[k]);
+  } else {
+    const float* p = (const float*)src + off;
+    for (long long k = 0; k < n; ++k) dst[k] = (double)p[k];
+  }
+}
+
+static double sign3(double g) { return (g > 0.0) - (g < 0.0); } /* sign(0) = 0 */
+
+/*
+ * Sequence-level per-example statistics (Section 2.3, "Dense layers in
+ * sequence-level architectures"): for each example b the gradient is the
+ * contraction over that sequence's tokens only,
+ *     G_b[o,i] = sum_t dY[b,t,o] * X[b,t,i],
+ * phi is applied to the whole G_b (after the sum over t) and the results are
+ * summed over b (Eq. (2), Eq. (3), and the sign statistic of Section 3.1).
+ *
+ *   sum_g   [d_out*d_in]  = sum_b G_b                (the ordinary batch gradient)
+ *   sum_g2  [d_out*d_in]  = sum_b G_b^2
+ *   sum_sgn [d_out*d_in]  = sum_b sign(G_b),  sign(0) = 0
+ *   max_abs [B]           = max_{o,i} |G_b[o,i]|
+ *   n_small [d_out*d_in]  = number of examples b with |G_b[o,i]| <= small_rel * max_abs[b]
+ *                           (entries whose sign a lower-precision evaluation may flip)
+ * Any output pointer may be NULL.  Returns 0, or 1 on bad arguments / allocation failure.
+ */
+int oracle_linear_stats(const void* X, const void* dY, int is_bf16, int B, int T, int d_in, int d_out,
+                        double small_rel, double* sum_g, double* sum_g2, double* sum_sgn,
+                        double* max_abs, int32_t* n_small) {
+  if (!X || !dY || B < 0 || T < 0 || d_in <= 0 || d_out <= 0) return 1;
+  long long n = (long long)d_out * d_in;
+  double* G = (double*)malloc(sizeof(double) * (size_t)n);
+  double* xb = (double*)malloc(sizeof(double) * (size_t)((long long)(T > 0 ? T : 1) * d_in));
+  double* yb = (double*)malloc(sizeof(double) * (size_t)((long long)(T > 0 ? T : 1) * d_out));
+  if (!G || !xb || !yb) { free(G); free(xb); free(yb); return 1; }
+  for (long long k = 0; k < n; ++k) {
+    if (sum_g) sum_g[k] = 0.0;
+    if (sum_g2) sum_g2[k] = 0.0;
+    if (sum_sgn) sum_sgn[k] = 0.0;
+    if (n_small) n_small[k] = 0;
+  }
+  for (int b = 0; b < B; ++b) {
+    widen_rows(X, is_bf16, (long long)b * T, T, d_in, xb);
+    widen_rows(dY, is_bf16, (long long)b * T, T, d_out, yb);
+    /* G_b = dY_b^T X_b, contracted over this example's T tokens. */
+#pragma omp parallel for schedule(static)
+    for (int o = 0; o < d_out; ++o) {
+      double* g = G + (long long)o * d_in;
+      for (int i = 0; i < d_in; ++i) g[i] = 0.0;
+      for (int t = 0; t < T; ++t) {
+        double lam = yb[(long long)t * d_out + o];
+        const double* h = xb + (long long)t * d_in;
+        for (int i = 0; i < d_in; ++i) g[i] += lam * h[i];
+      }
+    }
+    double mx = 0.0;
+    for (long long k = 0; k < n; ++k) {
+      double a = fabs(G[k]);
+      if (a > mx) mx = a;
+    }
+    if (max_abs) max_abs[b] = mx;
+    /* phi, then the sum over examples. */
+    for (long long k = 0; k < n; ++k) {
+      double g = G[k];
+      if (sum_g) sum_g[k] += g;
+      if (sum_g2) sum_g2[k] += g * g;
+      if (sum_sgn) sum_sgn[k] += sign3(g);
+      if (n_small && fabs(g) <= small_rel * mx) n_small[k] += 1;
+    }
+  }
+  free(G); free(xb); free(yb);
+  return 0;
+}
+
+/*
+ * Per-token second moment (Section 2.3, the "per-token" alternative):
+ *     S'[o,i] = sum_{b,t} dY[b,t,o]^2 * X[b,t,i]^2 ,
+ * one term per (example, token) row; B and T only enter as the row count.
+ */
+int oracle_token_sqstats(const void* X, const void* dY, int is_bf16, int B, int T, int d_in, int d_out,
+                         double* out) {
+  if (!X || !dY || !out || B < 0 || T < 0 || d_in <= 0 || d_out <= 0) return 1;
+  long long rows = (long long)B * T;
+  long long n = (long long)d_out * d_in;
+  double* xr = (double*)malloc(sizeof(double) * (size_t)d_in);
+  double* yr = (double*)malloc(sizeof(double) * (size_t)d_out);
+  if (!xr || !yr) { free(xr); free(yr); return 1; }
+  for (long long k = 0; k < n; ++k) out[k] = 0.0;
+  for (long long r = 0; r < rows; ++r) {
+    widen_rows(X, is_bf16, r, 1, d_in, xr);
+    widen_rows(dY, is_bf16, r, 1, d_out, yr);
+    for (int i = 0; i < d_in; ++i) xr[i] = xr[i] * xr[i];
+#pragma omp parallel for schedule(static)
+    for (int o = 0; o < d_out; ++o) {
+      double l2 = yr[o] * yr[o];
+      double* s = out + (long long)o * d_in;
+      for (int i = 0; i < d_in; ++i) s[i] += l2 * xr[i];
+    }
+  }
+  free(xr); free(yr);
+  return 0;
+}
+
+/*
+ * One MicroAdam step (Algorithm 1, MicroAdam branch; Eq. (3) for nu):
+ *   mu = s * sum_g / B                       average per-example gradient, g_b = s * G_b
+ *   nu = s^2 * sum_g2 / B                    average element-wise square
+ *   m  = beta1 m + (1 - beta1) mu
+ *   v  = beta2 v + (1 - beta2) nu
+ *   mh = m / (1 - beta1^t),  vh = v / (1 - beta2^t)
+ *   u  = mh / (sqrt(vh) + eps)               eps_inside_sqrt == 0  (Section 3.2.3's form)
+ *   u  = mh / sqrt(eps + vh)                 eps_inside_sqrt != 0  (Algorithm 1 as printed)
+ *   theta = theta - lr * u - wd * theta      decay not multiplied by lr (Appendix E)
+ * theta, m, v are updated in place.  step is 1-based.
+ */
+int oracle_microadam_step(double* theta, double* m, double* v, const double* sum_g, const double* sum_g2,
+                          long long n, int B, double grad_scale, double lr, double beta1, double beta2,
+                          double eps, int eps_inside_sqrt, double weight_decay, int step) {
+  if (!theta || !m || !v || !sum_g || !sum_g2 || n < 0 || B < 1 || step < 1) return 1;
+  double c1 = 1.0 - pow(beta1, (double)step);
+  double c2 = 1.0 - pow(beta2, (double)step);
+  for (long long k = 0; k < n; ++k) {
+    double mu = grad_scale * sum_g[k] / (double)B;
+    double nu = grad_scale * grad_scale * sum_g2[k] / (double)B;
+    m[k] = beta1 * m[k] + (1.0 - beta1) * mu;
+    v[k] = beta2 * v[k] + (1.0 - beta2) * nu;
+    double mh = m[k] / c1;
+    double vh = v[k] / c2;
+    double u = eps_inside_sqrt ? mh / sqrt(eps + vh) : mh / (sqrt(vh) + eps);
+    theta[k] = theta[k] - lr * u - weight_decay * theta[k];
+  }
+  return 0;
+}
+
+/*
+ * One MicroSignSGD step (Section 3.1: EMA o avg o sign):
+ *   sbar = sum_sgn / B                       average of per-example signs
+ *   m    = beta m + (1 - beta) sbar          plain EMA, no bias correction
+ *   theta = theta - lr * m - wd * theta
+ */
+int oracle_microsignsgd_step(double* theta, double* m, const double* sum_sgn, long long n, int B,
+                             double lr, double beta, double weight_decay) {
+  if (!theta || !m || !sum_sgn || n < 0 || B < 1) return 1;
+  for (long long k = 0; k < n; ++k) {
+    double sbar = sum_sgn[k] / (double)B;
+    m[k] = beta * m[k] + (1.0 - beta) * sbar;
+    theta[k] = theta[k] - lr * m[k] - weight_decay * theta[k];
+  }
+  return 0;
+}
+
+/* Number of OpenMP threads the loops above will use (1 when built without OpenMP). */
+#ifdef _OPENMP
+#include <omp.h>
+int oracle_num_threads(void) { return omp_get_max_threads(); }
+#else
+int oracle_num_threads(void) { return 1; }
+#endif
