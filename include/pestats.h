@@ -1,0 +1,139 @@
+/*
+ * pestats -- per-example gradient statistics for linear layers on NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every pointer is a DEVICE pointer unless its name starts with "h_" or the comment says
+ * "host".  The caller owns every buffer and the stream; the library allocates nothing, keeps no
+ * state between calls apart from the process-wide path override below, and enqueues its work
+ * asynchronously on `stream` (0 = the legacy default stream).  Functions return a pe_status_t and
+ * never throw.  Errors detected on the host (bad arguments, unsupported shape, CUDA launch
+ * failure) are returned immediately and nothing is enqueued.  Errors detected on the device (a
+ * bounded wait inside a kernel that ran out) are latched in a device status word that
+ * pe_get_async_status() reads back.
+ *
+ * Layout conventions (row-major, contiguous):
+ *   X   [B, T, d_in]   activations entering the layer            (the paper's H, "BLD")
+ *   dY  [B, T, d_out]  cotangents of the layer's output          (the paper's Lambda, "BLF")
+ *   per-example gradient  G_b = dY_b^T X_b  is [d_out, d_in]     (transpose of the paper's D x F)
+ *   every statistic is [d_out, d_in] fp32.
+ * There is no CPU fallback: on a machine without an sm_100 GPU the compute calls return
+ * PE_ERR_ARCH or PE_ERR_CUDA.
+ */
+#ifndef PESTATS_H_
+#define PESTATS_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PE_OK = 0,
+  PE_ERR_NULL = 1,              /* a required pointer is NULL */
+  PE_ERR_DIM = 2,               /* a size is zero/negative/too large, or step < 1, or B < 1 */
+  PE_ERR_ALIGN = 3,             /* a pointer is not aligned as documented */
+  PE_ERR_UNSUPPORTED_SHAPE = 4, /* the forced path cannot run this shape */
+  PE_ERR_PHI = 5,               /* phi is not one of pe_phi_t */
+  PE_ERR_ARCH = 6,              /* current device is not compute capability 10.x */
+  PE_ERR_CUDA = 7,              /* a CUDA runtime/driver call failed */
+  PE_ERR_TIMEOUT = 8,           /* a bounded device-side wait ran out (see pe_get_async_status) */
+  PE_ERR_WORKSPACE = 9          /* workspace missing or smaller than *_workspace_bytes() */
+} pe_status_t;
+
+/* The elementwise function applied to each per-example gradient before the sum over examples
+ * (Eq. (2): the nonlinear statistic (1/B) sum_i phi(grad f(theta; x_i)); square gives Eq. (3)'s
+ * nu_micro, sign gives the MicroSignSGD statistic of Section 3.1).  sign(0) = 0. */
+typedef enum { PE_PHI_IDENTITY = 0, PE_PHI_SQUARE = 1, PE_PHI_SIGN = 2 } pe_phi_t;
+
+/* Which kernel family a call may use.  AUTO picks the tensor-core kernel whenever the shape allows
+ * it (bf16 inputs, d_in % 8 == 0, d_out % 8 == 0) and the SIMT kernel otherwise. */
+typedef enum { PE_PATH_AUTO = 0, PE_PATH_SIMT = 1, PE_PATH_TENSOR = 2 } pe_path_t;
+
+typedef struct CUstream_st* pe_stream_t; /* a cudaStream_t */
+
+/*
+ * Sequence-level per-example statistics of a linear layer (Section 2.3, "Dense layers in
+ * sequence-level architectures"; Eq. (2)).  For every example b the gradient
+ *     G_b[o,i] = sum_{t<T} dY[b,t,o] * X[b,t,i]
+ * is formed on chip (it is never written to global memory), and
+ *     out_mean[o,i] = sum_b G_b[o,i]            (the ordinary batch weight gradient, NOT divided by B)
+ *     out_stat[o,i] = sum_b phi(G_b[o,i])
+ * X, dY: bf16, 16-byte aligned.  out_mean, out_stat: fp32 [d_out, d_in], 16-byte aligned, OVERWRITTEN;
+ * either may be NULL to skip it (not both).  Products are exact in fp32 and accumulated in fp32.
+ * B, T >= 0 (B == 0 or T == 0 writes zeros, and X, dY may then be NULL); d_in, d_out >= 1; B*T*max(d_in,d_out) < 2^40.
+ * When the batch is split across thread blocks the partial sums are combined with fp32 atomic
+ * adds, so the low bits of out_mean / the square statistic may differ between runs; the sign
+ * statistic is always exact-integer valued.
+ */
+pe_status_t pe_linear_stats(const void* X, const void* dY, int B, int T, int d_in, int d_out,
+                            pe_phi_t phi, float* out_mean, float* out_stat, pe_stream_t stream);
+
+/* Same for fp32 inputs (4-byte aligned suffices); always the SIMT kernel, fp32 FMA accumulation. */
+pe_status_t pe_linear_stats_f32(const float* X, const float* dY, int B, int T, int d_in, int d_out,
+                                pe_phi_t phi, float* out_mean, float* out_stat, pe_stream_t stream);
+
+/*
+ * Per-token second moment (Section 2.3, the "per-token" alternative):
+ *     out_stat[o,i] = sum_{b,t} dY[b,t,o]^2 * X[b,t,i]^2  =  ((dY o dY)^T (X o X))[o,i].
+ * B and T only enter through the row count B*T.  bf16 inputs.  On the tensor-core path the
+ * squared operands are rounded to bf16 once and staged in `workspace` (device memory, 256-byte
+ * aligned, at least pe_token_sqstats_workspace_bytes() bytes, contents undefined afterwards);
+ * the SIMT path squares in fp32 and ignores the workspace (it may then be NULL).
+ */
+pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_in, int d_out,
+                             float* out_stat, void* workspace, size_t workspace_bytes,
+                             pe_stream_t stream);
+pe_status_t pe_token_sqstats_f32(const float* X, const float* dY, int B, int T, int d_in, int d_out,
+                                 float* out_stat, pe_stream_t stream);
+/* Bytes of workspace pe_token_sqstats needs for this shape under the current path setting (0 when
+ * the SIMT kernel will be used). */
+size_t pe_token_sqstats_workspace_bytes(int B, int T, int d_in, int d_out);
+
+/*
+ * One MicroAdam step over n parameters (Algorithm 1, MicroAdam branch; Eq. (3)):
+ *     mu = s*sum_g/B;  nu = s^2*sum_g2/B;   m = beta1*m + (1-beta1)*mu;   v = beta2*v + (1-beta2)*nu
+ *     mh = m/(1-beta1^step);  vh = v/(1-beta2^step)
+ *     u  = mh/(sqrt(vh)+eps)            if eps_inside_sqrt == 0  (the form of Section 3.2.3)
+ *     u  = mh/sqrt(eps+vh)              otherwise                (Algorithm 1 as printed)
+ *     theta = theta - lr*u - weight_decay*theta                  (decay not scaled by lr, Appendix E)
+ * theta, m, v: fp32 [n], updated in place.  sum_g, sum_g2: fp32 [n], the out_mean / out_stat(square)
+ * of pe_linear_stats.  s = grad_scale converts the passed sums to sums of per-example gradients
+ * (1 if dY came from sum_b f_b, B if it came from the mean loss).  theta_lp: optional bf16 [n] copy
+ * of the new theta (NULL to skip).  step is 1-based.  All pointers 16-byte aligned.
+ */
+pe_status_t microadam_step(float* theta, void* theta_lp, float* m, float* v, const float* sum_g,
+                           const float* sum_g2, long long n, int B, float grad_scale, float lr,
+                           float beta1, float beta2, float eps, int eps_inside_sqrt,
+                           float weight_decay, int step, pe_stream_t stream);
+
+/*
+ * One MicroSignSGD step (Section 3.1: EMA o avg o sign):
+ *     sbar = sum_sign/B;   m = beta*m + (1-beta)*sbar;   theta = theta - lr*m - weight_decay*theta
+ * sum_sign: fp32 [n], the out_stat(sign) of pe_linear_stats.  No bias correction.
+ */
+pe_status_t microsignsgd_step(float* theta, void* theta_lp, float* m, const float* sum_sign,
+                              long long n, int B, float lr, float beta, float weight_decay,
+                              pe_stream_t stream);
+
+/* Human-readable name of a status code (static storage). */
+const char* pe_status_string(pe_status_t status);
+
+/* Synchronises `stream`, then reads and clears the device status word.  Returns PE_OK, PE_ERR_TIMEOUT
+ * (a kernel gave up on a bounded wait; its outputs are invalid), or PE_ERR_CUDA.  If `detail` is not
+ * NULL it receives a host int identifying the wait that expired (0 if none). */
+pe_status_t pe_get_async_status(pe_stream_t stream, int* detail);
+
+/* Process-wide override of the kernel family (for tests and benchmarks). Returns the previous value. */
+int pe_set_path(int path /* pe_path_t */);
+/* The family the most recent pe_linear_stats / pe_token_sqstats call on this thread's process used
+ * (PE_PATH_SIMT or PE_PATH_TENSOR; PE_PATH_AUTO if none yet). */
+int pe_last_path(void);
+/* Number of kernels the library has launched since load (or since the last reset to 0 via
+ * pe_reset_launch_count). */
+long long pe_launch_count(void);
+void pe_reset_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PESTATS_H_ */

@@ -1,0 +1,245 @@
+"""ctypes binding of ``libpestats.so``: same names as the C ABI, argument marshalling only.
+
+Tensors are passed as raw device pointers (``tensor.data_ptr()``) together with the current CUDA
+stream; every computation happens in the library's kernels.  There is no fallback: if the library
+has not been built, or a call returns an error status, a :class:`PestatsError` is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+__all__ = [
+    "PestatsError", "PHI_IDENTITY", "PHI_SQUARE", "PHI_SIGN", "PATH_AUTO", "PATH_SIMT", "PATH_TENSOR",
+    "EXPORTED_SYMBOLS", "library_path", "load_library", "pe_linear_stats", "pe_linear_stats_f32",
+    "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_workspace_bytes", "microadam_step",
+    "microsignsgd_step", "pe_status_string", "pe_get_async_status", "pe_set_path", "pe_last_path",
+    "pe_launch_count", "pe_reset_launch_count",
+]
+
+PHI_IDENTITY, PHI_SQUARE, PHI_SIGN = 0, 1, 2
+PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+_PHI_NAMES = {"identity": PHI_IDENTITY, "square": PHI_SQUARE, "sign": PHI_SIGN}
+
+# every symbol include/pestats.h declares
+EXPORTED_SYMBOLS = [
+    "pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32",
+    "pe_token_sqstats_workspace_bytes", "microadam_step", "microsignsgd_step", "pe_status_string",
+    "pe_get_async_status", "pe_set_path", "pe_last_path", "pe_launch_count", "pe_reset_launch_count",
+]
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libpestats.so")
+_lib = None
+
+
+class PestatsError(RuntimeError):
+    """A libpestats call failed; ``status`` holds the pe_status_t code."""
+
+    def __init__(self, fn: str, status: int, text: str):
+        super().__init__(f"{fn} failed: {text} ({status})")
+        self.status = status
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the in-tree CUDA library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise PestatsError("load_library", -1,
+                           f"{_LIB_PATH} not found; build it with `python -m paper_2510_00236_b200.build`")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i, f, ll, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_longlong, ctypes.c_size_t
+    lib.pe_linear_stats.argtypes = [vp, vp, i, i, i, i, i, vp, vp, vp]
+    lib.pe_linear_stats_f32.argtypes = [vp, vp, i, i, i, i, i, vp, vp, vp]
+    lib.pe_token_sqstats.argtypes = [vp, vp, i, i, i, i, vp, vp, sz, vp]
+    lib.pe_token_sqstats_f32.argtypes = [vp, vp, i, i, i, i, vp, vp]
+    lib.pe_token_sqstats_workspace_bytes.argtypes = [i, i, i, i]
+    lib.pe_token_sqstats_workspace_bytes.restype = sz
+    lib.microadam_step.argtypes = [vp, vp, vp, vp, vp, vp, ll, i, f, f, f, f, f, i, f, i, vp]
+    lib.microsignsgd_step.argtypes = [vp, vp, vp, vp, ll, i, f, f, f, vp]
+    lib.pe_status_string.argtypes = [i]
+    lib.pe_status_string.restype = ctypes.c_char_p
+    lib.pe_get_async_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
+    lib.pe_set_path.argtypes = [i]
+    lib.pe_last_path.argtypes = []
+    lib.pe_launch_count.argtypes = []
+    lib.pe_launch_count.restype = ll
+    lib.pe_reset_launch_count.argtypes = []
+    lib.pe_reset_launch_count.restype = None
+    for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32",
+                 "microadam_step", "microsignsgd_step", "pe_get_async_status", "pe_set_path", "pe_last_path"):
+        getattr(lib, name).restype = i
+    _lib = lib
+    return lib
+
+
+def pe_status_string(status: int) -> str:
+    return load_library().pe_status_string(int(status)).decode()
+
+
+def _check(fn: str, status: int):
+    if status != 0:
+        raise PestatsError(fn, status, pe_status_string(status))
+
+
+def _stream(t: torch.Tensor) -> int:
+    return torch.cuda.current_stream(t.device).cuda_stream
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _phi(phi) -> int:
+    return _PHI_NAMES[phi] if isinstance(phi, str) else int(phi)
+
+
+def _dev_ctx(t: torch.Tensor):
+    if not t.is_cuda:
+        raise PestatsError("binding", -1, "tensors must live on a CUDA device (there is no CPU path)")
+    return torch.cuda.device(t.device)
+
+
+def _io_check(X, dY, dtype):
+    if X.dtype != dtype or dY.dtype != dtype:
+        raise TypeError(f"X and dY must be {dtype}")
+    if X.dim() != 3 or dY.dim() != 3 or X.shape[:2] != dY.shape[:2]:
+        raise ValueError("X must be [B,T,d_in] and dY [B,T,d_out] with equal B and T")
+    if not (X.is_contiguous() and dY.is_contiguous()):
+        raise ValueError("X and dY must be contiguous")
+    B, T, d_in = X.shape
+    return B, T, d_in, dY.shape[2]
+
+
+def _out_check(name, t, d_out, d_in):
+    if t is not None and (t.dtype != torch.float32 or tuple(t.shape) != (d_out, d_in) or not t.is_contiguous()):
+        raise ValueError(f"{name} must be a contiguous float32 [d_out, d_in] tensor")
+
+
+def pe_linear_stats(X, dY, phi, out_mean=None, out_stat=None):
+    """out_mean = sum_b G_b, out_stat = sum_b phi(G_b) with G_b = dY_b^T X_b (bf16 inputs).
+    Buffers are allocated when both are omitted; returns (out_mean, out_stat)."""
+    B, T, d_in, d_out = _io_check(X, dY, torch.bfloat16)
+    if out_mean is None and out_stat is None:
+        out_mean = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)
+        out_stat = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)
+    _out_check("out_mean", out_mean, d_out, d_in)
+    _out_check("out_stat", out_stat, d_out, d_in)
+    with _dev_ctx(X):
+        _check("pe_linear_stats", load_library().pe_linear_stats(
+            X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, _phi(phi), _ptr(out_mean), _ptr(out_stat), _stream(X)))
+    return out_mean, out_stat
+
+
+def pe_linear_stats_f32(X, dY, phi, out_mean=None, out_stat=None):
+    """fp32-input variant of :func:`pe_linear_stats`."""
+    B, T, d_in, d_out = _io_check(X, dY, torch.float32)
+    if out_mean is None and out_stat is None:
+        out_mean = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)
+        out_stat = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)
+    _out_check("out_mean", out_mean, d_out, d_in)
+    _out_check("out_stat", out_stat, d_out, d_in)
+    with _dev_ctx(X):
+        _check("pe_linear_stats_f32", load_library().pe_linear_stats_f32(
+            X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, _phi(phi), _ptr(out_mean), _ptr(out_stat), _stream(X)))
+    return out_mean, out_stat
+
+
+def pe_token_sqstats_workspace_bytes(B, T, d_in, d_out) -> int:
+    return int(load_library().pe_token_sqstats_workspace_bytes(int(B), int(T), int(d_in), int(d_out)))
+
+
+def pe_token_sqstats(X, dY, out_stat=None, workspace=None):
+    """Per-token second moment sum_{b,t} dY^2 X^2 (bf16 inputs).  ``workspace`` is a uint8 CUDA tensor of
+    at least pe_token_sqstats_workspace_bytes(...) bytes; allocated when omitted."""
+    B, T, d_in, d_out = _io_check(X, dY, torch.bfloat16)
+    if out_stat is None:
+        out_stat = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)
+    _out_check("out_stat", out_stat, d_out, d_in)
+    need = pe_token_sqstats_workspace_bytes(B, T, d_in, d_out)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=X.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    with _dev_ctx(X):
+        _check("pe_token_sqstats", load_library().pe_token_sqstats(
+            X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, out_stat.data_ptr(), _ptr(workspace), ws_bytes, _stream(X)))
+    return out_stat
+
+
+def pe_token_sqstats_f32(X, dY, out_stat=None):
+    B, T, d_in, d_out = _io_check(X, dY, torch.float32)
+    if out_stat is None:
+        out_stat = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)
+    _out_check("out_stat", out_stat, d_out, d_in)
+    with _dev_ctx(X):
+        _check("pe_token_sqstats_f32", load_library().pe_token_sqstats_f32(
+            X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, out_stat.data_ptr(), _stream(X)))
+    return out_stat
+
+
+def _flat_f32(name, t, n=None):
+    if t.dtype != torch.float32 or not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous float32")
+    if n is not None and t.numel() != n:
+        raise ValueError(f"{name} has {t.numel()} elements, expected {n}")
+    return t.numel()
+
+
+def microadam_step(theta, m, v, sum_g, sum_g2, B, *, lr, beta1, beta2, eps, step, grad_scale=1.0,
+                   eps_inside_sqrt=False, weight_decay=0.0, theta_lp=None):
+    """In-place MicroAdam update of (theta, m, v) from sum_b G_b and sum_b G_b^2."""
+    n = _flat_f32("theta", theta)
+    for name, t in (("m", m), ("v", v), ("sum_g", sum_g), ("sum_g2", sum_g2)):
+        _flat_f32(name, t, n)
+    if theta_lp is not None and (theta_lp.dtype != torch.bfloat16 or theta_lp.numel() != n or not theta_lp.is_contiguous()):
+        raise ValueError("theta_lp must be contiguous bfloat16 with theta's element count")
+    with _dev_ctx(theta):
+        _check("microadam_step", load_library().microadam_step(
+            theta.data_ptr(), _ptr(theta_lp), m.data_ptr(), v.data_ptr(), sum_g.data_ptr(), sum_g2.data_ptr(), n, int(B),
+            float(grad_scale), float(lr), float(beta1), float(beta2), float(eps), int(bool(eps_inside_sqrt)),
+            float(weight_decay), int(step), _stream(theta)))
+
+
+def microsignsgd_step(theta, m, sum_sign, B, *, lr, beta, weight_decay=0.0, theta_lp=None):
+    """In-place MicroSignSGD update of (theta, m) from sum_b sign(G_b)."""
+    n = _flat_f32("theta", theta)
+    _flat_f32("m", m, n)
+    _flat_f32("sum_sign", sum_sign, n)
+    if theta_lp is not None and (theta_lp.dtype != torch.bfloat16 or theta_lp.numel() != n or not theta_lp.is_contiguous()):
+        raise ValueError("theta_lp must be contiguous bfloat16 with theta's element count")
+    with _dev_ctx(theta):
+        _check("microsignsgd_step", load_library().microsignsgd_step(
+            theta.data_ptr(), _ptr(theta_lp), m.data_ptr(), sum_sign.data_ptr(), n, int(B), float(lr), float(beta),
+            float(weight_decay), _stream(theta)))
+
+
+def pe_get_async_status(device=None):
+    """Synchronises the current stream of ``device``; returns (status, detail). status 0 = OK."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    detail = ctypes.c_int(0)
+    with torch.cuda.device(dev):
+        st = load_library().pe_get_async_status(torch.cuda.current_stream(dev).cuda_stream, ctypes.byref(detail))
+    return int(st), int(detail.value)
+
+
+def pe_set_path(path: int) -> int:
+    return int(load_library().pe_set_path(int(path)))
+
+
+def pe_last_path() -> int:
+    return int(load_library().pe_last_path())
+
+
+def pe_launch_count() -> int:
+    return int(load_library().pe_launch_count())
+
+
+def pe_reset_launch_count() -> None:
+    load_library().pe_reset_launch_count()

@@ -1,0 +1,391 @@
+// C-ABI entry points of libpestats: argument validation, path selection, tensor-map creation and
+// kernel launches.  Everything that computes runs in the CUDA kernels included below.
+#include <atomic>
+#include <cstdint>
+#include <cstdlib>
+#include <cstring>
+#include <cmath>
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "../../include/pestats.h"
+#include "pe_optim.cuh"
+#include "pe_simt.cuh"
+#include "pe_tc.cuh"
+
+namespace pe {
+
+__device__ unsigned int g_dev_status = 0;   // first device-side wait that gave up (0 = none)
+
+static std::atomic<int> g_path{PE_PATH_AUTO};
+static std::atomic<int> g_last_path{PE_PATH_AUTO};
+static std::atomic<long long> g_launches{0};
+
+constexpr int MAX_DEVICES = 64;
+struct DeviceInfo {
+  std::atomic<int> state{0};     // 0 unknown, 1 ready, -1 failed
+  int cc_major = 0, sm_count = 0;
+  unsigned int* status_ptr = nullptr;
+  bool tc_attr_set[3] = {false, false, false};
+};
+static DeviceInfo g_dev[MAX_DEVICES];
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static std::atomic<EncodeTiledFn> g_encode{nullptr};
+
+static pe_status_t device_info(DeviceInfo** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) { cudaGetLastError(); return PE_ERR_CUDA; }
+  DeviceInfo& d = g_dev[dev];
+  if (d.state.load() == 0) {
+    int major = 0, sms = 0;
+    void* sp = nullptr;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      cudaGetLastError();
+      return PE_ERR_CUDA;
+    }
+    d.cc_major = major;
+    d.sm_count = sms;
+    if (major == 10) {
+      if (cudaGetSymbolAddress(&sp, g_dev_status) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
+      d.status_ptr = static_cast<unsigned int*>(sp);
+    }
+    d.state.store(1);
+  }
+  *out = &d;
+  return d.cc_major == 10 ? PE_OK : PE_ERR_ARCH;
+}
+
+static EncodeTiledFn encode_fn() {
+  EncodeTiledFn f = g_encode.load();
+  if (f) return f;
+  void* sym = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+      q != cudaDriverEntryPointSuccess || !sym) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  f = reinterpret_cast<EncodeTiledFn>(sym);
+  g_encode.store(f);
+  return f;
+}
+
+static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+static pe_status_t check_launch() {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return PE_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return PE_OK;
+}
+
+// bf16 [B, T, d] row-major viewed as a 3-D tensor (d, T, B); one box = 64 features x TC_BK tokens of
+// one example, 128-byte swizzled.  Tokens past T and features past d read as zero.
+static pe_status_t make_operand_map(CUtensorMap* m, const void* base, int B, int T, int d) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return PE_ERR_CUDA;
+  cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)T, (cuuint64_t)B};
+  cuuint64_t strides[2] = {(cuuint64_t)d * 2ull, (cuuint64_t)T * (cuuint64_t)d * 2ull};
+  cuuint32_t box[3] = {64u, (cuuint32_t)TC_BK, 1u};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? PE_OK : PE_ERR_CUDA;
+}
+
+static bool tc_shape_ok(int B, int T, int d_in, int d_out) {
+  if (B < 1 || T < 1) return false;
+  if ((d_in % 8) || (d_out % 8)) return false;                        // 16-byte row pitch for TMA
+  if ((long long)T * (d_in > d_out ? d_in : d_out) * 2ll >= (1ll << 40)) return false;   // TMA stride limit
+  return true;
+}
+
+// Batch slices per tile: minimise (waves of thread blocks) x (examples per slice) plus a flush term.
+static int choose_nsplit(long long tiles, int B, int T, int slots, int max_split) {
+  int best = 1;
+  double best_cost = 1e300;
+  int tt = T < 32 ? 32 : T;
+  for (int ns = 1; ns <= max_split && ns <= B; ++ns) {
+    long long waves = (tiles * ns + slots - 1) / slots;
+    long long per = ((long long)B + ns - 1) / ns;
+    double cost = (double)waves * ((double)per * tt + (ns > 1 ? 512.0 : 128.0));
+    if (cost < best_cost * 0.999) { best_cost = cost; best = ns; }
+  }
+  return best;
+}
+
+static pe_status_t zero_outputs(float* a, float* b, size_t bytes, cudaStream_t st) {
+  if (a && cudaMemsetAsync(a, 0, bytes, st) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
+  if (b && cudaMemsetAsync(b, 0, bytes, st) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
+  return PE_OK;
+}
+
+template <int PHI>
+static pe_status_t launch_tc_inst(DeviceInfo* di, const CUtensorMap& mx, const CUtensorMap& my, const TcParams& p,
+                                  dim3 grid, cudaStream_t st) {
+  if (!di->tc_attr_set[PHI]) {
+    if (cudaFuncSetAttribute(tc_stats_kernel<PHI>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES) != cudaSuccess) {
+      cudaGetLastError();
+      return PE_ERR_CUDA;
+    }
+    di->tc_attr_set[PHI] = true;
+  }
+  tc_stats_kernel<PHI><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(mx, my, p);
+  return check_launch();
+}
+
+// Tensor-core launch.  per_example = 0 runs the plain contraction over all B*T rows.
+static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int B, int T, int d_in, int d_out, int phi,
+                             int per_example, float* out_mean, float* out_stat, cudaStream_t st) {
+  CUtensorMap mx, my;
+  pe_status_t rc = make_operand_map(&mx, X, B, T, d_in);
+  if (rc != PE_OK) return rc;
+  rc = make_operand_map(&my, dY, B, T, d_out);
+  if (rc != PE_OK) return rc;
+  const int tiles_n = (d_in + TC_TILE_N - 1) / TC_TILE_N, tiles_m = (d_out + TC_TILE_M - 1) / TC_TILE_M;
+  if (tiles_m > 65535) return PE_ERR_DIM;
+  const int ns = choose_nsplit((long long)tiles_n * tiles_m, B, T, di->sm_count, 16);
+  if (ns > 1) {
+    rc = zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
+    if (rc != PE_OK) return rc;
+  }
+  TcParams p;
+  p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = per_example;
+  p.out_mean = out_mean; p.out_stat = out_stat; p.dev_status = di->status_ptr;
+  dim3 grid(tiles_n, tiles_m, ns);
+  if (!per_example || phi == PE_PHI_IDENTITY) return launch_tc_inst<0>(di, mx, my, p, grid, st);
+  if (phi == PE_PHI_SQUARE) return launch_tc_inst<1>(di, mx, my, p, grid, st);
+  return launch_tc_inst<2>(di, mx, my, p, grid, st);
+}
+
+template <typename TIn, int MODE>
+static pe_status_t launch_simt(DeviceInfo* di, const TIn* X, const TIn* dY, int B, int T, int d_in, int d_out, int phi,
+                               float* out_mean, float* out_stat, cudaStream_t st) {
+  const int tx = (d_in + SIMT_TILE - 1) / SIMT_TILE, ty = (d_out + SIMT_TILE - 1) / SIMT_TILE;
+  if (ty > 65535) return PE_ERR_DIM;
+  const int ns = choose_nsplit((long long)tx * ty, B, T, di->sm_count * 3, 64);
+  if (ns > 1) {
+    pe_status_t rc = zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
+    if (rc != PE_OK) return rc;
+  }
+  simt_stats_kernel<TIn, MODE><<<dim3(tx, ty, ns), SIMT_THREADS, 0, st>>>(X, dY, B, T, d_in, d_out, phi, out_mean, out_stat);
+  return check_launch();
+}
+
+static pe_status_t validate_stats(const void* X, const void* dY, int B, int T, int d_in, int d_out, const float* o1,
+                                  const float* o2, bool need_both_null_check, size_t in_align) {
+  if (B < 0 || T < 0 || d_in < 1 || d_out < 1) return PE_ERR_DIM;
+  if ((!X || !dY) && B > 0 && T > 0) return PE_ERR_NULL;      // empty inputs may be NULL
+  if (need_both_null_check && !o1 && !o2) return PE_ERR_NULL;
+  if ((long long)B * T * (long long)(d_in > d_out ? d_in : d_out) >= (1ll << 40)) return PE_ERR_DIM;
+  if ((long long)d_in * d_out >= (1ll << 40)) return PE_ERR_DIM;
+  if (!aligned(X, in_align) || !aligned(dY, in_align)) return PE_ERR_ALIGN;
+  if ((o1 && !aligned(o1, 16)) || (o2 && !aligned(o2, 16))) return PE_ERR_ALIGN;
+  return PE_OK;
+}
+
+template <typename TIn>
+static pe_status_t linear_stats_impl(const TIn* X, const TIn* dY, int B, int T, int d_in, int d_out, pe_phi_t phi,
+                                     float* out_mean, float* out_stat, cudaStream_t st, bool allow_tc) {
+  pe_status_t rc = validate_stats(X, dY, B, T, d_in, d_out, out_mean, out_stat, true, allow_tc ? 16 : 4);
+  if (rc != PE_OK) return rc;
+  if (phi != PE_PHI_IDENTITY && phi != PE_PHI_SQUARE && phi != PE_PHI_SIGN) return PE_ERR_PHI;
+  DeviceInfo* di = nullptr;
+  rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  if (B == 0 || T == 0) return zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
+  const int forced = g_path.load();
+  const bool tc_ok = allow_tc && tc_shape_ok(B, T, d_in, d_out);
+  if (forced == PE_PATH_TENSOR && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
+  if (tc_ok && forced != PE_PATH_SIMT) {
+    if constexpr (sizeof(TIn) == 2) {
+      g_last_path.store(PE_PATH_TENSOR);
+      if (phi == PE_PHI_IDENTITY) {
+        // phi = identity: both outputs are the plain contraction over all B*T rows.
+        float* first = out_mean ? out_mean : out_stat;
+        rc = launch_tc(di, X, dY, B, T, d_in, d_out, phi, 0, first, nullptr, st);
+        if (rc == PE_OK && out_mean && out_stat) {
+          if (cudaMemcpyAsync(out_stat, out_mean, (size_t)d_in * d_out * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
+            cudaGetLastError();
+            return PE_ERR_CUDA;
+          }
+        }
+        return rc;
+      }
+      return launch_tc(di, X, dY, B, T, d_in, d_out, phi, 1, out_mean, out_stat, st);
+    }
+  }
+  g_last_path.store(PE_PATH_SIMT);
+  return launch_simt<TIn, MODE_STATS>(di, X, dY, B, T, d_in, d_out, (int)phi, out_mean, out_stat, st);
+}
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static int grid_for(long long work_items, int sm_count) {
+  long long blocks = (work_items + OPT_THREADS - 1) / OPT_THREADS;
+  long long cap = (long long)sm_count * 8;
+  if (blocks < 1) blocks = 1;
+  return (int)(blocks < cap ? blocks : cap);
+}
+
+}  // namespace pe
+
+using namespace pe;
+
+extern "C" {
+
+pe_status_t pe_linear_stats(const void* X, const void* dY, int B, int T, int d_in, int d_out, pe_phi_t phi,
+                            float* out_mean, float* out_stat, pe_stream_t stream) {
+  return linear_stats_impl<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T,
+                                          d_in, d_out, phi, out_mean, out_stat, reinterpret_cast<cudaStream_t>(stream), true);
+}
+
+pe_status_t pe_linear_stats_f32(const float* X, const float* dY, int B, int T, int d_in, int d_out, pe_phi_t phi,
+                                float* out_mean, float* out_stat, pe_stream_t stream) {
+  return linear_stats_impl<float>(X, dY, B, T, d_in, d_out, phi, out_mean, out_stat, reinterpret_cast<cudaStream_t>(stream), false);
+}
+
+size_t pe_token_sqstats_workspace_bytes(int B, int T, int d_in, int d_out) {
+  if (g_path.load() == PE_PATH_SIMT || !tc_shape_ok(B, T, d_in, d_out)) return 0;
+  const size_t rows = (size_t)B * (size_t)T;
+  return align_up(rows * d_in * 2, 256) + align_up(rows * d_out * 2, 256);
+}
+
+pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_stat,
+                             void* workspace, size_t workspace_bytes, pe_stream_t stream) {
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (!out_stat) return PE_ERR_NULL;
+  pe_status_t rc = validate_stats(X, dY, B, T, d_in, d_out, out_stat, nullptr, false, 16);
+  if (rc != PE_OK) return rc;
+  DeviceInfo* di = nullptr;
+  rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  if (B == 0 || T == 0) return zero_outputs(out_stat, nullptr, (size_t)d_in * d_out * sizeof(float), st);
+  const int forced = g_path.load();
+  const bool tc_ok = tc_shape_ok(B, T, d_in, d_out);
+  if (forced == PE_PATH_TENSOR && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
+  if (tc_ok && forced != PE_PATH_SIMT) {
+    const size_t rows = (size_t)B * (size_t)T;
+    const size_t x_bytes = align_up(rows * d_in * 2, 256), y_bytes = align_up(rows * d_out * 2, 256);
+    if (!workspace || workspace_bytes < x_bytes + y_bytes) return PE_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return PE_ERR_ALIGN;
+    __nv_bfloat16* x2 = static_cast<__nv_bfloat16*>(workspace);
+    __nv_bfloat16* y2 = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + x_bytes);
+    const long long nx = (long long)rows * d_in, ny = (long long)rows * d_out;
+    square_bf16_kernel<<<grid_for(nx / 8 + 8, di->sm_count), OPT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(X), x2, nx);
+    if ((rc = check_launch()) != PE_OK) return rc;
+    square_bf16_kernel<<<grid_for(ny / 8 + 8, di->sm_count), OPT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(dY), y2, ny);
+    if ((rc = check_launch()) != PE_OK) return rc;
+    // B and T only enter through B*T: regroup the rows into 64-token "examples" when possible so
+    // the batch split has many units to balance.
+    int Bp = B, Tp = T;
+    if (T % TC_BK == 0 && rows / TC_BK < (size_t)(1u << 30)) { Bp = (int)(rows / TC_BK); Tp = TC_BK; }
+    g_last_path.store(PE_PATH_TENSOR);
+    return launch_tc(di, x2, y2, Bp, Tp, d_in, d_out, PE_PHI_IDENTITY, 0, nullptr, out_stat, st);
+  }
+  g_last_path.store(PE_PATH_SIMT);
+  return launch_simt<__nv_bfloat16, MODE_TOKEN>(di, static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T,
+                                                d_in, d_out, 0, nullptr, out_stat, st);
+}
+
+pe_status_t pe_token_sqstats_f32(const float* X, const float* dY, int B, int T, int d_in, int d_out, float* out_stat,
+                                 pe_stream_t stream) {
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (!out_stat) return PE_ERR_NULL;
+  pe_status_t rc = validate_stats(X, dY, B, T, d_in, d_out, out_stat, nullptr, false, 4);
+  if (rc != PE_OK) return rc;
+  DeviceInfo* di = nullptr;
+  rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  if (B == 0 || T == 0) return zero_outputs(out_stat, nullptr, (size_t)d_in * d_out * sizeof(float), st);
+  g_last_path.store(PE_PATH_SIMT);
+  return launch_simt<float, MODE_TOKEN>(di, X, dY, B, T, d_in, d_out, 0, nullptr, out_stat, st);
+}
+
+pe_status_t microadam_step(float* theta, void* theta_lp, float* m, float* v, const float* sum_g, const float* sum_g2,
+                           long long n, int B, float grad_scale, float lr, float beta1, float beta2, float eps,
+                           int eps_inside_sqrt, float weight_decay, int step, pe_stream_t stream) {
+  if (!theta || !m || !v || !sum_g || !sum_g2) return PE_ERR_NULL;
+  if (n < 0 || B < 1 || step < 1) return PE_ERR_DIM;
+  if (!aligned(theta, 16) || !aligned(m, 16) || !aligned(v, 16) || !aligned(sum_g, 16) || !aligned(sum_g2, 16) ||
+      (theta_lp && !aligned(theta_lp, 16)))
+    return PE_ERR_ALIGN;
+  DeviceInfo* di = nullptr;
+  pe_status_t rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  if (n == 0) return PE_OK;
+  AdamParams p;
+  p.mu_scale = (float)((double)grad_scale / (double)B);
+  p.nu_scale = (float)((double)grad_scale * (double)grad_scale / (double)B);
+  p.beta1 = beta1; p.beta2 = beta2;
+  p.inv_c1 = (float)(1.0 / (1.0 - std::pow((double)beta1, (double)step)));
+  p.inv_c2 = (float)(1.0 / (1.0 - std::pow((double)beta2, (double)step)));
+  p.eps = eps; p.lr = lr; p.wd = weight_decay; p.eps_inside = eps_inside_sqrt ? 1 : 0;
+  microadam_kernel<<<grid_for(n / 4 + 4, di->sm_count), OPT_THREADS, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      theta, static_cast<__nv_bfloat16*>(theta_lp), m, v, sum_g, sum_g2, n, p);
+  return check_launch();
+}
+
+pe_status_t microsignsgd_step(float* theta, void* theta_lp, float* m, const float* sum_sign, long long n, int B, float lr,
+                              float beta, float weight_decay, pe_stream_t stream) {
+  if (!theta || !m || !sum_sign) return PE_ERR_NULL;
+  if (n < 0 || B < 1) return PE_ERR_DIM;
+  if (!aligned(theta, 16) || !aligned(m, 16) || !aligned(sum_sign, 16) || (theta_lp && !aligned(theta_lp, 16))) return PE_ERR_ALIGN;
+  DeviceInfo* di = nullptr;
+  pe_status_t rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  if (n == 0) return PE_OK;
+  SignParams p;
+  p.inv_B = (float)(1.0 / (double)B); p.beta = beta; p.lr = lr; p.wd = weight_decay;
+  microsignsgd_kernel<<<grid_for(n / 4 + 4, di->sm_count), OPT_THREADS, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      theta, static_cast<__nv_bfloat16*>(theta_lp), m, sum_sign, n, p);
+  return check_launch();
+}
+
+const char* pe_status_string(pe_status_t s) {
+  switch (s) {
+    case PE_OK: return "PE_OK";
+    case PE_ERR_NULL: return "PE_ERR_NULL";
+    case PE_ERR_DIM: return "PE_ERR_DIM";
+    case PE_ERR_ALIGN: return "PE_ERR_ALIGN";
+    case PE_ERR_UNSUPPORTED_SHAPE: return "PE_ERR_UNSUPPORTED_SHAPE";
+    case PE_ERR_PHI: return "PE_ERR_PHI";
+    case PE_ERR_ARCH: return "PE_ERR_ARCH";
+    case PE_ERR_CUDA: return "PE_ERR_CUDA";
+    case PE_ERR_TIMEOUT: return "PE_ERR_TIMEOUT";
+    case PE_ERR_WORKSPACE: return "PE_ERR_WORKSPACE";
+  }
+  return "PE_ERR_UNKNOWN";
+}
+
+pe_status_t pe_get_async_status(pe_stream_t stream, int* detail) {
+  if (detail) *detail = 0;
+  DeviceInfo* di = nullptr;
+  pe_status_t rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
+  unsigned int word = 0;
+  if (cudaMemcpy(&word, di->status_ptr, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
+  if (word == 0) return PE_OK;
+  if (cudaMemset(di->status_ptr, 0, sizeof word) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
+  if (detail) *detail = (int)word;
+  return PE_ERR_TIMEOUT;
+}
+
+int pe_set_path(int path) {
+  if (path < PE_PATH_AUTO || path > PE_PATH_TENSOR) return -1;
+  return g_path.exchange(path);
+}
+int pe_last_path(void) { return g_last_path.load(); }
+long long pe_launch_count(void) { return g_launches.load(); }
+void pe_reset_launch_count(void) { g_launches.store(0); }
+
+}  // extern "C"

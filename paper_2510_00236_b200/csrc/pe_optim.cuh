@@ -1,0 +1,141 @@
+// Fused elementwise parameter updates that consume the per-example statistics.  Pure streaming
+// kernels: every operand is read once and every result written once with 128-bit accesses, so the
+// bound is HBM bandwidth (MicroAdam 32 B/parameter, MicroSignSGD 20 B/parameter, +2 B with the
+// bf16 weight copy).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+namespace pe {
+
+struct AdamParams {
+  float mu_scale;    // s / B
+  float nu_scale;    // s^2 / B
+  float beta1, beta2;
+  float inv_c1, inv_c2;   // 1/(1-beta1^t), 1/(1-beta2^t)
+  float eps, lr, wd;
+  int eps_inside;
+};
+
+// Algorithm 1, MicroAdam branch, for one parameter.
+__device__ __forceinline__ void adam_one(float& th, float& m, float& v, float sg, float sg2, const AdamParams& p) {
+  float mu = sg * p.mu_scale;
+  float nu = sg2 * p.nu_scale;
+  m = fmaf(p.beta1, m, (1.f - p.beta1) * mu);
+  v = fmaf(p.beta2, v, (1.f - p.beta2) * nu);
+  float mh = m * p.inv_c1;
+  float vh = v * p.inv_c2;
+  float u = p.eps_inside ? mh / sqrtf(p.eps + vh) : mh / (sqrtf(vh) + p.eps);
+  th = th - p.lr * u - p.wd * th;
+}
+
+__device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
+
+constexpr int OPT_THREADS = 256;
+
+__global__ void __launch_bounds__(OPT_THREADS)
+microadam_kernel(float* __restrict__ theta, __nv_bfloat16* __restrict__ theta_lp, float* __restrict__ m,
+                 float* __restrict__ v, const float* __restrict__ sum_g, const float* __restrict__ sum_g2,
+                 long long n, AdamParams p) {
+  const long long n4 = n >> 2;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x; k < n4; k += stride) {
+    float4 th = reinterpret_cast<float4*>(theta)[k];
+    float4 mm = reinterpret_cast<float4*>(m)[k];
+    float4 vv = reinterpret_cast<float4*>(v)[k];
+    float4 g = ld_stream(reinterpret_cast<const float4*>(sum_g) + k);
+    float4 g2 = ld_stream(reinterpret_cast<const float4*>(sum_g2) + k);
+    adam_one(th.x, mm.x, vv.x, g.x, g2.x, p);
+    adam_one(th.y, mm.y, vv.y, g.y, g2.y, p);
+    adam_one(th.z, mm.z, vv.z, g.z, g2.z, p);
+    adam_one(th.w, mm.w, vv.w, g.w, g2.w, p);
+    reinterpret_cast<float4*>(theta)[k] = th;
+    reinterpret_cast<float4*>(m)[k] = mm;
+    reinterpret_cast<float4*>(v)[k] = vv;
+    if (theta_lp) {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(th.x, th.y);
+      __nv_bfloat162 hi = __floats2bfloat162_rn(th.z, th.w);
+      uint2 pk;
+      pk.x = *reinterpret_cast<unsigned int*>(&lo);
+      pk.y = *reinterpret_cast<unsigned int*>(&hi);
+      reinterpret_cast<uint2*>(theta_lp)[k] = pk;
+    }
+  }
+  // ragged tail (n % 4 elements)
+  long long k = (n4 << 2) + (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (k < n) {
+    float th = theta[k], mm = m[k], vv = v[k];
+    adam_one(th, mm, vv, sum_g[k], sum_g2[k], p);
+    theta[k] = th; m[k] = mm; v[k] = vv;
+    if (theta_lp) theta_lp[k] = __float2bfloat16_rn(th);
+  }
+}
+
+struct SignParams {
+  float inv_B, beta, lr, wd;
+};
+
+// Section 3.1, MicroSignSGD = EMA o avg o sign, for one parameter.
+__device__ __forceinline__ void sign_one(float& th, float& m, float ss, const SignParams& p) {
+  float sbar = ss * p.inv_B;
+  m = fmaf(p.beta, m, (1.f - p.beta) * sbar);
+  th = th - p.lr * m - p.wd * th;
+}
+
+__global__ void __launch_bounds__(OPT_THREADS)
+microsignsgd_kernel(float* __restrict__ theta, __nv_bfloat16* __restrict__ theta_lp, float* __restrict__ m,
+                    const float* __restrict__ sum_sign, long long n, SignParams p) {
+  const long long n4 = n >> 2;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x; k < n4; k += stride) {
+    float4 th = reinterpret_cast<float4*>(theta)[k];
+    float4 mm = reinterpret_cast<float4*>(m)[k];
+    float4 s = ld_stream(reinterpret_cast<const float4*>(sum_sign) + k);
+    sign_one(th.x, mm.x, s.x, p);
+    sign_one(th.y, mm.y, s.y, p);
+    sign_one(th.z, mm.z, s.z, p);
+    sign_one(th.w, mm.w, s.w, p);
+    reinterpret_cast<float4*>(theta)[k] = th;
+    reinterpret_cast<float4*>(m)[k] = mm;
+    if (theta_lp) {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(th.x, th.y);
+      __nv_bfloat162 hi = __floats2bfloat162_rn(th.z, th.w);
+      uint2 pk;
+      pk.x = *reinterpret_cast<unsigned int*>(&lo);
+      pk.y = *reinterpret_cast<unsigned int*>(&hi);
+      reinterpret_cast<uint2*>(theta_lp)[k] = pk;
+    }
+  }
+  long long k = (n4 << 2) + (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (k < n) {
+    float th = theta[k], mm = m[k];
+    sign_one(th, mm, sum_sign[k], p);
+    theta[k] = th; m[k] = mm;
+    if (theta_lp) theta_lp[k] = __float2bfloat16_rn(th);
+  }
+}
+
+// Elementwise square of a bf16 array, rounded back to bf16 (operand staging for the tensor-core
+// per-token statistic).  n8 = number of 8-element (16-byte) groups; tail handled by the last threads.
+__global__ void __launch_bounds__(OPT_THREADS)
+square_bf16_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, long long n) {
+  const long long n8 = n >> 3;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x; k < n8; k += stride) {
+    uint4 raw = __ldcs(reinterpret_cast<const uint4*>(src) + k);
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float2 f = __bfloat1622float2(h[j]);
+      h[j] = __floats2bfloat162_rn(f.x * f.x, f.y * f.y);
+    }
+    reinterpret_cast<uint4*>(dst)[k] = raw;
+  }
+  long long k = (n8 << 3) + (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (k < n) {
+    float f = __bfloat162float(src[k]);
+    dst[k] = __float2bfloat16_rn(f * f);
+  }
+}
+
+}  // namespace pe

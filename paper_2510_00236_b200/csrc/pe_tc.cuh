@@ -1,0 +1,237 @@
+// Tensor-core kernel for the sequence-level per-example statistics (Section 2.3; Eq. (2)).
+//
+// One thread block owns a 128 x 128 tile of the [d_out, d_in] output and a contiguous slice of the
+// batch.  For every example of the slice the tile of G_b = dY_b^T X_b is formed by tcgen05 MMAs
+// (bf16 operands staged by TMA in 128-byte-swizzled shared memory, fp32 accumulator in tensor
+// memory), read back by the epilogue warps, passed through phi and added to two register-resident
+// running sums (sum_b phi(G_b) and sum_b G_b).  The per-example tile never leaves the SM.
+//
+// Warp roles (12 warps):  0 = TMA producer, 1 = MMA issuer, 2 = TMEM allocator, 3 = idle,
+// 4..11 = epilogue (warp w reads TMEM lanes 32*(w%4)..+31, columns 64*((w-4)/4)..+63 of the tile).
+// The tensor-memory accumulator is ring-buffered (4 x 128 columns) so the MMAs of example b+1..b+3
+// overlap the epilogue of example b.
+//
+// Operand orientation: A = dY_b viewed as M = d_out x K = T and B = X_b viewed as N = d_in x K = T.
+// In global memory the contraction index (the token) is the slow one, so both operands are
+// "MN-major".  A TMA box is 64 features (128 bytes) x BK tokens; with the 128-byte swizzle that is
+// exactly the canonical MN-major layout of the MMA: 8-token x 64-feature atoms of 1 KiB, the next
+// 8 tokens 1 KiB further (stride byte offset), the next 64 features one box further (leading byte
+// offset).
+#pragma once
+#include "pe_sm100.cuh"
+
+namespace pe {
+
+constexpr int TC_TILE_M = 128;    // d_out rows per tile   (MMA M)
+constexpr int TC_TILE_N = 128;    // d_in columns per tile (MMA N)
+constexpr int TC_BK = 64;         // tokens per pipeline stage
+constexpr int TC_STAGES = 6;
+constexpr int TC_ACC_BUFS = 4;    // TMEM accumulator ring
+constexpr int TC_TMEM_COLS = TC_ACC_BUFS * TC_TILE_N;   // 512
+constexpr int TC_THREADS = 384;
+constexpr int TC_REGS_CONTROL = 64;     // setmaxnreg of warps 0..3
+constexpr int TC_REGS_EPILOGUE = 216;   // setmaxnreg of warps 4..11  (4*32*64 + 8*32*216 = 63488 <= 65536)
+constexpr int TC_BOX_BYTES = 64 * TC_BK * 2;                              // one 64-feature x BK-token box
+constexpr int TC_A_BYTES = (TC_TILE_M / 64) * TC_BOX_BYTES;               // 16 KiB
+constexpr int TC_B_BYTES = (TC_TILE_N / 64) * TC_BOX_BYTES;               // 16 KiB
+constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;                   // 32 KiB
+constexpr int TC_BAR_BYTES = 256;
+constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + TC_BAR_BYTES + 1024;   // + alignment slack
+
+// error codes latched in the device status word (which wait gave up)
+enum : int { TC_WAIT_EMPTY = 1, TC_WAIT_FULL = 2, TC_WAIT_ACC_EMPTY = 3, TC_WAIT_ACC_FULL = 4 };
+
+struct TcParams {
+  int B, T, d_in, d_out;
+  int nsplit;          // batch slices (gridDim.z); > 1 => outputs pre-zeroed, partials added atomically
+  int per_example;     // 1: reset the accumulator for every example and apply phi (statistics)
+                       // 0: one accumulation over the whole slice (plain contraction, phi = identity)
+  float* out_mean;     // may be NULL
+  float* out_stat;     // may be NULL
+  unsigned int* dev_status;
+};
+
+template <int PHI>
+__device__ __forceinline__ float phi_apply(float g) {
+  if (PHI == 1) return g * g;
+  if (PHI == 2) {
+    // sign(g) with sign(+-0) = 0: copy the sign bit onto 1.0f, then zero it when g == 0.
+    float s = __uint_as_float((__float_as_uint(g) & 0x80000000u) | 0x3f800000u);
+    return g != 0.f ? s : 0.f;
+  }
+  return g;
+}
+
+template <int PHI>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy, TcParams p) {
+  using namespace sm100;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + TC_STAGES * TC_STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (TC_STAGES + s); };
+  auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * TC_STAGES + a); };
+  auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * TC_STAGES + TC_ACC_BUFS + a); };
+  uint8_t* tail = smem_gen + TC_STAGES * TC_STAGE_BYTES + 8 * (2 * TC_STAGES + 2 * TC_ACC_BUFS);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile_n = blockIdx.x, tile_m = blockIdx.y;
+  const int b_begin = (int)(((long long)p.B * blockIdx.z) / p.nsplit);
+  const int b_end = (int)(((long long)p.B * (blockIdx.z + 1)) / p.nsplit);
+  const int nb = b_end - b_begin;
+  const int nk = (p.T + TC_BK - 1) / TC_BK;                 // stages per example
+  const int n_groups = p.per_example ? nb : (nb > 0 ? 1 : 0);
+  const int group_len = p.per_example ? 1 : nb;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < TC_ACC_BUFS; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 8); }
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 0 && lane == 0) { prefetch_tensormap(&tmap_x); prefetch_tensormap(&tmap_dy); }
+  if (warp == 2) { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TC_TMEM_COLS); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // Register budget: the epilogue warpgroups hold two 64-float running sums plus a 32-register TMEM
+  // read per thread; the producer / MMA warpgroup needs little.  Each setmaxnreg sits inside the
+  // branch of the role it applies to.
+  if (warp < 4) {
+    setmaxnreg_dec<TC_REGS_CONTROL>();
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int s = 0; uint32_t ph = 0;
+      bool ok = true;
+      for (int e = 0; e < nb && ok; ++e) {
+        const int b = b_begin + e;
+        for (int kc = 0; kc < nk; ++kc) {
+          if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_EMPTY)) { ok = false; break; }
+          mbar_arrive_expect_tx(full_bar(s), TC_STAGE_BYTES);
+          const uint32_t a_dst = smem_base + s * TC_STAGE_BYTES;
+          const uint32_t b_dst = a_dst + TC_A_BYTES;
+#pragma unroll
+          for (int g = 0; g < TC_TILE_M / 64; ++g)
+            tma_load_3d(a_dst + g * TC_BOX_BYTES, &tmap_dy, full_bar(s), tile_m * TC_TILE_M + g * 64, kc * TC_BK, b);
+#pragma unroll
+          for (int g = 0; g < TC_TILE_N / 64; ++g)
+            tma_load_3d(b_dst + g * TC_BOX_BYTES, &tmap_x, full_bar(s), tile_n * TC_TILE_N + g * 64, kc * TC_BK, b);
+          if (++s == TC_STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16_mn_major(TC_TILE_M, TC_TILE_N);
+      int s = 0; uint32_t ph = 0;
+      bool ok = true;
+      for (int grp = 0; grp < n_groups && ok; ++grp) {
+        const int buf = grp % TC_ACC_BUFS;
+        const uint32_t acc_ph = (uint32_t)(grp / TC_ACC_BUFS) & 1u;
+        if (!mbar_wait_bounded(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_ACC_EMPTY)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * TC_TILE_N);
+        uint32_t accumulate = 0;
+        for (int e = 0; e < group_len && ok; ++e) {
+          for (int kc = 0; kc < nk; ++kc) {
+            if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, p.dev_status, TC_WAIT_FULL)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a_src = smem_base + s * TC_STAGE_BYTES;
+            const uint32_t b_src = a_src + TC_A_BYTES;
+            const int t_left = p.T - kc * TC_BK;               // tokens of this example still to contract
+#pragma unroll
+            for (int k = 0; k < TC_BK / 16; ++k) {
+              if (k * 16 < t_left) {                             // rows past T are zero-filled by TMA; whole
+                const uint64_t ad = make_smem_desc_sw128(a_src + k * 2048, TC_BOX_BYTES, 1024);   // 16-token steps past T are skipped
+                const uint64_t bd = make_smem_desc_sw128(b_src + k * 2048, TC_BOX_BYTES, 1024);
+                umma_bf16_ss(d_tmem, ad, bd, idesc, accumulate);
+                accumulate = 1;
+              }
+            }
+            umma_commit(empty_bar(s));                           // stage reusable once these MMAs retire
+            if (++s == TC_STAGES) { s = 0; ph ^= 1u; }
+          }
+        }
+        if (ok) umma_commit(acc_full_bar(buf));                  // accumulator of this example complete
+      }
+    }
+  }
+  } else {
+    // ------------------------------------------------------------ epilogue
+    setmaxnreg_inc<TC_REGS_EPILOGUE>();
+    const int q = warp & 3;                 // TMEM lane quadrant this warp may access
+    const int h = (warp - 4) >> 2;          // column half of the tile
+    float acc_stat[64], acc_mean[64];
+#pragma unroll
+    for (int j = 0; j < 64; ++j) { acc_stat[j] = 0.f; acc_mean[j] = 0.f; }
+    bool ok = true;
+    for (int grp = 0; grp < n_groups; ++grp) {
+      const int buf = grp % TC_ACC_BUFS;
+      const uint32_t acc_ph = (uint32_t)(grp / TC_ACC_BUFS) & 1u;
+      if (!mbar_wait_bounded(acc_full_bar(buf), acc_ph, abort_flag, p.dev_status, TC_WAIT_ACC_FULL)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TC_TILE_N + h * 64);
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32_wait(taddr + c * 32, r);
+        if (c == 1) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acc_empty_bar(buf));        // buffer free for the next example's MMAs
+        }
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float g = __uint_as_float(r[j]);
+          acc_mean[c * 32 + j] += g;
+          if (PHI != 0) acc_stat[c * 32 + j] += phi_apply<PHI>(g);
+        }
+      }
+    }
+    if (ok && n_groups > 0) {
+      const int o = tile_m * TC_TILE_M + q * 32 + lane;
+      const int i_base = tile_n * TC_TILE_N + h * 64;
+      if (o < p.d_out) {
+        float* mrow = p.out_mean ? p.out_mean + (size_t)o * p.d_in : nullptr;
+        float* srow = p.out_stat ? p.out_stat + (size_t)o * p.d_in : nullptr;
+#pragma unroll
+        for (int j = 0; j < 64; j += 4) {
+          const int i = i_base + j;
+          if (i < p.d_in) {                                      // d_in % 8 == 0: a group of 4 is all in or all out
+            float4 vm = make_float4(acc_mean[j], acc_mean[j + 1], acc_mean[j + 2], acc_mean[j + 3]);
+            float4 vs = (PHI != 0) ? make_float4(acc_stat[j], acc_stat[j + 1], acc_stat[j + 2], acc_stat[j + 3]) : vm;
+            if (p.nsplit == 1) {
+              if (mrow) *reinterpret_cast<float4*>(mrow + i) = vm;
+              if (srow) *reinterpret_cast<float4*>(srow + i) = vs;
+            } else {
+              if (mrow) { atomicAdd(mrow + i, vm.x); atomicAdd(mrow + i + 1, vm.y); atomicAdd(mrow + i + 2, vm.z); atomicAdd(mrow + i + 3, vm.w); }
+              if (srow) { atomicAdd(srow + i, vs.x); atomicAdd(srow + i + 1, vs.y); atomicAdd(srow + i + 2, vs.z); atomicAdd(srow + i + 3, vs.w); }
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // A wait gave up.  Loads this block issued may still be landing in its shared memory: give them
+    // time (bounded) before the block exits and its shared memory is handed to another block.
+    const long long t0 = clock64();
+    while (clock64() - t0 < (1ll << 22)) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 2) { tc_fence_after(); tmem_dealloc(tmem_base, TC_TMEM_COLS); }
+}
+
+}  // namespace pe

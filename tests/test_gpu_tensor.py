@@ -1,0 +1,96 @@
+"""GPU parity of the tcgen05 tensor-core kernel against the oracle: small shapes that span several
+tiles with ragged tails, and the benchmark configurations at full size on sampled outputs."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2510_00236_b200 as pe
+from paper_2510_00236_b200 import inputs
+from parity_util import boundary_and_random, check_all, gpu_stats
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(autouse=True)
+def _tensor_path():
+    prev = pe.pe_set_path(pe.PATH_TENSOR)
+    yield
+    pe.pe_set_path(prev)
+
+
+def test_structured_single_tile_catches_layout_mistakes():
+    """Every (token, feature) pair gets a distinct small integer, exactly representable in bf16, so
+    a wrong swizzle, stride or operand orientation changes the result by whole numbers."""
+    B, T, d_in, d_out = 2, 64, 128, 128
+    t = torch.arange(T, dtype=torch.float32).view(1, T, 1)
+    X = ((t % 5) - 2 + (torch.arange(d_in).view(1, 1, d_in) % 7 - 3) + torch.arange(B).view(B, 1, 1)).to(torch.bfloat16)
+    dY = ((t % 3) - 1 + (torch.arange(d_out).view(1, 1, d_out) % 11 - 5) * 0.5 - torch.arange(B).view(B, 1, 1)).to(torch.bfloat16)
+    li = inputs.LayerInputs("structured", X.to(DEV).contiguous(), dY.to(DEV).contiguous())
+    rep = check_all(li, phis=("identity", "square", "sign"), tol=1e-6)
+    assert pe.pe_last_path() == pe.PATH_TENSOR
+    assert rep["sign_disagreements"] == 0
+
+
+@pytest.mark.parametrize("B,T,d_in,d_out", [
+    (3, 64, 128, 128),      # one tile, one stage per example
+    (5, 200, 136, 264),     # ragged tiles, T not a multiple of 16 or 64
+    (9, 16, 320, 192),      # short sequences: epilogue-bound regime
+    (2, 1, 64, 72),         # rank-one gradients
+    (1, 1000, 256, 128),    # single example
+    (70, 48, 8, 8),         # smallest widths the path takes, batch split across blocks
+    (40, 96, 384, 256),
+])
+def test_tensor_small_shapes_full_comparison(B, T, d_in, d_out):
+    li = inputs.gaussian_layer(B, T, d_in, d_out, seed=300 + 7 * B + T, device=DEV)
+    check_all(li, phis=("identity", "square", "sign"))
+    assert pe.pe_last_path() == pe.PATH_TENSOR
+
+
+def test_heavy_tailed_and_heterogeneous_small():
+    check_all(inputs.heavy_tailed_layer(12, 128, 256, 384, seed=41, device=DEV))
+    check_all(inputs.heterogeneous_layer(20, 64, 128, 256, seed=42, device=DEV))
+
+
+def test_unsplit_schedule_is_bit_reproducible():
+    li = inputs.gaussian_layer(4, 128, 2048, 2048, seed=43, device=DEV)     # 256 tiles >= SM count: no batch split
+    a = gpu_stats(li, "square")
+    b = gpu_stats(li, "square")
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+
+
+def test_config2_full_size_sampled_outputs():
+    li = inputs.config2(DEV)
+    rows = boundary_and_random(2048, 40, 1)
+    cols = boundary_and_random(512, 32, 2)
+    rep = check_all(li, rows, cols)
+    assert pe.pe_last_path() == pe.PATH_TENSOR
+    print("config2", rep)
+
+
+def test_config4_full_size_sampled_outputs():
+    li = inputs.config4(DEV)
+    rows = boundary_and_random(8192, 24, 3)
+    cols = boundary_and_random(2048, 24, 4)
+    rep = check_all(li, rows, cols)
+    print("config4", rep)
+    del li
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("B,T,d", [(16, 32, 1024), (16, 4096, 1024), (1024, 32, 1024), (128, 512, 4096), (1024, 512, 1024)])
+def test_config5_points_sampled_outputs(B, T, d):
+    li = inputs.config5_point(B, T, d, DEV)
+    rows = boundary_and_random(d, 16, 5)
+    cols = boundary_and_random(d, 16, 6)
+    check_all(li, rows, cols)
+    del li
+    torch.cuda.empty_cache()
+
+
+def test_token_stat_requires_workspace():
+    li = inputs.gaussian_layer(2, 64, 64, 64, seed=44, device=DEV)
+    out = torch.empty((64, 64), device=DEV)
+    lib = pe.load_library()
+    st = lib.pe_token_sqstats(li.X.data_ptr(), li.dY.data_ptr(), 2, 64, 64, 64, out.data_ptr(), None, 0, None)
+    assert st == 9      # PE_ERR_WORKSPACE

@@ -1,0 +1,80 @@
+"""CPU-only checks of the C-ABI boundary: the library builds, loads without a GPU, exports every
+function the header declares, and its host-side helpers behave."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2510_00236_b200 as pe
+from paper_2510_00236_b200 import build as pe_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    pe_build.build_library()
+    return pe.load_library()
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "pestats.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"\b([a-z_0-9]+)\s*\([^;{]*\)\s*;", text)
+    return sorted(set(names))
+
+
+def test_header_functions_are_all_exported_and_bound(lib):
+    declared = _declared_functions()
+    assert "pe_linear_stats" in declared and "microsignsgd_step" in declared
+    for name in declared:
+        assert hasattr(lib, name), f"{name} declared in pestats.h but not exported"
+    assert sorted(pe.EXPORTED_SYMBOLS) == declared
+    for name in declared:
+        assert hasattr(pe, name), f"binding lacks {name}"
+
+
+def test_status_strings_and_path_switch(lib):
+    assert pe.pe_status_string(0) == "PE_OK"
+    assert pe.pe_status_string(8) == "PE_ERR_TIMEOUT"
+    assert pe.pe_status_string(9) == "PE_ERR_WORKSPACE"
+    assert pe.pe_status_string(1234) == "PE_ERR_UNKNOWN"
+    prev = pe.pe_set_path(pe.PATH_SIMT)
+    assert pe.pe_set_path(prev) == pe.PATH_SIMT
+    assert pe.pe_set_path(77) == -1
+
+
+def test_host_side_validation_needs_no_gpu(lib):
+    # argument errors are reported before any CUDA call
+    assert lib.pe_linear_stats(None, None, 1, 1, 8, 8, 1, None, None, None) == 1          # PE_ERR_NULL
+    buf = ctypes.create_string_buffer(4096)
+    p = ctypes.addressof(buf)
+    p16 = (p + 15) & ~15
+    assert lib.pe_linear_stats(p16, p16, 1, 1, 8, 8, 1, None, None, None) == 1            # both outputs NULL
+    assert lib.pe_linear_stats(p16, p16, -1, 1, 8, 8, 1, p16, p16, None) == 2             # PE_ERR_DIM
+    assert lib.pe_linear_stats(None, None, 1, 1, 0, 8, 1, p16, p16, None) == 2
+    assert lib.pe_linear_stats(p16 + 2, p16, 1, 1, 8, 8, 1, p16, p16, None) == 3          # PE_ERR_ALIGN
+    assert lib.pe_linear_stats(p16, p16, 1, 1, 8, 8, 7, p16, p16, None) == 5              # PE_ERR_PHI
+    assert lib.microadam_step(p16, None, p16, p16, p16, p16, 4, 0, 1.0, 1e-3, 0.9, 0.99, 1e-8, 0, 0.0, 1, None) == 2
+    assert lib.microadam_step(p16, None, p16, p16, p16, p16, 4, 1, 1.0, 1e-3, 0.9, 0.99, 1e-8, 0, 0.0, 0, None) == 2
+    assert lib.microsignsgd_step(p16, None, None, p16, 4, 1, 1e-3, 0.9, 0.0, None) == 1
+
+
+def test_workspace_size_formula(lib):
+    prev = pe.pe_set_path(pe.PATH_AUTO)
+    try:
+        assert pe.pe_token_sqstats_workspace_bytes(64, 256, 512, 2048) == 64 * 256 * (512 + 2048) * 2
+        assert pe.pe_token_sqstats_workspace_bytes(3, 5, 8, 8) == 256 + 256          # rounded up to 256 B each
+        assert pe.pe_token_sqstats_workspace_bytes(3, 5, 7, 8) == 0                  # SIMT shape: no workspace
+        pe.pe_set_path(pe.PATH_SIMT)
+        assert pe.pe_token_sqstats_workspace_bytes(64, 256, 512, 2048) == 0
+    finally:
+        pe.pe_set_path(prev)
+
+
+def test_cpu_tensors_are_rejected_loudly():
+    import torch
+    X = torch.zeros(1, 2, 8, dtype=torch.bfloat16)
+    with pytest.raises(pe.PestatsError):
+        pe.pe_linear_stats(X, X, "square")
