@@ -1,0 +1,423 @@
+#!/usr/bin/env python
+"""Benchmark of the per-example-statistics hot path on B200.
+
+One step = one pass of the whole path over one batch of a transformer-MLP-shaped bf16 layer
+(B=64, T=256, d_in=512, d_out=2048; X ~ N(0,1), dY ~ N(0,1/T) with 10% of sequences x5):
+  pe_linear_stats(square)  -> sum_b G_b and sum_b G_b^2      (tcgen05 kernel)
+  pe_linear_stats(sign)    -> sum_b sign(G_b)                (tcgen05 kernel)
+  pe_token_sqstats         -> sum_{b,t} dY^2 X^2             (square pre-pass + tcgen05 kernel)
+  microadam_step           on fp32 master weights (+ bf16 copy)
+  microsignsgd_step        on a second set of master weights (+ bf16 copy)
+The metric is the contraction throughput of the step, 3 x 2*B*T*d_in*d_out flops per step, in TFLOP/s.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c4] [--impl ours|reference]
+
+With N > 1 (torchrun) every rank runs an independent replica of the same workload on its own GPU
+(the path has no exchange step); the reported value is the sum over ranks divided by the slowest
+rank's time.  `--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "per-example-stat TFLOP/s"
+UNIT = "TFLOP/s"
+WORKLOADS = {
+    # name: (B, T, d_in, d_out, rotating input sets)
+    "c2": (64, 256, 512, 2048, 6),
+    "c4": (256, 1024, 2048, 8192, 1),
+}
+ADAM = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8)
+SIGN = dict(lr=3.47e-3, beta=0.9)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16_tflops": float(d["bf16_tflops"]), "hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+def profile_traffic(workload: str):
+    """DRAM bytes per launch of the statistics kernel from the committed ncu summary, if present."""
+    path = os.path.join(ROOT, "profiles", f"tc_stats_kernel_{workload}.txt")
+    try:
+        for line in open(path):
+            if line.startswith("dram_bytes_per_launch:"):
+                return float(line.split(":")[1].split()[0])
+    except OSError:
+        pass
+    return None
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(self.gpu_index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx = float(parts[2])
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def make_state(pe, inputs, torch, name, dev, seed_offset=0):
+    B, T, d_in, d_out, nsets = WORKLOADS[name]
+    sets = []
+    for k in range(nsets):
+        if name == "c2":
+            li = inputs.heterogeneous_layer(B, T, d_in, d_out, seed=inputs.BASE_SEED + 2 + 1000 * k + seed_offset, device=dev,
+                                            name="c2", with_weights=(k == 0))
+        else:
+            li = inputs.heavy_tailed_layer(B, T, d_in, d_out, seed=inputs.BASE_SEED + 4 + 1000 * k + seed_offset, device=dev,
+                                           name="c4", with_weights=(k == 0))
+        sets.append(li)
+    n = d_out * d_in
+    f32 = dict(dtype=torch.float32, device=dev)
+    st = {
+        "shape": (B, T, d_in, d_out), "sets": sets,
+        "mean": torch.empty((d_out, d_in), **f32), "sq": torch.empty((d_out, d_in), **f32),
+        "sgn": torch.empty((d_out, d_in), **f32), "tok": torch.empty((d_out, d_in), **f32),
+        "ws": torch.empty(max(1, pe.pe_token_sqstats_workspace_bytes(B, T, d_in, d_out)), dtype=torch.uint8, device=dev),
+        "theta": sets[0].W.clone(), "m": torch.zeros((d_out, d_in), **f32), "v": torch.zeros((d_out, d_in), **f32),
+        "theta_lp": torch.empty((d_out, d_in), dtype=torch.bfloat16, device=dev),
+        "theta2": sets[0].W.clone(), "m2": torch.zeros((d_out, d_in), **f32),
+        "theta2_lp": torch.empty((d_out, d_in), dtype=torch.bfloat16, device=dev),
+        "n": n,
+    }
+    return st
+
+
+def run_step(pe, st, i, X=None, dY=None, ev=None):
+    B = st["shape"][0]
+    li = st["sets"][i % len(st["sets"])]
+    X = li.X if X is None else X
+    dY = li.dY if dY is None else dY
+    if ev is not None:
+        ev[0].record()
+    pe.pe_linear_stats(X, dY, pe.PHI_SQUARE, st["mean"], st["sq"])
+    if ev is not None:
+        ev[1].record()
+    pe.pe_linear_stats(X, dY, pe.PHI_SIGN, None, st["sgn"])
+    pe.pe_token_sqstats(X, dY, st["tok"], st["ws"])
+    pe.microadam_step(st["theta"], st["m"], st["v"], st["mean"], st["sq"], B, step=i + 1, theta_lp=st["theta_lp"], **ADAM)
+    pe.microsignsgd_step(st["theta2"], st["m2"], st["sgn"], B, theta_lp=st["theta2_lp"], **SIGN)
+
+
+def time_region(torch, fn, iters):
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(iters):
+        fn(i)
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / iters
+
+
+def time_each(torch, fn, iters=20, warmup=3):
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    ts = []
+    for i in range(iters):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); fn(i); b.record()
+        ts.append((a, b))
+    torch.cuda.synchronize()
+    v = sorted(x.elapsed_time(y) for x, y in ts)
+    return v[len(v) // 2], v[0]
+
+
+def oracle_sample(inputs, workload, n_rows, n_cols):
+    """Column-gathered sub-layer of the workload for the CPU oracle (full B and T)."""
+    import numpy as np
+    B, T, d_in, d_out, _ = WORKLOADS[workload]
+    if workload == "c2":
+        li = inputs.config2("cpu")
+    else:   # a reduced-batch stand-in keeps host generation bounded
+        li = inputs.heavy_tailed_layer(32, T, d_in, d_out, seed=inputs.BASE_SEED + 4, device="cpu", name="c4", with_weights=False)
+    rows = list(np.linspace(0, d_out - 1, n_rows).astype(int)) if n_rows < d_out else list(range(d_out))
+    cols = list(np.linspace(0, d_in - 1, n_cols).astype(int)) if n_cols < d_in else list(range(d_in))
+    sub = li if (n_rows >= d_out and n_cols >= d_in) else inputs.gather_columns(li, rows, cols)
+    return inputs.to_numpy_bits(sub.X), inputs.to_numpy_bits(sub.dY)
+
+
+def time_oracle(Xh, dYh):
+    import oracle
+    B, T, ni = Xh.shape
+    no = dYh.shape[2]
+    t0 = time.perf_counter()
+    st = oracle.linear_stats(Xh, dYh)
+    oracle.token_sqstats(Xh, dYh)
+    import numpy as np
+    z = np.zeros((no, ni))
+    oracle.microadam_step(z, z, z, st.sum_g, st.sum_g2, B, step=1, **ADAM)
+    oracle.microsignsgd_step(z, z, st.sum_sign, B, **SIGN)
+    dt = time.perf_counter() - t0
+    flops = 2 * 2.0 * B * T * ni * no      # the oracle forms G_b once for every phi, plus the per-token contraction
+    return dt, flops
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2510_00236_b200 import inputs
+    B, T, d_in, d_out, _ = WORKLOADS[args.workload]
+    n_rows, n_cols = min(d_out, 256), min(d_in, 256)
+    Xh, dYh = oracle_sample(inputs, args.workload, n_rows, n_cols)
+    for _ in range(max(1, min(args.warmup, 3))):
+        time_oracle(Xh, dYh)
+    t = 0.0
+    flops = 0.0
+    for _ in range(args.steps):
+        dt, fl = time_oracle(Xh, dYh)
+        t += dt
+        flops += fl
+    value = flops / t / 1e12
+    sample = f"{n_rows}x{n_cols} of the {d_out}x{d_in} outputs, B={Xh.shape[0]}, T={T} per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "B": B, "T": T, "d_in": d_in, "d_out": d_out, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import paper_2510_00236_b200 as pe
+    from paper_2510_00236_b200 import inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    pe.load_library()          # fails loudly when the CUDA library is missing
+
+    name = args.workload
+    B, T, d_in, d_out, nsets = WORKLOADS[name]
+    st = make_state(pe, inputs, torch, name, dev)
+    flops_one = 2.0 * B * T * d_in * d_out
+    flops_step = 3.0 * flops_one
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ------------------------------------------------------------ device-resident timing
+    for i in range(args.warmup):
+        run_step(pe, st, i)
+    status, detail = pe.pe_get_async_status(dev)
+    assert status == 0, f"device status {status}/{detail}"
+    assert pe.pe_last_path() == pe.PATH_TENSOR, "tensor-core path did not run"
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    barrier()
+    pe.pe_reset_launch_count()
+    kernel_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for i in range(args.steps):
+        run_step(pe, st, args.warmup + i, ev=kernel_events[i])
+    t_end.record()
+    barrier()
+    launches = pe.pe_launch_count()
+    ms_total = t_start.elapsed_time(t_end)
+    clocks = sampler.stop() if rank == 0 else None
+    kernel_ms = statistics.fmean(a.elapsed_time(b) for a, b in kernel_events)
+    if dist is not None:
+        tt = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    ms_step = ms_total / args.steps
+    value = world * flops_step / (ms_step * 1e-3) / 1e12
+
+    # ------------------------------------------------------------ end to end: host buffers in, statistics out
+    e2e_steps = max(3, min(20, args.steps // 5))
+    li0 = st["sets"][0]
+    hX = torch.empty(li0.X.shape, dtype=li0.X.dtype, pin_memory=True).copy_(li0.X)
+    hdY = torch.empty(li0.dY.shape, dtype=li0.dY.dtype, pin_memory=True).copy_(li0.dY)
+    dX, ddY = torch.empty_like(li0.X), torch.empty_like(li0.dY)
+    outs = [st["mean"], st["sq"], st["sgn"], st["tok"]]
+    houts = [torch.empty(o.shape, dtype=o.dtype, pin_memory=True) for o in outs]
+
+    def e2e_step(i):
+        dX.copy_(hX, non_blocking=True)
+        ddY.copy_(hdY, non_blocking=True)
+        run_step(pe, st, i, X=dX, dY=ddY)
+        for h, o in zip(houts, outs):
+            h.copy_(o, non_blocking=True)
+
+    for i in range(2):
+        e2e_step(i)
+    barrier()
+    ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ea.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    eb.record()
+    barrier()
+    e2e_ms = ea.elapsed_time(eb)
+    if dist is not None:
+        tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    e2e_value = world * flops_step / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    h2d = hX.numel() * hX.element_size() + hdY.numel() * hdY.element_size()
+    d2h = sum(o.numel() * o.element_size() for o in outs)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ------------------------------------------------------------ context numbers (rank 0, outside the timed region)
+    peaks = measured_peaks()
+    li = st["sets"][0]
+    extra = {}
+    med, best = time_each(torch, lambda i: pe.pe_linear_stats(li.X, li.dY, pe.PHI_SQUARE, st["mean"], st["sq"]))
+    extra["pe_linear_stats_square_us"] = {"median": med * 1e3, "best": best * 1e3, "tflops_median": flops_one / med / 1e9}
+    med_s, best_s = time_each(torch, lambda i: pe.pe_linear_stats(li.X, li.dY, pe.PHI_SIGN, None, st["sgn"]))
+    extra["pe_linear_stats_sign_us"] = {"median": med_s * 1e3, "best": best_s * 1e3, "tflops_median": flops_one / med_s / 1e9}
+    med_t, best_t = time_each(torch, lambda i: pe.pe_token_sqstats(li.X, li.dY, st["tok"], st["ws"]))
+    extra["pe_token_sqstats_us"] = {"median": med_t * 1e3, "best": best_t * 1e3, "tflops_median": flops_one / med_t / 1e9}
+    A2, B2 = li.dY.view(B * T, d_out), li.X.view(B * T, d_in)
+    med_g, best_g = time_each(torch, lambda i: torch.matmul(A2.t(), B2))
+    extra["cublas_wgrad_gemm_us"] = {"median": med_g * 1e3, "best": best_g * 1e3, "tflops_median": flops_one / med_g / 1e9,
+                                     "note": "torch.matmul(dY_flat^T, X_flat), bf16 in and out"}
+    extra["overhead_vs_gemm"] = med / med_g
+    n = st["n"]
+    big = 1 << 26       # update kernels on a parameter count far larger than L2 (64 Mi parameters)
+    bufs = [torch.zeros(big, device=dev) for _ in range(5)]
+    lp = torch.empty(big, dtype=torch.bfloat16, device=dev)
+    med_a, _ = time_each(torch, lambda i: pe.microadam_step(bufs[0], bufs[1], bufs[2], bufs[3], bufs[4], B, step=1, theta_lp=lp, **ADAM), iters=10)
+    med_sg, _ = time_each(torch, lambda i: pe.microsignsgd_step(bufs[0], bufs[1], bufs[3], B, theta_lp=lp, **SIGN), iters=10)
+    extra["microadam_step"] = {"params": big, "gbs": 34.0 * big / med_a / 1e6, "frac_of_hbm_peak": 34.0 * big / med_a / 1e6 / peaks["hbm_gbs"]}
+    extra["microsignsgd_step"] = {"params": big, "gbs": 22.0 * big / med_sg / 1e6, "frac_of_hbm_peak": 22.0 * big / med_sg / 1e6 / peaks["hbm_gbs"]}
+    del bufs, lp
+
+    achieved = flops_one / (kernel_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "tc_stats_kernel<square>", "achieved": achieved, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst)",
+                "traffic": profile_traffic(name), "avg_launch_ms": kernel_ms,
+                "algorithmic_flops_per_launch": flops_one,
+                "algorithmic_bytes_per_launch": 2.0 * B * T * (d_in + d_out) + 8.0 * d_in * d_out}
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline and world == 1:
+        import oracle
+        if name == "c2":
+            Xh, dYh = inputs.to_numpy_bits(li.X), inputs.to_numpy_bits(li.dY)
+            sample = "the full workload, once"
+        else:
+            Xh, dYh = oracle_sample(inputs, name, 256, 256)
+            sample = f"256x256 of the {d_out}x{d_in} outputs at B={Xh.shape[0]}, once"
+        dt, fl = time_oracle(Xh, dYh)
+        cpu_baseline = {"value": fl / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                        "sample": sample, "seconds": dt}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": name, "B": B, "T": T, "d_in": d_in, "d_out": d_out,
+                   "step": "pe_linear_stats(square)+pe_linear_stats(sign)+pe_token_sqstats+microadam_step+microsignsgd_step",
+                   "flops_per_step": flops_step, "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": f"{nsets} rotating input sets, {nsets * 2 * B * T * (d_in + d_out) / 1e6:.0f} MB in all (> 126 MB L2)"
+                         if nsets > 1 else "inputs larger than L2"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "cpu_baseline": cpu_baseline,
+        "extra": extra,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -75,10 +75,12 @@ pe_status_t pe_linear_stats_f32(const float* X, const float* dY, int B, int T, i
 /*
  * Per-token second moment (Section 2.3, the "per-token" alternative):
  *     out_stat[o,i] = sum_{b,t} dY[b,t,o]^2 * X[b,t,i]^2  =  ((dY o dY)^T (X o X))[o,i].
- * B and T only enter through the row count B*T.  bf16 inputs.  On the tensor-core path the
- * squared operands are rounded to bf16 once and staged in `workspace` (device memory, 256-byte
- * aligned, at least pe_token_sqstats_workspace_bytes() bytes, contents undefined afterwards);
- * the SIMT path squares in fp32 and ignores the workspace (it may then be NULL).
+ * B and T only enter through the row count B*T.  bf16 inputs.  On the tensor-core path (taken when
+ * the shape allows it and B*T >= 256) the squared operands are rounded to tf32 (11 significant bits,
+ * so every entry is within about 1e-3 relative of the exact sum) and staged as fp32 in `workspace`
+ * (device memory, 256-byte aligned, at least pe_token_sqstats_workspace_bytes() bytes, contents
+ * undefined afterwards); the SIMT path squares in fp32 and ignores the workspace (it may then be
+ * NULL).
  */
 pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_in, int d_out,
                              float* out_stat, void* workspace, size_t workspace_bytes,

@@ -28,7 +28,7 @@ struct DeviceInfo {
   std::atomic<int> state{0};     // 0 unknown, 1 ready, -1 failed
   int cc_major = 0, sm_count = 0;
   unsigned int* status_ptr = nullptr;
-  bool tc_attr_set[3] = {false, false, false};
+  bool tc_attr_set[4] = {false, false, false, false};
 };
 static DeviceInfo g_dev[MAX_DEVICES];
 
@@ -85,25 +85,39 @@ static pe_status_t check_launch() {
   return PE_OK;
 }
 
-// bf16 [B, T, d] row-major viewed as a 3-D tensor (d, T, B); one box = 64 features x TC_BK tokens of
-// one example, 128-byte swizzled.  Tokens past T and features past d read as zero.
-static pe_status_t make_operand_map(CUtensorMap* m, const void* base, int B, int T, int d) {
+// [B, T, d] row-major (bf16, or fp32 read as tf32) viewed as a 3-D tensor (d, T, B); one box = 128
+// bytes of features x BK tokens of one example, 128-byte swizzled (16-byte chunks for bf16, 32-byte
+// chunks for fp32: the MN-major tf32 MMA accepts no other layout).  Tokens past T and features past d read as zero.
+static pe_status_t make_operand_map(CUtensorMap* m, const void* base, int B, int T, int d, bool f32) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return PE_ERR_CUDA;
+  const cuuint64_t es = f32 ? 4ull : 2ull;
   cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)T, (cuuint64_t)B};
-  cuuint64_t strides[2] = {(cuuint64_t)d * 2ull, (cuuint64_t)T * (cuuint64_t)d * 2ull};
-  cuuint32_t box[3] = {64u, (cuuint32_t)TC_BK, 1u};
+  cuuint64_t strides[2] = {(cuuint64_t)d * es, (cuuint64_t)T * (cuuint64_t)d * es};
+  cuuint32_t box[3] = {(cuuint32_t)(f32 ? TcOperand<true>::BOX_FEATS : TcOperand<false>::BOX_FEATS),
+                       (cuuint32_t)(f32 ? TcOperand<true>::BK : TcOperand<false>::BK), 1u};
   cuuint32_t estr[3] = {1u, 1u, 1u};
-  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+  CUresult r = enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, f32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? PE_OK : PE_ERR_CUDA;
+}
+
+// The tensor-core per-token statistic rounds each squared operand to tf32 (relative error at most
+// 2^-11 per factor, so at most ~1e-3 on any entry, all terms being non-negative).  Tiny problems
+// gain nothing from the tensor cores and take the SIMT kernel (fp32 squares).
+constexpr long long TOKEN_TC_MIN_ROWS = 256;
+
+static bool tc_shape_ok(int B, int T, int d_in, int d_out);
+static bool token_tc_ok(int B, int T, int d_in, int d_out) {
+  return tc_shape_ok(B, T, d_in, d_out) && (long long)B * T >= TOKEN_TC_MIN_ROWS;
 }
 
 static bool tc_shape_ok(int B, int T, int d_in, int d_out) {
   if (B < 1 || T < 1) return false;
   if ((d_in % 8) || (d_out % 8)) return false;                        // 16-byte row pitch for TMA
-  if ((long long)T * (d_in > d_out ? d_in : d_out) * 2ll >= (1ll << 40)) return false;   // TMA stride limit
+  if ((long long)T * (d_in > d_out ? d_in : d_out) * 4ll >= (1ll << 40)) return false;   // TMA stride limit (fp32 staging included)
   return true;
 }
 
@@ -127,27 +141,28 @@ static pe_status_t zero_outputs(float* a, float* b, size_t bytes, cudaStream_t s
   return PE_OK;
 }
 
-template <int PHI>
+template <int PHI, bool TF32>
 static pe_status_t launch_tc_inst(DeviceInfo* di, const CUtensorMap& mx, const CUtensorMap& my, const TcParams& p,
                                   dim3 grid, cudaStream_t st) {
-  if (!di->tc_attr_set[PHI]) {
-    if (cudaFuncSetAttribute(tc_stats_kernel<PHI>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES) != cudaSuccess) {
+  constexpr int slot = TF32 ? 3 : PHI;
+  if (!di->tc_attr_set[slot]) {
+    if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES) != cudaSuccess) {
       cudaGetLastError();
       return PE_ERR_CUDA;
     }
-    di->tc_attr_set[PHI] = true;
+    di->tc_attr_set[slot] = true;
   }
-  tc_stats_kernel<PHI><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(mx, my, p);
+  tc_stats_kernel<PHI, TF32><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(mx, my, p);
   return check_launch();
 }
 
 // Tensor-core launch.  per_example = 0 runs the plain contraction over all B*T rows.
 static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int B, int T, int d_in, int d_out, int phi,
-                             int per_example, float* out_mean, float* out_stat, cudaStream_t st) {
+                             int per_example, float* out_mean, float* out_stat, cudaStream_t st, bool tf32 = false) {
   CUtensorMap mx, my;
-  pe_status_t rc = make_operand_map(&mx, X, B, T, d_in);
+  pe_status_t rc = make_operand_map(&mx, X, B, T, d_in, tf32);
   if (rc != PE_OK) return rc;
-  rc = make_operand_map(&my, dY, B, T, d_out);
+  rc = make_operand_map(&my, dY, B, T, d_out, tf32);
   if (rc != PE_OK) return rc;
   const int tiles_n = (d_in + TC_TILE_N - 1) / TC_TILE_N, tiles_m = (d_out + TC_TILE_M - 1) / TC_TILE_M;
   if (tiles_m > 65535) return PE_ERR_DIM;
@@ -160,9 +175,10 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = per_example;
   p.out_mean = out_mean; p.out_stat = out_stat; p.dev_status = di->status_ptr;
   dim3 grid(tiles_n, tiles_m, ns);
-  if (!per_example || phi == PE_PHI_IDENTITY) return launch_tc_inst<0>(di, mx, my, p, grid, st);
-  if (phi == PE_PHI_SQUARE) return launch_tc_inst<1>(di, mx, my, p, grid, st);
-  return launch_tc_inst<2>(di, mx, my, p, grid, st);
+  if (tf32) return launch_tc_inst<0, true>(di, mx, my, p, grid, st);
+  if (!per_example || phi == PE_PHI_IDENTITY) return launch_tc_inst<0, false>(di, mx, my, p, grid, st);
+  if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false>(di, mx, my, p, grid, st);
+  return launch_tc_inst<2, false>(di, mx, my, p, grid, st);
 }
 
 template <typename TIn, int MODE>
@@ -253,9 +269,9 @@ pe_status_t pe_linear_stats_f32(const float* X, const float* dY, int B, int T, i
 }
 
 size_t pe_token_sqstats_workspace_bytes(int B, int T, int d_in, int d_out) {
-  if (g_path.load() == PE_PATH_SIMT || !tc_shape_ok(B, T, d_in, d_out)) return 0;
+  if (g_path.load() == PE_PATH_SIMT || !token_tc_ok(B, T, d_in, d_out)) return 0;
   const size_t rows = (size_t)B * (size_t)T;
-  return align_up(rows * d_in * 2, 256) + align_up(rows * d_out * 2, 256);
+  return align_up(rows * d_in * 4, 256) + align_up(rows * d_out * 4, 256);
 }
 
 pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_stat,
@@ -269,26 +285,27 @@ pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_
   if (rc != PE_OK) return rc;
   if (B == 0 || T == 0) return zero_outputs(out_stat, nullptr, (size_t)d_in * d_out * sizeof(float), st);
   const int forced = g_path.load();
-  const bool tc_ok = tc_shape_ok(B, T, d_in, d_out);
-  if (forced == PE_PATH_TENSOR && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
+  const bool tc_ok = token_tc_ok(B, T, d_in, d_out);
+  if (forced == PE_PATH_TENSOR && !tc_shape_ok(B, T, d_in, d_out)) return PE_ERR_UNSUPPORTED_SHAPE;
   if (tc_ok && forced != PE_PATH_SIMT) {
     const size_t rows = (size_t)B * (size_t)T;
-    const size_t x_bytes = align_up(rows * d_in * 2, 256), y_bytes = align_up(rows * d_out * 2, 256);
+    const size_t x_bytes = align_up(rows * d_in * 4, 256), y_bytes = align_up(rows * d_out * 4, 256);
     if (!workspace || workspace_bytes < x_bytes + y_bytes) return PE_ERR_WORKSPACE;
     if (!aligned(workspace, 256)) return PE_ERR_ALIGN;
-    __nv_bfloat16* x2 = static_cast<__nv_bfloat16*>(workspace);
-    __nv_bfloat16* y2 = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + x_bytes);
+    float* x2 = static_cast<float*>(workspace);
+    float* y2 = reinterpret_cast<float*>(static_cast<char*>(workspace) + x_bytes);
     const long long nx = (long long)rows * d_in, ny = (long long)rows * d_out;
-    square_bf16_kernel<<<grid_for(nx / 8 + 8, di->sm_count), OPT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(X), x2, nx);
+    square_to_tf32_kernel<<<grid_for(nx / 8 + 8, di->sm_count), OPT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(X), x2, nx);
     if ((rc = check_launch()) != PE_OK) return rc;
-    square_bf16_kernel<<<grid_for(ny / 8 + 8, di->sm_count), OPT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(dY), y2, ny);
+    square_to_tf32_kernel<<<grid_for(ny / 8 + 8, di->sm_count), OPT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(dY), y2, ny);
     if ((rc = check_launch()) != PE_OK) return rc;
     // B and T only enter through B*T: regroup the rows into 64-token "examples" when possible so
     // the batch split has many units to balance.
+    constexpr int REGROUP = 2 * TcOperand<true>::BK;
     int Bp = B, Tp = T;
-    if (T % TC_BK == 0 && rows / TC_BK < (size_t)(1u << 30)) { Bp = (int)(rows / TC_BK); Tp = TC_BK; }
+    if (T % REGROUP == 0 && rows / REGROUP < (size_t)(1u << 30)) { Bp = (int)(rows / REGROUP); Tp = REGROUP; }
     g_last_path.store(PE_PATH_TENSOR);
-    return launch_tc(di, x2, y2, Bp, Tp, d_in, d_out, PE_PHI_IDENTITY, 0, nullptr, out_stat, st);
+    return launch_tc(di, x2, y2, Bp, Tp, d_in, d_out, PE_PHI_IDENTITY, 0, nullptr, out_stat, st, true);
   }
   g_last_path.store(PE_PATH_SIMT);
   return launch_simt<__nv_bfloat16, MODE_TOKEN>(di, static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T,

@@ -52,13 +52,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // code and raises the block-wide abort flag so that every other role leaves its loops as well.
 constexpr long long WAIT_CYCLE_LIMIT = 1ll << 32;
 
-// Returns false if the wait was abandoned (its own timeout, or another role's).
+// Returns false if the wait was abandoned (its own timeout, or another role's).  SLEEP_NS > 0 backs
+// off between polls: every poll is a shared-memory access, and shared-memory bandwidth is what the
+// MMA operand reads need, so roles that wait long (the epilogue warps) must not spin hot.
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                   unsigned int* dev_status, int code) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   unsigned int spins = 0;
   while (true) {
+    if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 0xff) == 0) {
       if (*abort_flag) return false;
@@ -99,37 +103,57 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 
 // ---------------------------------------------------------------- descriptors
 // Shared-memory matrix descriptor (64-bit): start address, leading / stride byte offsets (all >> 4),
-// descriptor version 1 (sm_100) at bit 46, swizzle mode at bits 61..63 (2 = 128-byte swizzle).
-__device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+// descriptor version 1 (sm_100) at bit 46, swizzle mode at bits 61..63.
+//   layout 2 = 128-byte swizzle of 16-byte chunks (8-row atoms)      -- 16-bit MN-major operands
+//   layout 1 = 128-byte swizzle of 32-byte chunks (4-row atoms)      -- the only MN-major form for tf32
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
   uint64_t d = 0;
   d |= (uint64_t)((saddr >> 4) & 0x3FFF);
   d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
   d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
   d |= (uint64_t)1 << 46;
-  d |= (uint64_t)2 << 61;
+  d |= (uint64_t)layout << 61;
   return d;
 }
-
-// Instruction descriptor for kind::f16 with bf16 A and B, fp32 accumulator, both operands MN-major
-// (the contraction index is the slow one in shared memory), shape M x N x 16.
-__host__ __device__ constexpr uint32_t make_idesc_bf16_mn_major(int M, int N) {
-  return (1u << 4)                      // D format: F32
-         | (1u << 7)                    // A format: BF16
-         | (1u << 10)                   // B format: BF16
-         | (1u << 15)                   // A is MN-major
-         | (1u << 16)                   // B is MN-major
-         | ((uint32_t)(N >> 3) << 17)   // N / 8
-         | ((uint32_t)(M >> 4) << 24);  // M / 16
+__device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return make_smem_desc(saddr, lbo_bytes, sbo_bytes, 2u);
 }
 
+// Instruction descriptor for kind::f16 with bf16 A and B (or kind::tf32 with tf32 A and B), fp32
+// accumulator, both operands MN-major (the contraction index is the slow one in shared memory),
+// shape M x N x (32 bytes of K).
+__host__ __device__ constexpr uint32_t make_idesc_mn_major(int M, int N, bool tf32) {
+  return (1u << 4)                          // D format: F32
+         | ((tf32 ? 2u : 1u) << 7)          // A format: BF16 = 1, TF32 = 2
+         | ((tf32 ? 2u : 1u) << 10)         // B format
+         | (1u << 15)                       // A is MN-major
+         | (1u << 16)                       // B is MN-major
+         | ((uint32_t)(N >> 3) << 17)       // N / 8
+         | ((uint32_t)(M >> 4) << 24);      // M / 16
+}
+__host__ __device__ constexpr uint32_t make_idesc_bf16_mn_major(int M, int N) { return make_idesc_mn_major(M, N, false); }
+
 // D[tmem] (+)= A[smem] * B[smem]; issued by a single thread.
+template <bool TF32>
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  if constexpr (TF32) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
+}
 __device__ __forceinline__ void umma_bf16_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
+  umma_ss<false>(d_tmem, adesc, bdesc, idesc, accumulate);
 }
 // Arrive once on `bar` when every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {

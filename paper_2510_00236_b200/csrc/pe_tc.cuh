@@ -6,14 +6,15 @@
 // memory), read back by the epilogue warps, passed through phi and added to two register-resident
 // running sums (sum_b phi(G_b) and sum_b G_b).  The per-example tile never leaves the SM.
 //
-// Warp roles (12 warps):  0 = TMA producer, 1 = MMA issuer, 2 = TMEM allocator, 3 = idle,
+// Warp roles (12 warps):  0 = TMA producer, 1 and 3 = MMA issuers, 2 = TMEM allocator,
 // 4..11 = epilogue (warp w reads TMEM lanes 32*(w%4)..+31, columns 64*((w-4)/4)..+63 of the tile).
-// The tensor-memory accumulator is ring-buffered (4 x 128 columns) so the MMAs of example b+1..b+3
-// overlap the epilogue of example b.
+// Two examples are in flight at once, one per issuer, each issuer double-buffering its accumulator
+// in tensor memory (4 x 128 columns in all), so the MMAs of later examples overlap the epilogue of
+// earlier ones.
 //
 // Operand orientation: A = dY_b viewed as M = d_out x K = T and B = X_b viewed as N = d_in x K = T.
 // In global memory the contraction index (the token) is the slow one, so both operands are
-// "MN-major".  A TMA box is 64 features (128 bytes) x BK tokens; with the 128-byte swizzle that is
+// "MN-major".  A TMA box is 128 bytes of features (64 bf16) x BK tokens; with the 128-byte swizzle that is
 // exactly the canonical MN-major layout of the MMA: 8-token x 64-feature atoms of 1 KiB, the next
 // 8 tokens 1 KiB further (stride byte offset), the next 64 features one box further (leading byte
 // offset).
@@ -24,19 +25,35 @@ namespace pe {
 
 constexpr int TC_TILE_M = 128;    // d_out rows per tile   (MMA M)
 constexpr int TC_TILE_N = 128;    // d_in columns per tile (MMA N)
-constexpr int TC_BK = 64;         // tokens per pipeline stage
 constexpr int TC_STAGES = 6;
 constexpr int TC_ACC_BUFS = 4;    // TMEM accumulator ring
 constexpr int TC_TMEM_COLS = TC_ACC_BUFS * TC_TILE_N;   // 512
 constexpr int TC_THREADS = 384;
 constexpr int TC_REGS_CONTROL = 64;     // setmaxnreg of warps 0..3
 constexpr int TC_REGS_EPILOGUE = 216;   // setmaxnreg of warps 4..11  (4*32*64 + 8*32*216 = 63488 <= 65536)
-constexpr int TC_BOX_BYTES = 64 * TC_BK * 2;                              // one 64-feature x BK-token box
-constexpr int TC_A_BYTES = (TC_TILE_M / 64) * TC_BOX_BYTES;               // 16 KiB
-constexpr int TC_B_BYTES = (TC_TILE_N / 64) * TC_BOX_BYTES;               // 16 KiB
-constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;                   // 32 KiB
+
+// Operand element type of the MMA.  bf16 (kind::f16, 16 tokens per instruction) for the per-example
+// statistics; tf32 (kind::tf32, fp32 storage, 8 tokens per instruction) for the per-token statistic,
+// whose squared operands need more than bf16's 8 significant bits.
+template <bool TF32>
+struct TcOperand {
+  static constexpr int ELEM_BYTES = TF32 ? 4 : 2;
+  static constexpr int BOX_FEATS = 128 / ELEM_BYTES;            // features per 128-byte swizzle row: 64 | 32
+  static constexpr int BK = TF32 ? 32 : 64;                     // tokens per pipeline stage
+  static constexpr int MMA_K = 32 / ELEM_BYTES;                 // tokens per MMA instruction: 16 | 8
+  static constexpr int BOX_BYTES = 128 * BK;                    // one box: BK tokens x 128 bytes
+  static constexpr int A_BYTES = (TC_TILE_M / BOX_FEATS) * BOX_BYTES;   // 16 KiB
+  static constexpr int B_BYTES = (TC_TILE_N / BOX_FEATS) * BOX_BYTES;   // 16 KiB
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;                 // 32 KiB
+  static constexpr int K_STEP_BYTES = MMA_K * 128;              // smem advance per MMA: 2048 | 1024
+  // MN-major swizzle atoms: bf16 = 8 tokens x 128 B with 16-byte chunks (descriptor layout 2, TMA
+  // SWIZZLE_128B); tf32 = 4 tokens x 128 B with 32-byte chunks (layout 1, TMA SWIZZLE_128B_ATOM_32B).
+  static constexpr uint32_t DESC_LAYOUT = TF32 ? 1u : 2u;
+  static constexpr uint32_t SBO_BYTES = TF32 ? 512u : 1024u;   // next swizzle atom along the tokens
+};
 constexpr int TC_BAR_BYTES = 256;
-constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + TC_BAR_BYTES + 1024;   // + alignment slack
+constexpr int TC_SMEM_BYTES = TC_STAGES * TcOperand<false>::STAGE_BYTES + TC_BAR_BYTES + 1024;   // + alignment slack
+static_assert(TcOperand<false>::STAGE_BYTES == TcOperand<true>::STAGE_BYTES, "stage size is shared");
 
 // error codes latched in the device status word (which wait gave up)
 enum : int { TC_WAIT_EMPTY = 1, TC_WAIT_FULL = 2, TC_WAIT_ACC_EMPTY = 3, TC_WAIT_ACC_FULL = 4 };
@@ -62,10 +79,12 @@ __device__ __forceinline__ float phi_apply(float g) {
   return g;
 }
 
-template <int PHI>
+template <int PHI, bool TF32>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy, TcParams p) {
   using namespace sm100;
+  using Op = TcOperand<TF32>;
+  constexpr int TC_BK = Op::BK, TC_BOX_BYTES = Op::BOX_BYTES, TC_A_BYTES = Op::A_BYTES, TC_STAGE_BYTES = Op::STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -84,8 +103,6 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   const int b_end = (int)(((long long)p.B * (blockIdx.z + 1)) / p.nsplit);
   const int nb = b_end - b_begin;
   const int nk = (p.T + TC_BK - 1) / TC_BK;                 // stages per example
-  const int n_groups = p.per_example ? nb : (nb > 0 ? 1 : 0);
-  const int group_len = p.per_example ? 1 : nb;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -105,65 +122,86 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   // branch of the role it applies to.
   if (warp < 4) {
     setmaxnreg_dec<TC_REGS_CONTROL>();
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      int s = 0; uint32_t ph = 0;
-      bool ok = true;
-      for (int e = 0; e < nb && ok; ++e) {
-        const int b = b_begin + e;
-        for (int kc = 0; kc < nk; ++kc) {
-          if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_EMPTY)) { ok = false; break; }
-          mbar_arrive_expect_tx(full_bar(s), TC_STAGE_BYTES);
-          const uint32_t a_dst = smem_base + s * TC_STAGE_BYTES;
-          const uint32_t b_dst = a_dst + TC_A_BYTES;
+    if (warp == 0) {
+      // ---------------------------------------------------------- TMA producer
+      // Stages are filled for two examples at a time, alternating between them: stage 2*kc of a pair
+      // belongs to its first example (issuer 0), stage 2*kc+1 to its second (issuer 1).
+      if (lane == 0) {
+        int s = 0; uint32_t ph = 0;
+        bool ok = true;
+        for (int e0 = 0; e0 < nb && ok; e0 += 2) {
+          const int n_in_pair = (e0 + 1 < nb) ? 2 : 1;
+          for (int kc = 0; kc < nk && ok; ++kc) {
+            for (int x = 0; x < n_in_pair; ++x) {
+              if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_EMPTY)) { ok = false; break; }
+              const int b = b_begin + e0 + x;
+              mbar_arrive_expect_tx(full_bar(s), TC_STAGE_BYTES);
+              const uint32_t a_dst = smem_base + s * TC_STAGE_BYTES;
+              const uint32_t b_dst = a_dst + TC_A_BYTES;
 #pragma unroll
-          for (int g = 0; g < TC_TILE_M / 64; ++g)
-            tma_load_3d(a_dst + g * TC_BOX_BYTES, &tmap_dy, full_bar(s), tile_m * TC_TILE_M + g * 64, kc * TC_BK, b);
+              for (int g = 0; g < TC_TILE_M / Op::BOX_FEATS; ++g)
+                tma_load_3d(a_dst + g * TC_BOX_BYTES, &tmap_dy, full_bar(s), tile_m * TC_TILE_M + g * Op::BOX_FEATS, kc * TC_BK, b);
 #pragma unroll
-          for (int g = 0; g < TC_TILE_N / 64; ++g)
-            tma_load_3d(b_dst + g * TC_BOX_BYTES, &tmap_x, full_bar(s), tile_n * TC_TILE_N + g * 64, kc * TC_BK, b);
-          if (++s == TC_STAGES) { s = 0; ph ^= 1u; }
+              for (int g = 0; g < TC_TILE_N / Op::BOX_FEATS; ++g)
+                tma_load_3d(b_dst + g * TC_BOX_BYTES, &tmap_x, full_bar(s), tile_n * TC_TILE_N + g * Op::BOX_FEATS, kc * TC_BK, b);
+              if (++s == TC_STAGES) { s = 0; ph ^= 1u; }
+            }
+          }
         }
       }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16_mn_major(TC_TILE_M, TC_TILE_N);
-      int s = 0; uint32_t ph = 0;
-      bool ok = true;
-      for (int grp = 0; grp < n_groups && ok; ++grp) {
-        const int buf = grp % TC_ACC_BUFS;
-        const uint32_t acc_ph = (uint32_t)(grp / TC_ACC_BUFS) & 1u;
-        if (!mbar_wait_bounded(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_ACC_EMPTY)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * TC_TILE_N);
+    } else if (warp == 1 || warp == 3) {
+      // ---------------------------------------------------------- MMA issuers
+      // Two issuing threads (one per warp).  A thread that has just queued MMAs stalls for a couple of
+      // hundred cycles on its next barrier probe, long enough to drain the tensor pipe; with two
+      // threads working on two different examples (own accumulators, alternate stages) one of them
+      // always has MMAs queued.  Issuer x owns examples x, x+2, ... of the slice and TMEM buffers
+      // 2x and 2x+1.
+      if (lane == 0) {
+        const int x = (warp == 1) ? 0 : 1;
+        constexpr uint32_t idesc = make_idesc_mn_major(TC_TILE_M, TC_TILE_N, TF32);
+        bool ok = true;
         uint32_t accumulate = 0;
-        for (int e = 0; e < group_len && ok; ++e) {
+        int i_local = 0;                                   // examples this issuer has started
+        for (int e = x; e < nb && ok; e += 2, ++i_local) {
+          const int grp = p.per_example ? i_local : 0;
+          const int buf = 2 * x + (grp & 1);
+          if (p.per_example || i_local == 0) {
+            const uint32_t acc_ph = (uint32_t)(grp >> 1) & 1u;
+            if (!mbar_wait_bounded(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_ACC_EMPTY)) { ok = false; break; }
+            tc_fence_after();
+            accumulate = 0;
+          }
+          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * TC_TILE_N);
+          // position of this example's stages in the producer's sequence
+          const int pair = e >> 1;
+          const bool paired = ((e | 1) < nb);              // the pair has two examples
+          const long long n0 = (long long)pair * 2 * nk;
           for (int kc = 0; kc < nk; ++kc) {
+            const long long n = n0 + (paired ? 2 * kc + x : kc);
+            const int s = (int)(n % TC_STAGES);
+            const uint32_t ph = (uint32_t)(n / TC_STAGES) & 1u;
             if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, p.dev_status, TC_WAIT_FULL)) { ok = false; break; }
             tc_fence_after();
             const uint32_t a_src = smem_base + s * TC_STAGE_BYTES;
             const uint32_t b_src = a_src + TC_A_BYTES;
-            const int t_left = p.T - kc * TC_BK;               // tokens of this example still to contract
+            const int t_left = p.T - kc * TC_BK;           // tokens of this example still to contract
 #pragma unroll
-            for (int k = 0; k < TC_BK / 16; ++k) {
-              if (k * 16 < t_left) {                             // rows past T are zero-filled by TMA; whole
-                const uint64_t ad = make_smem_desc_sw128(a_src + k * 2048, TC_BOX_BYTES, 1024);   // 16-token steps past T are skipped
-                const uint64_t bd = make_smem_desc_sw128(b_src + k * 2048, TC_BOX_BYTES, 1024);
-                umma_bf16_ss(d_tmem, ad, bd, idesc, accumulate);
+            for (int k = 0; k < TC_BK / Op::MMA_K; ++k) {
+              // rows past T are zero-filled by TMA; whole MMA steps past T are skipped
+              if (k * Op::MMA_K < t_left) {
+                const uint64_t ad = make_smem_desc(a_src + k * Op::K_STEP_BYTES, TC_BOX_BYTES, Op::SBO_BYTES, Op::DESC_LAYOUT);
+                const uint64_t bd = make_smem_desc(b_src + k * Op::K_STEP_BYTES, TC_BOX_BYTES, Op::SBO_BYTES, Op::DESC_LAYOUT);
+                umma_ss<TF32>(d_tmem, ad, bd, idesc, accumulate);
                 accumulate = 1;
               }
             }
-            umma_commit(empty_bar(s));                           // stage reusable once these MMAs retire
-            if (++s == TC_STAGES) { s = 0; ph ^= 1u; }
+            umma_commit(empty_bar(s));                     // stage reusable once these MMAs retire
           }
+          const bool last_of_group = p.per_example || (e + 2 >= nb);
+          if (ok && last_of_group) umma_commit(acc_full_bar(buf));   // accumulator complete
         }
-        if (ok) umma_commit(acc_full_bar(buf));                  // accumulator of this example complete
       }
     }
-  }
   } else {
     // ------------------------------------------------------------ epilogue
     setmaxnreg_inc<TC_REGS_EPILOGUE>();
@@ -173,9 +211,13 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 #pragma unroll
     for (int j = 0; j < 64; ++j) { acc_stat[j] = 0.f; acc_mean[j] = 0.f; }
     bool ok = true;
-    for (int grp = 0; grp < n_groups; ++grp) {
-      const int buf = grp % TC_ACC_BUFS;
-      const uint32_t acc_ph = (uint32_t)(grp / TC_ACC_BUFS) & 1u;
+    // per-example mode: one accumulator per example, in example order (example e -> issuer e&1).
+    // plain mode: one accumulator per issuer that had work.
+    const int n_acc = p.per_example ? nb : (nb >= 2 ? 2 : nb);
+    for (int a = 0; a < n_acc; ++a) {
+      const int x = a & 1, grp = p.per_example ? (a >> 1) : 0;
+      const int buf = 2 * x + (grp & 1);
+      const uint32_t acc_ph = (uint32_t)(grp >> 1) & 1u;
       if (!mbar_wait_bounded(acc_full_bar(buf), acc_ph, abort_flag, p.dev_status, TC_WAIT_ACC_FULL)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TC_TILE_N + h * 64);
@@ -186,7 +228,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         if (c == 1) {
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(acc_empty_bar(buf));        // buffer free for the next example's MMAs
+          if (lane == 0) mbar_arrive(acc_empty_bar(buf));        // buffer free for the issuer's next example
         }
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
@@ -196,7 +238,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         }
       }
     }
-    if (ok && n_groups > 0) {
+    if (ok && n_acc > 0) {
       const int o = tile_m * TC_TILE_M + q * 32 + lane;
       const int i_base = tile_n * TC_TILE_N + h * 64;
       if (o < p.d_out) {

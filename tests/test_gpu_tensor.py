@@ -27,9 +27,10 @@ def test_structured_single_tile_catches_layout_mistakes():
     X = ((t % 5) - 2 + (torch.arange(d_in).view(1, 1, d_in) % 7 - 3) + torch.arange(B).view(B, 1, 1)).to(torch.bfloat16)
     dY = ((t % 3) - 1 + (torch.arange(d_out).view(1, 1, d_out) % 11 - 5) * 0.5 - torch.arange(B).view(B, 1, 1)).to(torch.bfloat16)
     li = inputs.LayerInputs("structured", X.to(DEV).contiguous(), dY.to(DEV).contiguous())
-    rep = check_all(li, phis=("identity", "square", "sign"), tol=1e-6)
+    rep = check_all(li, phis=("identity", "square", "sign"), token=False, tol=1e-6)
     assert pe.pe_last_path() == pe.PATH_TENSOR
     assert rep["sign_disagreements"] == 0
+    check_all(li, phis=(), token=True)          # 128 rows: too few for bf16 squares, runs on the SIMT kernel
 
 
 @pytest.mark.parametrize("B,T,d_in,d_out", [
@@ -43,8 +44,10 @@ def test_structured_single_tile_catches_layout_mistakes():
 ])
 def test_tensor_small_shapes_full_comparison(B, T, d_in, d_out):
     li = inputs.gaussian_layer(B, T, d_in, d_out, seed=300 + 7 * B + T, device=DEV)
-    check_all(li, phis=("identity", "square", "sign"))
+    check_all(li, phis=("identity", "square", "sign"), token=False)
     assert pe.pe_last_path() == pe.PATH_TENSOR
+    check_all(li, phis=(), token=True)
+    assert pe.pe_last_path() == (pe.PATH_TENSOR if B * T >= 256 else pe.PATH_SIMT)
 
 
 def test_heavy_tailed_and_heterogeneous_small():
@@ -89,8 +92,8 @@ def test_config5_points_sampled_outputs(B, T, d):
 
 
 def test_token_stat_requires_workspace():
-    li = inputs.gaussian_layer(2, 64, 64, 64, seed=44, device=DEV)
+    li = inputs.gaussian_layer(4, 64, 64, 64, seed=44, device=DEV)
     out = torch.empty((64, 64), device=DEV)
     lib = pe.load_library()
-    st = lib.pe_token_sqstats(li.X.data_ptr(), li.dY.data_ptr(), 2, 64, 64, 64, out.data_ptr(), None, 0, None)
+    st = lib.pe_token_sqstats(li.X.data_ptr(), li.dY.data_ptr(), 4, 64, 64, 64, out.data_ptr(), None, 0, None)
     assert st == 9      # PE_ERR_WORKSPACE
