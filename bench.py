@@ -181,6 +181,33 @@ def time_each(torch, fn, iters=20, warmup=3):
     return v[len(v) // 2], v[0]
 
 
+def context_numbers(torch, pe, st, li, peaks, dev):
+    """Per-kernel timings taken alone, outside the timed region: each statistics call, the cuBLAS batch
+    weight-gradient GEMM of the same shape, and the update kernels on a parameter count far beyond L2."""
+    B, T, d_in, d_out = st["shape"]
+    flops_one = 2.0 * B * T * d_in * d_out
+    extra = {}
+    med, best = time_each(torch, lambda i: pe.pe_linear_stats(li.X, li.dY, pe.PHI_SQUARE, st["mean"], st["sq"]))
+    extra["pe_linear_stats_square_us"] = {"median": med * 1e3, "best": best * 1e3, "tflops_median": flops_one / med / 1e9}
+    med_s, best_s = time_each(torch, lambda i: pe.pe_linear_stats(li.X, li.dY, pe.PHI_SIGN, None, st["sgn"]))
+    extra["pe_linear_stats_sign_us"] = {"median": med_s * 1e3, "best": best_s * 1e3, "tflops_median": flops_one / med_s / 1e9}
+    med_t, best_t = time_each(torch, lambda i: pe.pe_token_sqstats(li.X, li.dY, st["tok"], st["ws"]))
+    extra["pe_token_sqstats_us"] = {"median": med_t * 1e3, "best": best_t * 1e3, "tflops_median": flops_one / med_t / 1e9}
+    A2, B2 = li.dY.view(B * T, d_out), li.X.view(B * T, d_in)
+    med_g, best_g = time_each(torch, lambda i: torch.matmul(A2.t(), B2))
+    extra["cublas_wgrad_gemm_us"] = {"median": med_g * 1e3, "best": best_g * 1e3, "tflops_median": flops_one / med_g / 1e9,
+                                     "note": "torch.matmul(dY_flat^T, X_flat), bf16 in and out"}
+    extra["overhead_vs_gemm"] = med / med_g
+    big = 1 << 26       # update kernels on a parameter count far larger than L2 (64 Mi parameters)
+    bufs = [torch.zeros(big, device=dev) for _ in range(5)]
+    lp = torch.empty(big, dtype=torch.bfloat16, device=dev)
+    med_a, _ = time_each(torch, lambda i: pe.microadam_step(bufs[0], bufs[1], bufs[2], bufs[3], bufs[4], B, step=1, theta_lp=lp, **ADAM), iters=10)
+    med_sg, _ = time_each(torch, lambda i: pe.microsignsgd_step(bufs[0], bufs[1], bufs[3], B, theta_lp=lp, **SIGN), iters=10)
+    extra["microadam_step"] = {"params": big, "gbs": 34.0 * big / med_a / 1e6, "frac_of_hbm_peak": 34.0 * big / med_a / 1e6 / peaks["hbm_gbs"]}
+    extra["microsignsgd_step"] = {"params": big, "gbs": 22.0 * big / med_sg / 1e6, "frac_of_hbm_peak": 22.0 * big / med_sg / 1e6 / peaks["hbm_gbs"]}
+    return extra
+
+
 def oracle_sample(inputs, workload, n_rows, n_cols):
     """Column-gathered sub-layer of the workload for the CPU oracle (full B and T)."""
     import numpy as np
@@ -250,6 +277,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quick", action="store_true", help="timed region only: skip the per-kernel context numbers and the CPU baseline")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
@@ -356,27 +384,7 @@ def main():
     # ------------------------------------------------------------ context numbers (rank 0, outside the timed region)
     peaks = measured_peaks()
     li = st["sets"][0]
-    extra = {}
-    med, best = time_each(torch, lambda i: pe.pe_linear_stats(li.X, li.dY, pe.PHI_SQUARE, st["mean"], st["sq"]))
-    extra["pe_linear_stats_square_us"] = {"median": med * 1e3, "best": best * 1e3, "tflops_median": flops_one / med / 1e9}
-    med_s, best_s = time_each(torch, lambda i: pe.pe_linear_stats(li.X, li.dY, pe.PHI_SIGN, None, st["sgn"]))
-    extra["pe_linear_stats_sign_us"] = {"median": med_s * 1e3, "best": best_s * 1e3, "tflops_median": flops_one / med_s / 1e9}
-    med_t, best_t = time_each(torch, lambda i: pe.pe_token_sqstats(li.X, li.dY, st["tok"], st["ws"]))
-    extra["pe_token_sqstats_us"] = {"median": med_t * 1e3, "best": best_t * 1e3, "tflops_median": flops_one / med_t / 1e9}
-    A2, B2 = li.dY.view(B * T, d_out), li.X.view(B * T, d_in)
-    med_g, best_g = time_each(torch, lambda i: torch.matmul(A2.t(), B2))
-    extra["cublas_wgrad_gemm_us"] = {"median": med_g * 1e3, "best": best_g * 1e3, "tflops_median": flops_one / med_g / 1e9,
-                                     "note": "torch.matmul(dY_flat^T, X_flat), bf16 in and out"}
-    extra["overhead_vs_gemm"] = med / med_g
-    n = st["n"]
-    big = 1 << 26       # update kernels on a parameter count far larger than L2 (64 Mi parameters)
-    bufs = [torch.zeros(big, device=dev) for _ in range(5)]
-    lp = torch.empty(big, dtype=torch.bfloat16, device=dev)
-    med_a, _ = time_each(torch, lambda i: pe.microadam_step(bufs[0], bufs[1], bufs[2], bufs[3], bufs[4], B, step=1, theta_lp=lp, **ADAM), iters=10)
-    med_sg, _ = time_each(torch, lambda i: pe.microsignsgd_step(bufs[0], bufs[1], bufs[3], B, theta_lp=lp, **SIGN), iters=10)
-    extra["microadam_step"] = {"params": big, "gbs": 34.0 * big / med_a / 1e6, "frac_of_hbm_peak": 34.0 * big / med_a / 1e6 / peaks["hbm_gbs"]}
-    extra["microsignsgd_step"] = {"params": big, "gbs": 22.0 * big / med_sg / 1e6, "frac_of_hbm_peak": 22.0 * big / med_sg / 1e6 / peaks["hbm_gbs"]}
-    del bufs, lp
+    extra = {} if args.quick else context_numbers(torch, pe, st, li, peaks, dev)
 
     achieved = flops_one / (kernel_ms * 1e-3) / 1e12
     roofline = {"bound": "tensor", "kernel": "tc_stats_kernel<square>", "achieved": achieved, "peak": peaks["bf16_tflops"],
@@ -386,7 +394,7 @@ def main():
                 "algorithmic_bytes_per_launch": 2.0 * B * T * (d_in + d_out) + 8.0 * d_in * d_out}
 
     cpu_baseline = None
-    if not args.no_cpu_baseline and world == 1:
+    if not args.no_cpu_baseline and not args.quick and world == 1:
         import oracle
         if name == "c2":
             Xh, dYh = inputs.to_numpy_bits(li.X), inputs.to_numpy_bits(li.dY)
