@@ -37,6 +37,7 @@ WORKLOADS = {
     # name: (B, T, d_in, d_out, rotating input sets)
     "c2": (64, 256, 512, 2048, 6),
     "c4": (256, 1024, 2048, 8192, 1),
+    "c4s": (16, 1024, 2048, 8192, 1),     # a 16-sequence slice of c4 (335 MB of inputs): small enough to profile
 }
 ADAM = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8)
 SIGN = dict(lr=3.47e-3, beta=0.9)
@@ -123,7 +124,7 @@ def make_state(pe, inputs, torch, name, dev, seed_offset=0):
                                             name="c2", with_weights=(k == 0))
         else:
             li = inputs.heavy_tailed_layer(B, T, d_in, d_out, seed=inputs.BASE_SEED + 4 + 1000 * k + seed_offset, device=dev,
-                                           name="c4", with_weights=(k == 0))
+                                           name=name, with_weights=(k == 0))
         sets.append(li)
     n = d_out * d_in
     f32 = dict(dtype=torch.float32, device=dev)
