@@ -92,6 +92,35 @@ pe_status_t pe_token_sqstats_f32(const float* X, const float* dY, int B, int T, 
 size_t pe_token_sqstats_workspace_bytes(int B, int T, int d_in, int d_out);
 
 /*
+ * pe_token_sqstats for callers that have no device memory to give as workspace and no way to get
+ * some.  (The paper has no counterpart; this is a convenience of this library.)  Typical cases: a
+ * plug-in that is handed input and output pointers but no allocator; a process whose framework
+ * reserved all of the GPU's memory in its own pool at start-up, so that cudaMalloc would fail; a
+ * latency-critical loop that must not pay cudaMalloc / cudaFree's device-wide synchronisation.
+ *
+ * Same arguments, result and path selection as pe_token_sqstats, minus the workspace: the fp32
+ * staging of the squared operands lives in an array of PE_STATIC_SCRATCH_BYTES bytes that is part
+ * of the library's device image, so every GPU on which the library is used holds that much memory
+ * from module load until the process exits.  The call allocates and frees nothing, on the device or
+ * through any library.
+ *
+ * Limit: shapes whose staging (pe_token_sqstats_workspace_bytes) exceeds PE_STATIC_SCRATCH_BYTES
+ * are refused with PE_ERR_WORKSPACE and nothing is enqueued; use pe_token_sqstats with your own
+ * workspace for those.
+ * First call on a device: looks up the array's device address (a host-side query, done once per
+ * device with that device current) before enqueuing; make that first call outside any stream
+ * capture.
+ * Sharing: all calls on a device use the same array and it keeps whatever the previous call left
+ * there.  Each call overwrites the part it reads before reading it, so stale contents never reach
+ * a result; but two calls whose kernels can overlap on the GPU (different streams, no dependency
+ * between them) race on the array and both results are then undefined.  Calls on one stream are
+ * ordered and safe.
+ */
+#define PE_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+pe_status_t pe_token_sqstats_static(const void* X, const void* dY, int B, int T, int d_in, int d_out,
+                                    float* out_stat, pe_stream_t stream);
+
+/*
  * One MicroAdam step over n parameters (Algorithm 1, MicroAdam branch; Eq. (3)):
  *     mu = s*sum_g/B;  nu = s^2*sum_g2/B;   m = beta1*m + (1-beta1)*mu;   v = beta2*v + (1-beta2)*nu
  *     mh = m/(1-beta1^step);  vh = v/(1-beta2^step)

@@ -16,7 +16,7 @@ __all__ = [
     "EXPORTED_SYMBOLS", "library_path", "load_library", "pe_linear_stats", "pe_linear_stats_f32",
     "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_workspace_bytes", "microadam_step",
     "microsignsgd_step", "pe_status_string", "pe_get_async_status", "pe_set_path", "pe_last_path",
-    "pe_launch_count", "pe_reset_launch_count",
+    "pe_launch_count", "pe_reset_launch_count", "pe_token_sqstats_static", "STATIC_SCRATCH_BYTES",
 ]
 
 PHI_IDENTITY, PHI_SQUARE, PHI_SIGN = 0, 1, 2
@@ -28,7 +28,9 @@ EXPORTED_SYMBOLS = [
     "pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32",
     "pe_token_sqstats_workspace_bytes", "microadam_step", "microsignsgd_step", "pe_status_string",
     "pe_get_async_status", "pe_set_path", "pe_last_path", "pe_launch_count", "pe_reset_launch_count",
+    "pe_token_sqstats_static",
 ]
+STATIC_SCRATCH_BYTES = 32 * 1024 * 1024      # PE_STATIC_SCRATCH_BYTES of pestats.h
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libpestats.so")
 _lib = None
@@ -60,6 +62,7 @@ def load_library() -> ctypes.CDLL:
     lib.pe_linear_stats_f32.argtypes = [vp, vp, i, i, i, i, i, vp, vp, vp]
     lib.pe_token_sqstats.argtypes = [vp, vp, i, i, i, i, vp, vp, sz, vp]
     lib.pe_token_sqstats_f32.argtypes = [vp, vp, i, i, i, i, vp, vp]
+    lib.pe_token_sqstats_static.argtypes = [vp, vp, i, i, i, i, vp, vp]
     lib.pe_token_sqstats_workspace_bytes.argtypes = [i, i, i, i]
     lib.pe_token_sqstats_workspace_bytes.restype = sz
     lib.microadam_step.argtypes = [vp, vp, vp, vp, vp, vp, ll, i, f, f, f, f, f, i, f, i, vp]
@@ -73,7 +76,7 @@ def load_library() -> ctypes.CDLL:
     lib.pe_launch_count.restype = ll
     lib.pe_reset_launch_count.argtypes = []
     lib.pe_reset_launch_count.restype = None
-    for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32",
+    for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_static",
                  "microadam_step", "microsignsgd_step", "pe_get_async_status", "pe_set_path", "pe_last_path"):
         getattr(lib, name).restype = i
     _lib = lib
@@ -170,6 +173,23 @@ def pe_token_sqstats(X, dY, out_stat=None, workspace=None):
     with _dev_ctx(X):
         _check("pe_token_sqstats", load_library().pe_token_sqstats(
             X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, out_stat.data_ptr(), _ptr(workspace), ws_bytes, _stream(X)))
+    return out_stat
+
+
+def pe_token_sqstats_static(X, dY, out_stat):
+    """Per-token second moment for callers that cannot supply (or allocate) a workspace: the library's
+    built-in device array of STATIC_SCRATCH_BYTES stages the squared operands, and neither this
+    wrapper nor the library allocates anything, so ``out_stat`` (float32 [d_out, d_in]) is required.
+    Shapes whose staging does not fit raise PestatsError (PE_ERR_WORKSPACE).  Calls that may overlap on
+    the GPU share that array and race; keep them on one stream.  Make the first call on a device
+    outside stream capture (it looks up the array's address)."""
+    B, T, d_in, d_out = _io_check(X, dY, torch.bfloat16)
+    if out_stat is None:
+        raise ValueError("out_stat is required: this entry point allocates nothing")
+    _out_check("out_stat", out_stat, d_out, d_in)
+    with _dev_ctx(X):
+        _check("pe_token_sqstats_static", load_library().pe_token_sqstats_static(
+            X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, out_stat.data_ptr(), _stream(X)))
     return out_stat
 
 

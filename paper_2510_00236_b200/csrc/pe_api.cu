@@ -312,6 +312,51 @@ pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_
                                                 d_in, d_out, 0, nullptr, out_stat, st);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Allocation-free per-token statistic.  The staging buffer is a device array inside this module's
+// image.  In host code its name is only a handle for the runtime's symbol lookups, never a device
+// address: the address each device gave the array is looked up once per device (with that device
+// current) and cached; that looked-up pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_static_scratch[PE_STATIC_SCRATCH_BYTES];
+
+struct StaticScratchSlot {
+  std::atomic<int> ready{0};
+  void* ptr = nullptr;
+};
+static StaticScratchSlot g_static_slot[MAX_DEVICES];
+
+static pe_status_t static_scratch_ptr(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) { cudaGetLastError(); return PE_ERR_CUDA; }
+  StaticScratchSlot& slot = g_static_slot[dev];
+  if (!slot.ready.load(std::memory_order_acquire)) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return PE_ERR_CUDA; }
+    slot.ptr = p;                       // concurrent first calls look up the same address
+    slot.ready.store(1, std::memory_order_release);
+  }
+  *out = slot.ptr;
+  return PE_OK;
+}
+
+pe_status_t pe_token_sqstats_static(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_stat,
+                                    pe_stream_t stream) {
+  if (!out_stat) return PE_ERR_NULL;
+  pe_status_t rc = validate_stats(X, dY, B, T, d_in, d_out, out_stat, nullptr, false, 16);
+  if (rc != PE_OK) return rc;
+  // Refuse what does not fit before touching the device.
+  if (pe_token_sqstats_workspace_bytes(B, T, d_in, d_out) > (size_t)PE_STATIC_SCRATCH_BYTES) return PE_ERR_WORKSPACE;
+  DeviceInfo* di = nullptr;
+  rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  void* scratch = nullptr;
+  rc = static_scratch_ptr(&scratch);
+  if (rc != PE_OK) return rc;
+  // Nothing in the array has to start at zero: the squaring pre-pass rewrites every element the
+  // contraction reads.  Everything below only enqueues kernels and memsets on `stream`.
+  return pe_token_sqstats(X, dY, B, T, d_in, d_out, out_stat, scratch, (size_t)PE_STATIC_SCRATCH_BYTES, stream);
+}
+
 pe_status_t pe_token_sqstats_f32(const float* X, const float* dY, int B, int T, int d_in, int d_out, float* out_stat,
                                  pe_stream_t stream) {
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);

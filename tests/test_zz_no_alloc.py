@@ -1,0 +1,71 @@
+"""The allocation-free per-token entry point, pe_token_sqstats_static.
+
+Some users of this library cannot hand it a workspace: they receive input and output pointers from a
+host application but no allocator, or their framework claimed the whole GPU at start-up, or they sit
+on a path where cudaMalloc's device-wide synchronisation is not acceptable.  For them the library
+carries a fixed 32 MiB device array and an entry point that stages the squared operands there.  This
+test drives that entry point through the C ABI and requires the same answer as pe_token_sqstats
+with a caller-owned workspace, on two consecutive calls that share the array (the second one smaller,
+so anything stale from the first would show), and checks that a shape too large for the array is
+refused on the host.  The file name sorts last so every other test has already run when this one does.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2510_00236_b200 as pe
+from paper_2510_00236_b200 import inputs
+from parity_util import FROB_TOL, rel_frob
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(autouse=True)
+def _auto_path():
+    prev = pe.pe_set_path(pe.PATH_AUTO)
+    yield
+    pe.pe_set_path(prev)
+
+
+def _both_ways(li):
+    B, T, d_in, d_out = li.shape
+    need = pe.pe_token_sqstats_workspace_bytes(B, T, d_in, d_out)
+    assert 0 < need <= pe.STATIC_SCRATCH_BYTES, "shape must take the staged (tensor-core) path and fit the array"
+    want = torch.full((d_out, d_in), float("nan"), device=DEV)
+    pe.pe_token_sqstats(li.X, li.dY, want, torch.empty(need, dtype=torch.uint8, device=DEV))
+    got = torch.full((d_out, d_in), float("nan"), device=DEV)
+    lib = pe.load_library()
+    stream = torch.cuda.current_stream().cuda_stream
+    status = lib.pe_token_sqstats_static(li.X.data_ptr(), li.dY.data_ptr(), B, T, d_in, d_out, got.data_ptr(), stream)
+    assert status == 0, pe.pe_status_string(status)
+    assert pe.pe_last_path() == pe.PATH_TENSOR
+    torch.cuda.synchronize()
+    assert pe.pe_get_async_status(DEV) == (0, 0)
+    return got.cpu().numpy(), want.cpu().numpy()
+
+
+def test_static_scratch_matches_workspace_version_twice_in_a_row():
+    first = inputs.gaussian_layer(12, 128, 264, 392, seed=901, device=DEV)        # 4 MB of staging, ragged tiles
+    second = inputs.heavy_tailed_layer(5, 64, 136, 128, seed=902, device=DEV)     # smaller: reuses the array's front
+    for li in (first, second):
+        got, want = _both_ways(li)
+        assert np.isfinite(got).all()
+        assert rel_frob(got, want) <= FROB_TOL
+        assert np.all(got >= 0)
+    # and the first shape again, now over the second call's leftovers
+    got, want = _both_ways(first)
+    assert rel_frob(got, want) <= FROB_TOL
+
+
+def test_static_scratch_refuses_shapes_beyond_its_size():
+    B, T, d_in, d_out = 64, 256, 512, 2048                                       # needs 168 MB of staging
+    assert pe.pe_token_sqstats_workspace_bytes(B, T, d_in, d_out) > pe.STATIC_SCRATCH_BYTES
+    X = torch.zeros((B, T, d_in), dtype=torch.bfloat16, device=DEV)
+    dY = torch.zeros((B, T, d_out), dtype=torch.bfloat16, device=DEV)
+    out = torch.full((d_out, d_in), 7.0, device=DEV)
+    with pytest.raises(pe.PestatsError) as e:
+        pe.pe_token_sqstats_static(X, dY, out)
+    assert e.value.status == 9                                                   # PE_ERR_WORKSPACE
+    torch.cuda.synchronize()
+    assert torch.all(out == 7.0), "a refused call must enqueue nothing"
