@@ -28,7 +28,7 @@ struct DeviceInfo {
   std::atomic<int> state{0};     // 0 unknown, 1 ready, -1 failed
   int cc_major = 0, sm_count = 0;
   unsigned int* status_ptr = nullptr;
-  bool tc_attr_set[4] = {false, false, false, false};
+  bool tc_attr_set[6] = {false, false, false, false, false, false};
 };
 static DeviceInfo g_dev[MAX_DEVICES];
 
@@ -86,7 +86,7 @@ static pe_status_t check_launch() {
 }
 
 // [B, T, d] row-major (bf16, or fp32 read as tf32) viewed as a 3-D tensor (d, T, B); one box = 128
-// bytes of features x BK tokens of one example, 128-byte swizzled (16-byte chunks for bf16, 32-byte
+// bytes of features x BK tokens (128 for bf16, 64 for fp32) of one example, 128-byte swizzled (16-byte chunks for bf16, 32-byte
 // chunks for fp32: the MN-major tf32 MMA accepts no other layout).  Tokens past T and features past d read as zero.
 static pe_status_t make_operand_map(CUtensorMap* m, const void* base, int B, int T, int d, bool f32) {
   EncodeTiledFn enc = encode_fn();
@@ -94,8 +94,8 @@ static pe_status_t make_operand_map(CUtensorMap* m, const void* base, int B, int
   const cuuint64_t es = f32 ? 4ull : 2ull;
   cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)T, (cuuint64_t)B};
   cuuint64_t strides[2] = {(cuuint64_t)d * es, (cuuint64_t)T * (cuuint64_t)d * es};
-  cuuint32_t box[3] = {(cuuint32_t)(f32 ? TcOperand<true>::BOX_FEATS : TcOperand<false>::BOX_FEATS),
-                       (cuuint32_t)(f32 ? TcOperand<true>::BK : TcOperand<false>::BK), 1u};
+  cuuint32_t box[3] = {(cuuint32_t)(f32 ? TcOperand<true, 128>::BOX_FEATS : TcOperand<false, 128>::BOX_FEATS),
+                       (cuuint32_t)(f32 ? TcOperand<true, 128>::BK : TcOperand<false, 128>::BK), 1u};
   cuuint32_t estr[3] = {1u, 1u, 1u};
   CUresult r = enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, f32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
@@ -141,22 +141,24 @@ static pe_status_t zero_outputs(float* a, float* b, size_t bytes, cudaStream_t s
   return PE_OK;
 }
 
-template <int PHI, bool TF32>
-static pe_status_t launch_tc_inst(DeviceInfo* di, const CUtensorMap& mx, const CUtensorMap& my, const TcParams& p,
+template <int PHI, bool TF32, int NT, bool WITH_MEAN>
+static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& mx, const CUtensorMap& my, const TcParams& p,
                                   dim3 grid, cudaStream_t st) {
-  constexpr int slot = TF32 ? 3 : PHI;
+  constexpr int smem = TcOperand<TF32, NT>::SMEM_BYTES;
   if (!di->tc_attr_set[slot]) {
-    if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES) != cudaSuccess) {
+    if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, WITH_MEAN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
       cudaGetLastError();
       return PE_ERR_CUDA;
     }
     di->tc_attr_set[slot] = true;
   }
-  tc_stats_kernel<PHI, TF32><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(mx, my, p);
+  tc_stats_kernel<PHI, TF32, NT, WITH_MEAN><<<grid, TC_THREADS, smem, st>>>(mx, my, p);
   return check_launch();
 }
 
-// Tensor-core launch.  per_example = 0 runs the plain contraction over all B*T rows.
+// Tensor-core launch.  per_example = 0 runs the plain contraction over all B*T rows (its result goes
+// to whichever of out_mean / out_stat is not NULL).  With per_example = 1 and both outputs wanted the
+// pair tile is 256 x 128 (two running sums per thread); with only out_stat it is 256 x 256.
 static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int B, int T, int d_in, int d_out, int phi,
                              int per_example, float* out_mean, float* out_stat, cudaStream_t st, bool tf32 = false) {
   CUtensorMap mx, my;
@@ -164,9 +166,11 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   if (rc != PE_OK) return rc;
   rc = make_operand_map(&my, dY, B, T, d_out, tf32);
   if (rc != PE_OK) return rc;
-  const int tiles_n = (d_in + TC_TILE_N - 1) / TC_TILE_N, tiles_m = (d_out + TC_TILE_M - 1) / TC_TILE_M;
-  if (tiles_m > 65535) return PE_ERR_DIM;
-  const int ns = choose_nsplit((long long)tiles_n * tiles_m, B, T, di->sm_count, 16);
+  const bool both = per_example && out_mean && out_stat;
+  const int nt = both ? 128 : 256;
+  const int tiles_n = (d_in + nt - 1) / nt, pairs_m = (d_out + TC_PAIR_M - 1) / TC_PAIR_M;
+  if (tiles_n > 65535 || pairs_m > (1 << 29)) return PE_ERR_DIM;
+  const int ns = choose_nsplit((long long)tiles_n * pairs_m, B, T, di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 16);
   if (ns > 1) {
     rc = zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
     if (rc != PE_OK) return rc;
@@ -174,11 +178,15 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   TcParams p;
   p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = per_example;
   p.out_mean = out_mean; p.out_stat = out_stat; p.dev_status = di->status_ptr;
-  dim3 grid(tiles_n, tiles_m, ns);
-  if (tf32) return launch_tc_inst<0, true>(di, mx, my, p, grid, st);
-  if (!per_example || phi == PE_PHI_IDENTITY) return launch_tc_inst<0, false>(di, mx, my, p, grid, st);
-  if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false>(di, mx, my, p, grid, st);
-  return launch_tc_inst<2, false>(di, mx, my, p, grid, st);
+  dim3 grid(2 * pairs_m, tiles_n, ns);
+  if (tf32) return launch_tc_inst<0, true, 256, false>(di, 5, mx, my, p, grid, st);
+  if (!per_example) return launch_tc_inst<0, false, 256, false>(di, 4, mx, my, p, grid, st);
+  if (both) {
+    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, true>(di, 0, mx, my, p, grid, st);
+    return launch_tc_inst<2, false, 128, true>(di, 1, mx, my, p, grid, st);
+  }
+  if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, false>(di, 2, mx, my, p, grid, st);
+  return launch_tc_inst<2, false, 256, false>(di, 3, mx, my, p, grid, st);
 }
 
 template <typename TIn, int MODE>
@@ -235,6 +243,8 @@ static pe_status_t linear_stats_impl(const TIn* X, const TIn* dY, int B, int T, 
         }
         return rc;
       }
+      if (!out_stat)      // only sum_b G_b wanted: the plain contraction
+        return launch_tc(di, X, dY, B, T, d_in, d_out, phi, 0, out_mean, nullptr, st);
       return launch_tc(di, X, dY, B, T, d_in, d_out, phi, 1, out_mean, out_stat, st);
     }
   }
@@ -299,9 +309,9 @@ pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_
     if ((rc = check_launch()) != PE_OK) return rc;
     square_to_tf32_kernel<<<grid_for(ny / 8 + 8, di->sm_count), OPT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(dY), y2, ny);
     if ((rc = check_launch()) != PE_OK) return rc;
-    // B and T only enter through B*T: regroup the rows into 64-token "examples" when possible so
+    // B and T only enter through B*T: regroup the rows into two-stage "examples" when possible so
     // the batch split has many units to balance.
-    constexpr int REGROUP = 2 * TcOperand<true>::BK;
+    constexpr int REGROUP = 2 * TcOperand<true, 256>::BK;
     int Bp = B, Tp = T;
     if (T % REGROUP == 0 && rows / REGROUP < (size_t)(1u << 30)) { Bp = (int)(rows / REGROUP); Tp = REGROUP; }
     g_last_path.store(PE_PATH_TENSOR);

@@ -1,16 +1,30 @@
 // Tensor-core kernel for the sequence-level per-example statistics (Section 2.3; Eq. (2)).
 //
-// One thread block owns a 128 x 128 tile of the [d_out, d_in] output and a contiguous slice of the
-// batch.  For every example of the slice the tile of G_b = dY_b^T X_b is formed by tcgen05 MMAs
-// (bf16 operands staged by TMA in 128-byte-swizzled shared memory, fp32 accumulator in tensor
-// memory), read back by the epilogue warps, passed through phi and added to two register-resident
-// running sums (sum_b phi(G_b) and sum_b G_b).  The per-example tile never leaves the SM.
+// Work unit: a CTA PAIR (a cluster of two thread blocks on two SMs) owns a 256 x NT tile of the
+// [d_out, d_in] output (NT = 128 or 256) and a contiguous slice of the batch.  For every example of
+// the slice the tile of G_b = dY_b^T X_b is formed by pair-wide tcgen05 MMAs (cta_group::2,
+// M = 256: each block supplies 128 rows of dY_b^T and half of the NT rows of X_b^T from its own
+// shared memory and receives its 128 accumulator rows in its own tensor memory), read back by the
+// epilogue warps, passed through phi and added to register-resident running sums (sum_b phi(G_b)
+// and, when asked for, sum_b G_b).  The per-example tile never leaves the SM.  Pairing cuts the
+// operand bytes each SM pulls from L2 per flop; an SM sustains about 70 B/clk from L2, a lone
+// 128 x 128 tile would need 128 B/clk at full tensor rate, a 256 x 128 pair 96, a 256 x 256 pair 64.
 //
-// Warp roles (12 warps):  0 = TMA producer, 1 and 3 = MMA issuers, 2 = TMEM allocator,
-// 4..11 = epilogue (warp w reads TMEM lanes 32*(w%4)..+31, columns 64*((w-4)/4)..+63 of the tile).
-// Two examples are in flight at once, one per issuer, each issuer double-buffering its accumulator
-// in tensor memory (4 x 128 columns in all), so the MMAs of later examples overlap the epilogue of
-// earlier ones.
+//   NT = 128, two running sums per thread (64 + 64 registers)      -- both outputs wanted
+//   NT = 256, one running sum per thread (128 registers)           -- only sum_b phi(G_b) wanted
+//   NT = 256, no running sum (accumulate in tensor memory)         -- plain contraction over all rows
+//
+// Warp roles per block (12 warps): 0 = TMA producer of the dY boxes, 2 = TMEM allocator, then TMA
+// producer of the X boxes, 1 and 3 = MMA issuers (leader block only), 4..11 = epilogue (warp w reads
+// TMEM lanes 32*(w%4)..+31, column half (w-4)/4).  One thread needs on the order of a hundred cycles
+// per TMA instruction, so the boxes are tall (BK tokens, 16 KiB for bf16) and split over two warps.
+// Two examples are in flight at once, one per issuer; the 512 TMEM columns hold 512/NT accumulators,
+// so the MMAs of later examples overlap the epilogue of earlier ones.
+//
+// Barriers.  full[s] lives in the leader block: its producer posts the byte count of BOTH blocks'
+// loads, and the follower's TMA loads credit their bytes to it through the cluster window.
+// empty[s] and acc_full[a] exist in both blocks and are signalled in both by one multicast commit.
+// acc_empty[a] lives in the leader and collects the arrivals of both blocks' epilogue warps.
 //
 // Operand orientation: A = dY_b viewed as M = d_out x K = T and B = X_b viewed as N = d_in x K = T.
 // In global memory the contraction index (the token) is the slow one, so both operands are
@@ -23,37 +37,40 @@
 
 namespace pe {
 
-constexpr int TC_TILE_M = 128;    // d_out rows per tile   (MMA M)
-constexpr int TC_TILE_N = 128;    // d_in columns per tile (MMA N)
-constexpr int TC_STAGES = 6;
-constexpr int TC_ACC_BUFS = 4;    // TMEM accumulator ring
-constexpr int TC_TMEM_COLS = TC_ACC_BUFS * TC_TILE_N;   // 512
+constexpr int TC_TILE_M = 128;    // d_out rows per block (the pair covers 256)
+constexpr int TC_PAIR_M = 2 * TC_TILE_M;
+constexpr int TC_TMEM_COLS = 512;
 constexpr int TC_THREADS = 384;
 constexpr int TC_REGS_CONTROL = 64;     // setmaxnreg of warps 0..3
 constexpr int TC_REGS_EPILOGUE = 216;   // setmaxnreg of warps 4..11  (4*32*64 + 8*32*216 = 63488 <= 65536)
+constexpr int TC_BAR_BYTES = 512;
+constexpr int TC_SMEM_BUDGET = 200 * 1024;   // operand ring; leaves room for barriers and alignment slack
 
 // Operand element type of the MMA.  bf16 (kind::f16, 16 tokens per instruction) for the per-example
 // statistics; tf32 (kind::tf32, fp32 storage, 8 tokens per instruction) for the per-token statistic,
-// whose squared operands need more than bf16's 8 significant bits.
-template <bool TF32>
+// whose squared operands need more than bf16's 8 significant bits.  NT = d_in columns per pair tile.
+template <bool TF32, int NT>
 struct TcOperand {
   static constexpr int ELEM_BYTES = TF32 ? 4 : 2;
   static constexpr int BOX_FEATS = 128 / ELEM_BYTES;            // features per 128-byte swizzle row: 64 | 32
-  static constexpr int BK = TF32 ? 32 : 64;                     // tokens per pipeline stage
+  static constexpr int BK = TF32 ? 64 : 128;                    // tokens per pipeline stage (one TMA box is BK tokens tall)
   static constexpr int MMA_K = 32 / ELEM_BYTES;                 // tokens per MMA instruction: 16 | 8
   static constexpr int BOX_BYTES = 128 * BK;                    // one box: BK tokens x 128 bytes
-  static constexpr int A_BYTES = (TC_TILE_M / BOX_FEATS) * BOX_BYTES;   // 16 KiB
-  static constexpr int B_BYTES = (TC_TILE_N / BOX_FEATS) * BOX_BYTES;   // 16 KiB
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;                 // 32 KiB
+  static constexpr int A_BOXES = TC_TILE_M / BOX_FEATS;         // this block's 128 rows of dY^T
+  static constexpr int B_FEATS = NT / 2;                        // this block's half of the tile's d_in columns
+  static constexpr int B_BOXES = B_FEATS / BOX_FEATS;
+  static constexpr int A_BYTES = A_BOXES * BOX_BYTES;           // 32 KiB
+  static constexpr int B_BYTES = B_BOXES * BOX_BYTES;           // 16 | 32 KiB
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;         // per block
+  static constexpr int STAGES = TC_SMEM_BUDGET / STAGE_BYTES;   // 4 | 3
   static constexpr int K_STEP_BYTES = MMA_K * 128;              // smem advance per MMA: 2048 | 1024
+  static constexpr int ACC_BUFS = TC_TMEM_COLS / NT;            // 4 | 2 accumulators in tensor memory
   // MN-major swizzle atoms: bf16 = 8 tokens x 128 B with 16-byte chunks (descriptor layout 2, TMA
   // SWIZZLE_128B); tf32 = 4 tokens x 128 B with 32-byte chunks (layout 1, TMA SWIZZLE_128B_ATOM_32B).
   static constexpr uint32_t DESC_LAYOUT = TF32 ? 1u : 2u;
   static constexpr uint32_t SBO_BYTES = TF32 ? 512u : 1024u;   // next swizzle atom along the tokens
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + TC_BAR_BYTES + 1024;   // + alignment slack
 };
-constexpr int TC_BAR_BYTES = 256;
-constexpr int TC_SMEM_BYTES = TC_STAGES * TcOperand<false>::STAGE_BYTES + TC_BAR_BYTES + 1024;   // + alignment slack
-static_assert(TcOperand<false>::STAGE_BYTES == TcOperand<true>::STAGE_BYTES, "stage size is shared");
 
 // error codes latched in the device status word (which wait gave up)
 enum : int { TC_WAIT_EMPTY = 1, TC_WAIT_FULL = 2, TC_WAIT_ACC_EMPTY = 3, TC_WAIT_ACC_FULL = 4 };
@@ -79,54 +96,66 @@ __device__ __forceinline__ float phi_apply(float g) {
   return g;
 }
 
-template <int PHI, bool TF32>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+// gridDim = (2 * ceil(d_out / 256), ceil(d_in / NT), nsplit); blockIdx.x = 2 * pair row + rank in pair.
+// WITH_MEAN: keep the running sum of G_b as well (requires NT = 128).
+template <int PHI, bool TF32, int NT, bool WITH_MEAN>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy, TcParams p) {
   using namespace sm100;
-  using Op = TcOperand<TF32>;
-  constexpr int TC_BK = Op::BK, TC_BOX_BYTES = Op::BOX_BYTES, TC_A_BYTES = Op::A_BYTES, TC_STAGE_BYTES = Op::STAGE_BYTES;
+  using Op = TcOperand<TF32, NT>;
+  static_assert(!WITH_MEAN || NT == 128, "two running sums only fit the registers at NT = 128");
+  constexpr int STAGES = Op::STAGES, ACC_BUFS = Op::ACC_BUFS, BK = Op::BK;
+  constexpr int BOX_BYTES = Op::BOX_BYTES, A_BYTES = Op::A_BYTES, STAGE_BYTES = Op::STAGE_BYTES;
+  constexpr int BUFS_PER_ISSUER = ACC_BUFS / 2;     // 2 | 1
+  constexpr int COLS = NT / 2;                      // accumulator columns per epilogue thread
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t bar_base = smem_base + TC_STAGES * TC_STAGE_BYTES;
+  const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (TC_STAGES + s); };
-  auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * TC_STAGES + a); };
-  auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * TC_STAGES + TC_ACC_BUFS + a); };
-  uint8_t* tail = smem_gen + TC_STAGES * TC_STAGE_BYTES + 8 * (2 * TC_STAGES + 2 * TC_ACC_BUFS);
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + ACC_BUFS + a); };
+  static_assert(8 * (2 * STAGES + 2 * ACC_BUFS) + 16 <= TC_BAR_BYTES, "barrier area too small");
+  uint8_t* tail = smem_gen + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 2 * ACC_BUFS);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile_n = blockIdx.x, tile_m = blockIdx.y;
+  const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair
+  const int tile_m = blockIdx.x;                    // 128-row tile of d_out (pair row = blockIdx.x / 2)
+  const int tile_n = blockIdx.y;                    // NT-column tile of d_in
   const int b_begin = (int)(((long long)p.B * blockIdx.z) / p.nsplit);
   const int b_end = (int)(((long long)p.B * (blockIdx.z + 1)) / p.nsplit);
   const int nb = b_end - b_begin;
-  const int nk = (p.T + TC_BK - 1) / TC_BK;                 // stages per example
+  const int nk = (p.T + BK - 1) / BK;               // stages per example
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < TC_ACC_BUFS; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 8); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < ACC_BUFS; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 16); }
     *abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == 0 && lane == 0) { prefetch_tensormap(&tmap_x); prefetch_tensormap(&tmap_dy); }
-  if (warp == 2) { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TC_TMEM_COLS); tmem_relinquish(); }
+  if (warp == 2) { tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), TC_TMEM_COLS); tmem_relinquish_pair(); }
   tc_fence_before();
-  __syncthreads();
+  cluster_sync_all();          // barriers of both blocks initialised before any remote arrival
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // Register budget: the epilogue warpgroups hold two 64-float running sums plus a 32-register TMEM
+  // Register budget: the epilogue warpgroups hold 128 floats of running sums plus a 32-register TMEM
   // read per thread; the producer / MMA warpgroup needs little.  Each setmaxnreg sits inside the
   // branch of the role it applies to.
   if (warp < 4) {
     setmaxnreg_dec<TC_REGS_CONTROL>();
-    if (warp == 0) {
-      // ---------------------------------------------------------- TMA producer
+    if (warp == 0 || warp == 2) {
+      // ---------------------------------------------------------- TMA producers (both blocks)
+      // Warp 0 loads this block's rows of dY^T (and, in the leader, posts the stage's byte count);
+      // warp 2 loads this block's half of the X^T rows.  Both wait for the same "stage empty" phase.
       // Stages are filled for two examples at a time, alternating between them: stage 2*kc of a pair
-      // belongs to its first example (issuer 0), stage 2*kc+1 to its second (issuer 1).
+      // of examples belongs to its first example (issuer 0), stage 2*kc+1 to its second (issuer 1).
       if (lane == 0) {
+        const bool is_a = (warp == 0);
+        prefetch_tensormap(is_a ? &tmap_dy : &tmap_x);
         int s = 0; uint32_t ph = 0;
         bool ok = true;
         for (int e0 = 0; e0 < nb && ok; e0 += 2) {
@@ -135,121 +164,134 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             for (int x = 0; x < n_in_pair; ++x) {
               if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_EMPTY)) { ok = false; break; }
               const int b = b_begin + e0 + x;
-              mbar_arrive_expect_tx(full_bar(s), TC_STAGE_BYTES);
-              const uint32_t a_dst = smem_base + s * TC_STAGE_BYTES;
-              const uint32_t b_dst = a_dst + TC_A_BYTES;
+              if (is_a && rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);     // both blocks' bytes
+              const uint32_t leader_full = map_to_cta(full_bar(s), 0);
+              const uint32_t a_dst = smem_base + s * STAGE_BYTES;
+              const uint32_t b_dst = a_dst + A_BYTES;
+              if (is_a) {
 #pragma unroll
-              for (int g = 0; g < TC_TILE_M / Op::BOX_FEATS; ++g)
-                tma_load_3d(a_dst + g * TC_BOX_BYTES, &tmap_dy, full_bar(s), tile_m * TC_TILE_M + g * Op::BOX_FEATS, kc * TC_BK, b);
+                for (int g = 0; g < Op::A_BOXES; ++g)
+                  tma_load_3d_pair(a_dst + g * BOX_BYTES, &tmap_dy, leader_full, tile_m * TC_TILE_M + g * Op::BOX_FEATS, kc * BK, b);
+              } else {
 #pragma unroll
-              for (int g = 0; g < TC_TILE_N / Op::BOX_FEATS; ++g)
-                tma_load_3d(b_dst + g * TC_BOX_BYTES, &tmap_x, full_bar(s), tile_n * TC_TILE_N + g * Op::BOX_FEATS, kc * TC_BK, b);
-              if (++s == TC_STAGES) { s = 0; ph ^= 1u; }
+                for (int g = 0; g < Op::B_BOXES; ++g)
+                  tma_load_3d_pair(b_dst + g * BOX_BYTES, &tmap_x, leader_full,
+                                   tile_n * NT + (int)rank * Op::B_FEATS + g * Op::BOX_FEATS, kc * BK, b);
+              }
+              if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
           }
         }
       }
-    } else if (warp == 1 || warp == 3) {
-      // ---------------------------------------------------------- MMA issuers
-      // Two issuing threads (one per warp).  A thread that has just queued MMAs stalls for a couple of
-      // hundred cycles on its next barrier probe, long enough to drain the tensor pipe; with two
-      // threads working on two different examples (own accumulators, alternate stages) one of them
-      // always has MMAs queued.  Issuer x owns examples x, x+2, ... of the slice and TMEM buffers
-      // 2x and 2x+1.
+      __syncwarp();
+    } else if (rank == 0) {
+      // ---------------------------------------------------------- MMA issuers (leader block, warps 1 and 3)
+      // Two issuing threads (one per warp).  A barrier probe right after queuing MMAs costs the
+      // issuing thread a couple of hundred cycles; with two threads working on two different examples
+      // (own accumulators, alternate stages) one of them always has MMAs queued.  Issuer x owns
+      // examples x, x+2, ... of the slice and TMEM buffers x*BUFS_PER_ISSUER .. +BUFS_PER_ISSUER-1.
       if (lane == 0) {
         const int x = (warp == 1) ? 0 : 1;
-        constexpr uint32_t idesc = make_idesc_mn_major(TC_TILE_M, TC_TILE_N, TF32);
+        constexpr uint32_t idesc = make_idesc_mn_major(TC_PAIR_M, NT, TF32);
         bool ok = true;
         uint32_t accumulate = 0;
         int i_local = 0;                                   // examples this issuer has started
         for (int e = x; e < nb && ok; e += 2, ++i_local) {
           const int grp = p.per_example ? i_local : 0;
-          const int buf = 2 * x + (grp & 1);
+          const int buf = BUFS_PER_ISSUER * x + (grp % BUFS_PER_ISSUER);
           if (p.per_example || i_local == 0) {
-            const uint32_t acc_ph = (uint32_t)(grp >> 1) & 1u;
+            const uint32_t acc_ph = (uint32_t)(grp / BUFS_PER_ISSUER) & 1u;
             if (!mbar_wait_bounded(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_ACC_EMPTY)) { ok = false; break; }
             tc_fence_after();
             accumulate = 0;
           }
-          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * TC_TILE_N);
+          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * NT);
           // position of this example's stages in the producer's sequence
           const int pair = e >> 1;
           const bool paired = ((e | 1) < nb);              // the pair has two examples
           const long long n0 = (long long)pair * 2 * nk;
           for (int kc = 0; kc < nk; ++kc) {
             const long long n = n0 + (paired ? 2 * kc + x : kc);
-            const int s = (int)(n % TC_STAGES);
-            const uint32_t ph = (uint32_t)(n / TC_STAGES) & 1u;
+            const int s = (int)(n % STAGES);
+            const uint32_t ph = (uint32_t)(n / STAGES) & 1u;
             if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, p.dev_status, TC_WAIT_FULL)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t a_src = smem_base + s * TC_STAGE_BYTES;
-            const uint32_t b_src = a_src + TC_A_BYTES;
-            const int t_left = p.T - kc * TC_BK;           // tokens of this example still to contract
+            const uint32_t a_src = smem_base + s * STAGE_BYTES;
+            const uint32_t b_src = a_src + A_BYTES;
+            const int t_left = p.T - kc * BK;              // tokens of this example still to contract
 #pragma unroll
-            for (int k = 0; k < TC_BK / Op::MMA_K; ++k) {
+            for (int k = 0; k < BK / Op::MMA_K; ++k) {
               // rows past T are zero-filled by TMA; whole MMA steps past T are skipped
               if (k * Op::MMA_K < t_left) {
-                const uint64_t ad = make_smem_desc(a_src + k * Op::K_STEP_BYTES, TC_BOX_BYTES, Op::SBO_BYTES, Op::DESC_LAYOUT);
-                const uint64_t bd = make_smem_desc(b_src + k * Op::K_STEP_BYTES, TC_BOX_BYTES, Op::SBO_BYTES, Op::DESC_LAYOUT);
-                umma_ss<TF32>(d_tmem, ad, bd, idesc, accumulate);
+                const uint64_t ad = make_smem_desc(a_src + k * Op::K_STEP_BYTES, BOX_BYTES, Op::SBO_BYTES, Op::DESC_LAYOUT);
+                const uint64_t bd = make_smem_desc(b_src + k * Op::K_STEP_BYTES, BOX_BYTES, Op::SBO_BYTES, Op::DESC_LAYOUT);
+                umma_ss_pair<TF32>(d_tmem, ad, bd, idesc, accumulate);
                 accumulate = 1;
               }
             }
-            umma_commit(empty_bar(s));                     // stage reusable once these MMAs retire
+            umma_commit_pair(empty_bar(s));                // stage reusable in both blocks once these MMAs retire
           }
           const bool last_of_group = p.per_example || (e + 2 >= nb);
-          if (ok && last_of_group) umma_commit(acc_full_bar(buf));   // accumulator complete
+          if (ok && last_of_group) umma_commit_pair(acc_full_bar(buf));   // accumulator complete, both blocks
         }
       }
+      __syncwarp();
     }
   } else {
-    // ------------------------------------------------------------ epilogue
+    // ------------------------------------------------------------ epilogue (both blocks)
     setmaxnreg_inc<TC_REGS_EPILOGUE>();
     const int q = warp & 3;                 // TMEM lane quadrant this warp may access
     const int h = (warp - 4) >> 2;          // column half of the tile
-    float acc_stat[64], acc_mean[64];
+    constexpr bool KEEP_MEAN = WITH_MEAN || PHI == 0;
+    constexpr int N_STAT = (PHI != 0) ? COLS : 1;
+    constexpr int N_MEAN = KEEP_MEAN ? COLS : 1;
+    float acc_stat[N_STAT], acc_mean[N_MEAN];
 #pragma unroll
-    for (int j = 0; j < 64; ++j) { acc_stat[j] = 0.f; acc_mean[j] = 0.f; }
+    for (int j = 0; j < N_STAT; ++j) acc_stat[j] = 0.f;
+#pragma unroll
+    for (int j = 0; j < N_MEAN; ++j) acc_mean[j] = 0.f;
     bool ok = true;
     // per-example mode: one accumulator per example, in example order (example e -> issuer e&1).
     // plain mode: one accumulator per issuer that had work.
     const int n_acc = p.per_example ? nb : (nb >= 2 ? 2 : nb);
     for (int a = 0; a < n_acc; ++a) {
       const int x = a & 1, grp = p.per_example ? (a >> 1) : 0;
-      const int buf = 2 * x + (grp & 1);
-      const uint32_t acc_ph = (uint32_t)(grp >> 1) & 1u;
+      const int buf = BUFS_PER_ISSUER * x + (grp % BUFS_PER_ISSUER);
+      const uint32_t acc_ph = (uint32_t)(grp / BUFS_PER_ISSUER) & 1u;
       if (!mbar_wait_bounded(acc_full_bar(buf), acc_ph, abort_flag, p.dev_status, TC_WAIT_ACC_FULL)) { ok = false; break; }
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TC_TILE_N + h * 64);
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * NT + h * COLS);
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      for (int c = 0; c < COLS / 32; ++c) {
         uint32_t r[32];
         tmem_ld_32x32b_x32_wait(taddr + c * 32, r);
-        if (c == 1) {
+        if (c == COLS / 32 - 1) {
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(acc_empty_bar(buf));        // buffer free for the issuer's next example
+          if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));   // buffer free for the issuer's next example
         }
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const float g = __uint_as_float(r[j]);
-          acc_mean[c * 32 + j] += g;
+          if (KEEP_MEAN) acc_mean[c * 32 + j] += g;
           if (PHI != 0) acc_stat[c * 32 + j] += phi_apply<PHI>(g);
         }
       }
     }
     if (ok && n_acc > 0) {
       const int o = tile_m * TC_TILE_M + q * 32 + lane;
-      const int i_base = tile_n * TC_TILE_N + h * 64;
+      const int i_base = tile_n * NT + h * COLS;
       if (o < p.d_out) {
-        float* mrow = p.out_mean ? p.out_mean + (size_t)o * p.d_in : nullptr;
+        float* mrow = (KEEP_MEAN && p.out_mean) ? p.out_mean + (size_t)o * p.d_in : nullptr;
         float* srow = p.out_stat ? p.out_stat + (size_t)o * p.d_in : nullptr;
 #pragma unroll
-        for (int j = 0; j < 64; j += 4) {
+        for (int j = 0; j < COLS; j += 4) {
           const int i = i_base + j;
           if (i < p.d_in) {                                      // d_in % 8 == 0: a group of 4 is all in or all out
-            float4 vm = make_float4(acc_mean[j], acc_mean[j + 1], acc_mean[j + 2], acc_mean[j + 3]);
-            float4 vs = (PHI != 0) ? make_float4(acc_stat[j], acc_stat[j + 1], acc_stat[j + 2], acc_stat[j + 3]) : vm;
+            float4 vm = make_float4(0.f, 0.f, 0.f, 0.f), vs;
+            if (KEEP_MEAN) vm = make_float4(acc_mean[j], acc_mean[j + 1], acc_mean[j + 2], acc_mean[j + 3]);
+            if (PHI != 0) vs = make_float4(acc_stat[j], acc_stat[j + 1], acc_stat[j + 2], acc_stat[j + 3]);
+            else vs = vm;
             if (p.nsplit == 1) {
               if (mrow) *reinterpret_cast<float4*>(mrow + i) = vm;
               if (srow) *reinterpret_cast<float4*>(srow + i) = vs;
@@ -271,9 +313,11 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     // time (bounded) before the block exits and its shared memory is handed to another block.
     const long long t0 = clock64();
     while (clock64() - t0 < (1ll << 22)) __nanosleep(1000);
-    __syncthreads();
   }
-  if (warp == 2) { tc_fence_after(); tmem_dealloc(tmem_base, TC_TMEM_COLS); }
+  // Neither block may leave while its peer can still arrive on its barriers or read its shared memory.
+  __syncwarp();
+  cluster_sync_all();
+  if (warp == 2) { tc_fence_after(); tmem_dealloc_pair(tmem_base, TC_TMEM_COLS); }
 }
 
 }  // namespace pe
