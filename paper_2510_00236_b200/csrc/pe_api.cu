@@ -86,16 +86,15 @@ static pe_status_t check_launch() {
 }
 
 // [B, T, d] row-major (bf16, or fp32 read as tf32) viewed as a 3-D tensor (d, T, B); one box = 128
-// bytes of features x BK tokens (128 for bf16, 64 for fp32) of one example, 128-byte swizzled (16-byte chunks for bf16, 32-byte
+// bytes of features x one pipeline stage of tokens of one example, 128-byte swizzled (16-byte chunks for bf16, 32-byte
 // chunks for fp32: the MN-major tf32 MMA accepts no other layout).  Tokens past T and features past d read as zero.
-static pe_status_t make_operand_map(CUtensorMap* m, const void* base, int B, int T, int d, bool f32) {
+static pe_status_t make_operand_map(CUtensorMap* m, const void* base, int B, int T, int d, bool f32, int box_feats, int box_tokens) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return PE_ERR_CUDA;
   const cuuint64_t es = f32 ? 4ull : 2ull;
   cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)T, (cuuint64_t)B};
   cuuint64_t strides[2] = {(cuuint64_t)d * es, (cuuint64_t)T * (cuuint64_t)d * es};
-  cuuint32_t box[3] = {(cuuint32_t)(f32 ? TcOperand<true, 128>::BOX_FEATS : TcOperand<false, 128>::BOX_FEATS),
-                       (cuuint32_t)(f32 ? TcOperand<true, 128>::BK : TcOperand<false, 128>::BK), 1u};
+  cuuint32_t box[3] = {(cuuint32_t)box_feats, (cuuint32_t)box_tokens, 1u};
   cuuint32_t estr[3] = {1u, 1u, 1u};
   CUresult r = enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, f32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
@@ -161,13 +160,15 @@ static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& m
 // pair tile is 256 x 128 (two running sums per thread); with only out_stat it is 256 x 256.
 static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int B, int T, int d_in, int d_out, int phi,
                              int per_example, float* out_mean, float* out_stat, cudaStream_t st, bool tf32 = false) {
-  CUtensorMap mx, my;
-  pe_status_t rc = make_operand_map(&mx, X, B, T, d_in, tf32);
-  if (rc != PE_OK) return rc;
-  rc = make_operand_map(&my, dY, B, T, d_out, tf32);
-  if (rc != PE_OK) return rc;
   const bool both = per_example && out_mean && out_stat;
   const int nt = both ? 128 : 256;
+  const int box_feats = tf32 ? TcOperand<true, 256>::BOX_FEATS : TcOperand<false, 256>::BOX_FEATS;
+  const int box_tokens = tf32 ? TcOperand<true, 256>::BK : (both ? TcOperand<false, 128>::BK : TcOperand<false, 256>::BK);
+  CUtensorMap mx, my;
+  pe_status_t rc = make_operand_map(&mx, X, B, T, d_in, tf32, box_feats, box_tokens);
+  if (rc != PE_OK) return rc;
+  rc = make_operand_map(&my, dY, B, T, d_out, tf32, box_feats, box_tokens);
+  if (rc != PE_OK) return rc;
   const int tiles_n = (d_in + nt - 1) / nt, pairs_m = (d_out + TC_PAIR_M - 1) / TC_PAIR_M;
   if (tiles_n > 65535 || pairs_m > (1 << 29)) return PE_ERR_DIM;
   const int ns = choose_nsplit((long long)tiles_n * pairs_m, B, T, di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 16);

@@ -53,16 +53,20 @@ template <bool TF32, int NT>
 struct TcOperand {
   static constexpr int ELEM_BYTES = TF32 ? 4 : 2;
   static constexpr int BOX_FEATS = 128 / ELEM_BYTES;            // features per 128-byte swizzle row: 64 | 32
-  static constexpr int BK = TF32 ? 64 : 128;                    // tokens per pipeline stage (one TMA box is BK tokens tall)
+  // tokens per pipeline stage (one TMA box is BK tokens tall), chosen so that the ring has an EVEN
+  // number of stages: with two MMA issuers taking alternate stages every slot then always belongs
+  // to the same issuer (see the parity note at the issuer's wait).
+  static constexpr int BK = TF32 ? 32 : (NT == 128 ? 128 : 64);
   static constexpr int MMA_K = 32 / ELEM_BYTES;                 // tokens per MMA instruction: 16 | 8
   static constexpr int BOX_BYTES = 128 * BK;                    // one box: BK tokens x 128 bytes
   static constexpr int A_BOXES = TC_TILE_M / BOX_FEATS;         // this block's 128 rows of dY^T
   static constexpr int B_FEATS = NT / 2;                        // this block's half of the tile's d_in columns
   static constexpr int B_BOXES = B_FEATS / BOX_FEATS;
-  static constexpr int A_BYTES = A_BOXES * BOX_BYTES;           // 32 KiB
-  static constexpr int B_BYTES = B_BOXES * BOX_BYTES;           // 16 | 32 KiB
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;         // per block
-  static constexpr int STAGES = TC_SMEM_BUDGET / STAGE_BYTES;   // 4 | 3
+  static constexpr int A_BYTES = A_BOXES * BOX_BYTES;           // 32 KiB (NT = 128) | 16 KiB
+  static constexpr int B_BYTES = B_BOXES * BOX_BYTES;           // 16 KiB
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;         // per block: 48 KiB | 32 KiB
+  static constexpr int STAGES = TC_SMEM_BUDGET / STAGE_BYTES;   // 4 | 6
+  static_assert(STAGES % 2 == 0, "slots must alternate between the two issuers");
   static constexpr int K_STEP_BYTES = MMA_K * 128;              // smem advance per MMA: 2048 | 1024
   static constexpr int ACC_BUFS = TC_TMEM_COLS / NT;            // 4 | 2 accumulators in tensor memory
   // MN-major swizzle atoms: bf16 = 8 tokens x 128 B with 16-byte chunks (descriptor layout 2, TMA
@@ -214,6 +218,14 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             const long long n = n0 + (paired ? 2 * kc + x : kc);
             const int s = (int)(n % STAGES);
             const uint32_t ph = (uint32_t)(n / STAGES) & 1u;
+            // A parity wait is only meaningful when the waiter is at most one phase away from the
+            // barrier.  Slots of this issuer's own parity are waited on phase after phase, so that
+            // holds.  In an unpaired last example the issuer also consumes the other issuer's slots;
+            // there it first makes sure the slot's previous phase (the other issuer's data) has
+            // landed, otherwise a slot still in that phase would satisfy the wait for the next one.
+            if (!paired && ((s & 1) != x) && n >= STAGES) {
+              if (!mbar_wait_bounded(full_bar(s), ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_FULL)) { ok = false; break; }
+            }
             if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, p.dev_status, TC_WAIT_FULL)) { ok = false; break; }
             tc_fence_after();
             const uint32_t a_src = smem_base + s * STAGE_BYTES;

@@ -50,6 +50,43 @@ def test_tensor_small_shapes_full_comparison(B, T, d_in, d_out):
     assert pe.pe_last_path() == (pe.PATH_TENSOR if B * T >= 256 else pe.PATH_SIMT)
 
 
+@pytest.mark.parametrize("B,T,d_in,d_out", [(5, 200, 136, 264), (9, 16, 320, 192), (33, 300, 520, 264), (2, 1, 64, 72)])
+def test_single_output_calls_use_the_wide_tile_and_match(B, T, d_in, d_out):
+    """Asking for only sum_b phi(G_b) (or only sum_b G_b) takes the 256 x 256 pair tile (or the plain
+    contraction); both must agree with the oracle like the two-output call does."""
+    from parity_util import FROB_TOL, check_sign, oracle_on, rel_frob
+    li = inputs.gaussian_layer(B, T, d_in, d_out, seed=900 + B, device=DEV)
+    st, _ = oracle_on(li)
+    for phi in ("square", "sign"):
+        stat = torch.full((d_out, d_in), float("nan"), device=DEV)
+        pe.pe_linear_stats(li.X, li.dY, phi, None, stat)
+        mean = torch.full((d_out, d_in), float("nan"), device=DEV)
+        pe.pe_linear_stats(li.X, li.dY, phi, mean, None)
+        torch.cuda.synchronize()
+        assert rel_frob(mean.cpu().numpy(), st.sum_g) <= FROB_TOL
+        if phi == "square":
+            assert rel_frob(stat.cpu().numpy(), st.sum_g2) <= FROB_TOL
+        else:
+            check_sign(stat.cpu().numpy(), st)
+    assert pe.pe_get_async_status(DEV) == (0, 0)
+
+
+def test_odd_batch_slices_and_long_sequences_single_output():
+    """An odd number of examples per slice ends on an unpaired example whose stages run through both
+    issuers' slots; long sequences make that tail many stages long."""
+    from parity_util import FROB_TOL, check_sign, oracle_on, rel_frob
+    li = inputs.gaussian_layer(3, 2000, 264, 520, seed=77, device=DEV)
+    st, tok = oracle_on(li)
+    for both in (True, False):
+        stat = torch.full((520, 264), float("nan"), device=DEV)
+        mean = torch.full((520, 264), float("nan"), device=DEV) if both else None
+        pe.pe_linear_stats(li.X, li.dY, "square", mean, stat)
+        torch.cuda.synchronize()
+        assert rel_frob(stat.cpu().numpy(), st.sum_g2) <= FROB_TOL
+    assert rel_frob(pe.pe_token_sqstats(li.X, li.dY).cpu().numpy(), tok) <= FROB_TOL
+    assert pe.pe_get_async_status(DEV) == (0, 0)
+
+
 def test_heavy_tailed_and_heterogeneous_small():
     check_all(inputs.heavy_tailed_layer(12, 128, 256, 384, seed=41, device=DEV))
     check_all(inputs.heterogeneous_layer(20, 64, 128, 256, seed=42, device=DEV))
