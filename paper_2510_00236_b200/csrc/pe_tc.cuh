@@ -156,7 +156,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       // Warp 0 loads this block's rows of dY^T (and, in the leader, posts the stage's byte count);
       // warp 2 loads this block's half of the X^T rows.  Both wait for the same "stage empty" phase.
       // Stages are filled for two examples at a time, alternating between them: stage 2*kc of a pair
-      // of examples belongs to its first example (issuer 0), stage 2*kc+1 to its second (issuer 1).
+      // of examples belongs to its first example (issuer 0, even slots), stage 2*kc+1 to its second
+      // (issuer 1, odd slots); the ring has an even number of slots.
       if (lane == 0) {
         const bool is_a = (warp == 0);
         prefetch_tensormap(is_a ? &tmap_dy : &tmap_x);
@@ -184,6 +185,9 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
               }
               if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
+            // An unpaired last example leaves the second issuer's slot of every step unused, so
+            // that each slot is only ever consumed by the issuer of its own parity.
+            if (n_in_pair == 1) { if (++s == STAGES) { s = 0; ph ^= 1u; } }
           }
         }
       }
@@ -211,21 +215,14 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
           }
           const uint32_t d_tmem = tmem_base + (uint32_t)(buf * NT);
           // position of this example's stages in the producer's sequence
-          const int pair = e >> 1;
-          const bool paired = ((e | 1) < nb);              // the pair has two examples
-          const long long n0 = (long long)pair * 2 * nk;
+          const long long n0 = (long long)(e >> 1) * 2 * nk;
           for (int kc = 0; kc < nk; ++kc) {
-            const long long n = n0 + (paired ? 2 * kc + x : kc);
+            const long long n = n0 + 2 * kc + x;
             const int s = (int)(n % STAGES);
             const uint32_t ph = (uint32_t)(n / STAGES) & 1u;
-            // A parity wait is only meaningful when the waiter is at most one phase away from the
-            // barrier.  Slots of this issuer's own parity are waited on phase after phase, so that
-            // holds.  In an unpaired last example the issuer also consumes the other issuer's slots;
-            // there it first makes sure the slot's previous phase (the other issuer's data) has
-            // landed, otherwise a slot still in that phase would satisfy the wait for the next one.
-            if (!paired && ((s & 1) != x) && n >= STAGES) {
-              if (!mbar_wait_bounded(full_bar(s), ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_FULL)) { ok = false; break; }
-            }
+            // A parity wait is only meaningful while the waiter is at most one phase away from the
+            // barrier.  Every slot this issuer waits on has its own parity (x), so it sees each of
+            // the slot's phases in turn and that always holds.
             if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, p.dev_status, TC_WAIT_FULL)) { ok = false; break; }
             tc_fence_after();
             const uint32_t a_src = smem_base + s * STAGE_BYTES;
