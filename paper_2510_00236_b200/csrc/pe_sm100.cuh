@@ -254,6 +254,11 @@ __device__ __forceinline__ void tmem_ld_32x32b_x64_wait(uint32_t taddr, uint32_t
       : "memory");
 }
 
+// One 16-byte reduction: adds four consecutive floats to global memory (p 16-byte aligned).
+__device__ __forceinline__ void red_add_f32x4(float* p, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N>

@@ -305,8 +305,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
               if (mrow) *reinterpret_cast<float4*>(mrow + i) = vm;
               if (srow) *reinterpret_cast<float4*>(srow + i) = vs;
             } else {
-              if (mrow) { atomicAdd(mrow + i, vm.x); atomicAdd(mrow + i + 1, vm.y); atomicAdd(mrow + i + 2, vm.z); atomicAdd(mrow + i + 3, vm.w); }
-              if (srow) { atomicAdd(srow + i, vs.x); atomicAdd(srow + i + 1, vs.y); atomicAdd(srow + i + 2, vs.z); atomicAdd(srow + i + 3, vs.w); }
+              if (mrow) red_add_f32x4(mrow + i, vm.x, vm.y, vm.z, vm.w);
+              if (srow) red_add_f32x4(srow + i, vs.x, vs.y, vs.z, vs.w);
             }
           }
         }
