@@ -12,7 +12,7 @@ import os
 import torch
 
 __all__ = [
-    "PestatsError", "PHI_IDENTITY", "PHI_SQUARE", "PHI_SIGN", "PATH_AUTO", "PATH_SIMT", "PATH_TENSOR",
+    "PestatsError", "PHI_IDENTITY", "PHI_SQUARE", "PHI_SIGN", "PATH_AUTO", "PATH_SIMT", "PATH_TENSOR", "PATH_TENSOR_NARROW",
     "EXPORTED_SYMBOLS", "library_path", "load_library", "pe_linear_stats", "pe_linear_stats_f32",
     "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_workspace_bytes", "microadam_step",
     "microsignsgd_step", "pe_status_string", "pe_get_async_status", "pe_set_path", "pe_last_path",
@@ -20,7 +20,7 @@ __all__ = [
 ]
 
 PHI_IDENTITY, PHI_SQUARE, PHI_SIGN = 0, 1, 2
-PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_NARROW = 0, 1, 2, 3
 _PHI_NAMES = {"identity": PHI_IDENTITY, "square": PHI_SQUARE, "sign": PHI_SIGN}
 
 # every symbol include/pestats.h declares

@@ -22,13 +22,14 @@ __device__ unsigned int g_dev_status = 0;   // first device-side wait that gave 
 static std::atomic<int> g_path{PE_PATH_AUTO};
 static std::atomic<int> g_last_path{PE_PATH_AUTO};
 static std::atomic<long long> g_launches{0};
+constexpr int TC_MEAN_TMEM_MIN_T = 96;
 
 constexpr int MAX_DEVICES = 64;
 struct DeviceInfo {
   std::atomic<int> state{0};     // 0 unknown, 1 ready, -1 failed
   int cc_major = 0, sm_count = 0;
   unsigned int* status_ptr = nullptr;
-  bool tc_attr_set[6] = {false, false, false, false, false, false};
+  bool tc_attr_set[8] = {false, false, false, false, false, false, false, false};
 };
 static DeviceInfo g_dev[MAX_DEVICES];
 
@@ -140,18 +141,18 @@ static pe_status_t zero_outputs(float* a, float* b, size_t bytes, cudaStream_t s
   return PE_OK;
 }
 
-template <int PHI, bool TF32, int NT, bool WITH_MEAN>
+template <int PHI, bool TF32, int NT, int MEAN>
 static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& mx, const CUtensorMap& my, const TcParams& p,
                                   dim3 grid, cudaStream_t st) {
   constexpr int smem = TcOperand<TF32, NT>::SMEM_BYTES;
   if (!di->tc_attr_set[slot]) {
-    if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, WITH_MEAN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+    if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
       cudaGetLastError();
       return PE_ERR_CUDA;
     }
     di->tc_attr_set[slot] = true;
   }
-  tc_stats_kernel<PHI, TF32, NT, WITH_MEAN><<<grid, TC_THREADS, smem, st>>>(mx, my, p);
+  tc_stats_kernel<PHI, TF32, NT, MEAN><<<grid, TC_THREADS, smem, st>>>(mx, my, p);
   return check_launch();
 }
 
@@ -161,9 +162,12 @@ static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& m
 static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int B, int T, int d_in, int d_out, int phi,
                              int per_example, float* out_mean, float* out_stat, cudaStream_t st, bool tf32 = false) {
   const bool both = per_example && out_mean && out_stat;
-  const int nt = both ? 128 : 256;
+  // Both outputs: sum_b G_b in tensor memory beside a 256-wide accumulator, unless the sequences are
+  // so short that the per-example drain of that single accumulator would dominate.
+  const bool mean_regs = both && (T < TC_MEAN_TMEM_MIN_T || g_path.load() == PE_PATH_TENSOR_NARROW);
+  const int nt = mean_regs ? 128 : 256;
   const int box_feats = tf32 ? TcOperand<true, 256>::BOX_FEATS : TcOperand<false, 256>::BOX_FEATS;
-  const int box_tokens = tf32 ? TcOperand<true, 256>::BK : (both ? TcOperand<false, 128>::BK : TcOperand<false, 256>::BK);
+  const int box_tokens = tf32 ? TcOperand<true, 256>::BK : (mean_regs ? TcOperand<false, 128>::BK : TcOperand<false, 256>::BK);
   CUtensorMap mx, my;
   pe_status_t rc = make_operand_map(&mx, X, B, T, d_in, tf32, box_feats, box_tokens);
   if (rc != PE_OK) return rc;
@@ -180,14 +184,18 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = per_example;
   p.out_mean = out_mean; p.out_stat = out_stat; p.dev_status = di->status_ptr;
   dim3 grid(2 * pairs_m, tiles_n, ns);
-  if (tf32) return launch_tc_inst<0, true, 256, false>(di, 5, mx, my, p, grid, st);
-  if (!per_example) return launch_tc_inst<0, false, 256, false>(di, 4, mx, my, p, grid, st);
-  if (both) {
-    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, true>(di, 0, mx, my, p, grid, st);
-    return launch_tc_inst<2, false, 128, true>(di, 1, mx, my, p, grid, st);
+  if (tf32) return launch_tc_inst<0, true, 256, MEAN_NONE>(di, 5, mx, my, p, grid, st);
+  if (!per_example) return launch_tc_inst<0, false, 256, MEAN_NONE>(di, 4, mx, my, p, grid, st);
+  if (mean_regs) {
+    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, MEAN_REGS>(di, 0, mx, my, p, grid, st);
+    return launch_tc_inst<2, false, 128, MEAN_REGS>(di, 1, mx, my, p, grid, st);
   }
-  if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, false>(di, 2, mx, my, p, grid, st);
-  return launch_tc_inst<2, false, 256, false>(di, 3, mx, my, p, grid, st);
+  if (both) {
+    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, MEAN_TMEM>(di, 6, mx, my, p, grid, st);
+    return launch_tc_inst<2, false, 256, MEAN_TMEM>(di, 7, mx, my, p, grid, st);
+  }
+  if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, MEAN_NONE>(di, 2, mx, my, p, grid, st);
+  return launch_tc_inst<2, false, 256, MEAN_NONE>(di, 3, mx, my, p, grid, st);
 }
 
 template <typename TIn, int MODE>
@@ -228,7 +236,7 @@ static pe_status_t linear_stats_impl(const TIn* X, const TIn* dY, int B, int T, 
   if (B == 0 || T == 0) return zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
   const int forced = g_path.load();
   const bool tc_ok = allow_tc && tc_shape_ok(B, T, d_in, d_out);
-  if (forced == PE_PATH_TENSOR && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
+  if ((forced == PE_PATH_TENSOR || forced == PE_PATH_TENSOR_NARROW) && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
   if (tc_ok && forced != PE_PATH_SIMT) {
     if constexpr (sizeof(TIn) == 2) {
       g_last_path.store(PE_PATH_TENSOR);
@@ -297,7 +305,7 @@ pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_
   if (B == 0 || T == 0) return zero_outputs(out_stat, nullptr, (size_t)d_in * d_out * sizeof(float), st);
   const int forced = g_path.load();
   const bool tc_ok = token_tc_ok(B, T, d_in, d_out);
-  if (forced == PE_PATH_TENSOR && !tc_shape_ok(B, T, d_in, d_out)) return PE_ERR_UNSUPPORTED_SHAPE;
+  if ((forced == PE_PATH_TENSOR || forced == PE_PATH_TENSOR_NARROW) && !tc_shape_ok(B, T, d_in, d_out)) return PE_ERR_UNSUPPORTED_SHAPE;
   if (tc_ok && forced != PE_PATH_SIMT) {
     const size_t rows = (size_t)B * (size_t)T;
     const size_t x_bytes = align_up(rows * d_in * 4, 256), y_bytes = align_up(rows * d_out * 4, 256);
@@ -454,7 +462,7 @@ pe_status_t pe_get_async_status(pe_stream_t stream, int* detail) {
 }
 
 int pe_set_path(int path) {
-  if (path < PE_PATH_AUTO || path > PE_PATH_TENSOR) return -1;
+  if (path < PE_PATH_AUTO || path > PE_PATH_TENSOR_NARROW) return -1;
   return g_path.exchange(path);
 }
 int pe_last_path(void) { return g_last_path.load(); }

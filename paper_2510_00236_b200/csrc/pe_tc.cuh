@@ -10,16 +10,21 @@
 // operand bytes each SM pulls from L2 per flop; an SM sustains about 70 B/clk from L2, a lone
 // 128 x 128 tile would need 128 B/clk at full tensor rate, a 256 x 128 pair 96, a 256 x 256 pair 64.
 //
-//   NT = 128, two running sums per thread (64 + 64 registers)      -- both outputs wanted
-//   NT = 256, one running sum per thread (128 registers)           -- only sum_b phi(G_b) wanted
-//   NT = 256, no running sum (accumulate in tensor memory)         -- plain contraction over all rows
+//   MEAN_REGS, NT = 128: two running sums per thread (64 + 64 registers)         -- both outputs, short sequences
+//   MEAN_TMEM, NT = 256: sum_b phi(G_b) in 128 registers per thread, sum_b G_b in
+//                        tensor memory beside ONE per-example accumulator, one issuer -- both outputs
+//   MEAN_NONE, NT = 256: one running sum per thread (128 registers)               -- only sum_b phi(G_b) wanted
+//   PHI = 0,   NT = 256: no per-example reset (accumulate in tensor memory)        -- plain contraction over all rows
 //
 // Warp roles per block (12 warps): 0 = TMA producer of the dY boxes, 2 = TMEM allocator, then TMA
 // producer of the X boxes, 1 and 3 = MMA issuers (leader block only), 4..11 = epilogue (warp w reads
 // TMEM lanes 32*(w%4)..+31, column half (w-4)/4).  One thread needs on the order of a hundred cycles
 // per TMA instruction, so the boxes are tall (BK tokens, 16 KiB for bf16) and split over two warps.
 // Two examples are in flight at once, one per issuer; the 512 TMEM columns hold 512/NT accumulators,
-// so the MMAs of later examples overlap the epilogue of earlier ones.
+// so the MMAs of later examples overlap the epilogue of earlier ones.  (MEAN_TMEM has one issuer and
+// one accumulator: while the epilogue drains it the producers keep filling the ring, and the issuer
+// then works the backlog off at full tensor rate, which absorbs the pause as long as the operand
+// supply, not the tensor pipe, is what bounds the example.)
 //
 // Barriers.  full[s] lives in the leader block: its producer posts the byte count of BOTH blocks'
 // loads, and the follower's TMA loads credit their bytes to it through the cluster window.
@@ -100,17 +105,22 @@ __device__ __forceinline__ float phi_apply(float g) {
   return g;
 }
 
+enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2 };   // where sum_b G_b is kept in per-example mode
+
 // gridDim = (2 * ceil(d_out / 256), ceil(d_in / NT), nsplit); blockIdx.x = 2 * pair row + rank in pair.
-// WITH_MEAN: keep the running sum of G_b as well (requires NT = 128).
-template <int PHI, bool TF32, int NT, bool WITH_MEAN>
+template <int PHI, bool TF32, int NT, int MEAN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy, TcParams p) {
   using namespace sm100;
   using Op = TcOperand<TF32, NT>;
-  static_assert(!WITH_MEAN || NT == 128, "two running sums only fit the registers at NT = 128");
-  constexpr int STAGES = Op::STAGES, ACC_BUFS = Op::ACC_BUFS, BK = Op::BK;
+  static_assert(MEAN != MEAN_REGS || NT == 128, "two running sums only fit the registers at NT = 128");
+  static_assert(MEAN != MEAN_TMEM || (NT == 256 && PHI != 0), "the tensor-memory mean sits beside one 256-column accumulator");
+  constexpr int STAGES = Op::STAGES, BK = Op::BK;
   constexpr int BOX_BYTES = Op::BOX_BYTES, A_BYTES = Op::A_BYTES, STAGE_BYTES = Op::STAGE_BYTES;
-  constexpr int BUFS_PER_ISSUER = ACC_BUFS / 2;     // 2 | 1
+  constexpr int ISSUERS = (MEAN == MEAN_TMEM) ? 1 : 2;
+  constexpr int ACC_BUFS = (MEAN == MEAN_TMEM) ? 1 : Op::ACC_BUFS;
+  constexpr int BUFS_PER_ISSUER = ACC_BUFS / ISSUERS;     // 2 | 1
+  constexpr int MEAN_COL0 = 256;                    // first tensor-memory column of the MEAN_TMEM running sum
   constexpr int COLS = NT / 2;                      // accumulator columns per epilogue thread
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -155,16 +165,16 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       // ---------------------------------------------------------- TMA producers (both blocks)
       // Warp 0 loads this block's rows of dY^T (and, in the leader, posts the stage's byte count);
       // warp 2 loads this block's half of the X^T rows.  Both wait for the same "stage empty" phase.
-      // Stages are filled for two examples at a time, alternating between them: stage 2*kc of a pair
-      // of examples belongs to its first example (issuer 0, even slots), stage 2*kc+1 to its second
-      // (issuer 1, odd slots); the ring has an even number of slots.
+      // With two issuers, stages are filled for two examples at a time, alternating between them:
+      // stage 2*kc of a pair of examples belongs to its first example (issuer 0, even slots), stage
+      // 2*kc+1 to its second (issuer 1, odd slots); the ring has an even number of slots.
       if (lane == 0) {
         const bool is_a = (warp == 0);
         prefetch_tensormap(is_a ? &tmap_dy : &tmap_x);
         int s = 0; uint32_t ph = 0;
         bool ok = true;
-        for (int e0 = 0; e0 < nb && ok; e0 += 2) {
-          const int n_in_pair = (e0 + 1 < nb) ? 2 : 1;
+        for (int e0 = 0; e0 < nb && ok; e0 += ISSUERS) {
+          const int n_in_pair = (e0 + ISSUERS <= nb) ? ISSUERS : 1;
           for (int kc = 0; kc < nk && ok; ++kc) {
             for (int x = 0; x < n_in_pair; ++x) {
               if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_EMPTY)) { ok = false; break; }
@@ -187,12 +197,12 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             }
             // An unpaired last example leaves the second issuer's slot of every step unused, so
             // that each slot is only ever consumed by the issuer of its own parity.
-            if (n_in_pair == 1) { if (++s == STAGES) { s = 0; ph ^= 1u; } }
+            if (n_in_pair < ISSUERS) { if (++s == STAGES) { s = 0; ph ^= 1u; } }
           }
         }
       }
       __syncwarp();
-    } else if (rank == 0) {
+    } else if (rank == 0 && (warp == 1 || ISSUERS == 2)) {
       // ---------------------------------------------------------- MMA issuers (leader block, warps 1 and 3)
       // Two issuing threads (one per warp).  A barrier probe right after queuing MMAs costs the
       // issuing thread a couple of hundred cycles; with two threads working on two different examples
@@ -204,7 +214,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         bool ok = true;
         uint32_t accumulate = 0;
         int i_local = 0;                                   // examples this issuer has started
-        for (int e = x; e < nb && ok; e += 2, ++i_local) {
+        for (int e = x; e < nb && ok; e += ISSUERS, ++i_local) {
           const int grp = p.per_example ? i_local : 0;
           const int buf = BUFS_PER_ISSUER * x + (grp % BUFS_PER_ISSUER);
           if (p.per_example || i_local == 0) {
@@ -215,9 +225,9 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
           }
           const uint32_t d_tmem = tmem_base + (uint32_t)(buf * NT);
           // position of this example's stages in the producer's sequence
-          const long long n0 = (long long)(e >> 1) * 2 * nk;
+          const long long n0 = (long long)(e / ISSUERS) * ISSUERS * nk;
           for (int kc = 0; kc < nk; ++kc) {
-            const long long n = n0 + 2 * kc + x;
+            const long long n = n0 + ISSUERS * kc + x;
             const int s = (int)(n % STAGES);
             const uint32_t ph = (uint32_t)(n / STAGES) & 1u;
             // A parity wait is only meaningful while the waiter is at most one phase away from the
@@ -240,7 +250,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             }
             umma_commit_pair(empty_bar(s));                // stage reusable in both blocks once these MMAs retire
           }
-          const bool last_of_group = p.per_example || (e + 2 >= nb);
+          const bool last_of_group = p.per_example || (e + ISSUERS >= nb);
           if (ok && last_of_group) umma_commit_pair(acc_full_bar(buf));   // accumulator complete, both blocks
         }
       }
@@ -251,7 +261,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     setmaxnreg_inc<TC_REGS_EPILOGUE>();
     const int q = warp & 3;                 // TMEM lane quadrant this warp may access
     const int h = (warp - 4) >> 2;          // column half of the tile
-    constexpr bool KEEP_MEAN = WITH_MEAN || PHI == 0;
+    constexpr bool KEEP_MEAN = MEAN == MEAN_REGS || PHI == 0;     // running sum of G_b in registers
     constexpr int N_STAT = (PHI != 0) ? COLS : 1;
     constexpr int N_MEAN = KEEP_MEAN ? COLS : 1;
     float acc_stat[N_STAT], acc_mean[N_MEAN];
@@ -262,14 +272,40 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     bool ok = true;
     // per-example mode: one accumulator per example, in example order (example e -> issuer e&1).
     // plain mode: one accumulator per issuer that had work.
-    const int n_acc = p.per_example ? nb : (nb >= 2 ? 2 : nb);
+    const int n_acc = p.per_example ? nb : (nb >= ISSUERS ? ISSUERS : nb);
+    const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
     for (int a = 0; a < n_acc; ++a) {
-      const int x = a & 1, grp = p.per_example ? (a >> 1) : 0;
+      const int x = a % ISSUERS, grp = p.per_example ? (a / ISSUERS) : 0;
       const int buf = BUFS_PER_ISSUER * x + (grp % BUFS_PER_ISSUER);
       const uint32_t acc_ph = (uint32_t)(grp / BUFS_PER_ISSUER) & 1u;
       if (!mbar_wait_bounded(acc_full_bar(buf), acc_ph, abort_flag, p.dev_status, TC_WAIT_ACC_FULL)) { ok = false; break; }
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * NT + h * COLS);
+      const uint32_t taddr = lane_base + (uint32_t)(buf * NT + h * COLS);
+      if constexpr (MEAN == MEAN_TMEM) {
+        // sum_b G_b lives in tensor-memory columns MEAN_COL0.. of the same lanes: read it with G_b,
+        // add, write it back (the first example just writes G_b).
+        const uint32_t maddr = lane_base + (uint32_t)(MEAN_COL0 + h * COLS);
+#pragma unroll
+        for (int c = 0; c < COLS / 16; ++c) {
+          uint32_t r[16], m[16];
+          if (a == 0) tmem_ld_32x32b_x16_wait(taddr + c * 16, r);
+          else tmem_ld_32x32b_x16_pair_wait(taddr + c * 16, r, maddr + c * 16, m);
+          if (c == COLS / 16 - 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));   // G_b read: the issuer may start the next example
+          }
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float g = __uint_as_float(r[j]);
+            acc_stat[c * 16 + j] += phi_apply<PHI>(g);
+            if (a != 0) r[j] = __float_as_uint(g + __uint_as_float(m[j]));
+          }
+          tmem_st_32x32b_x16(maddr + c * 16, r);
+        }
+        tmem_st_wait();
+        continue;
+      }
 #pragma unroll
       for (int c = 0; c < COLS / 32; ++c) {
         uint32_t r[32];
@@ -291,8 +327,26 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       const int o = tile_m * TC_TILE_M + q * 32 + lane;
       const int i_base = tile_n * NT + h * COLS;
       if (o < p.d_out) {
-        float* mrow = (KEEP_MEAN && p.out_mean) ? p.out_mean + (size_t)o * p.d_in : nullptr;
+        float* mrow = ((KEEP_MEAN || MEAN == MEAN_TMEM) && p.out_mean) ? p.out_mean + (size_t)o * p.d_in : nullptr;
         float* srow = p.out_stat ? p.out_stat + (size_t)o * p.d_in : nullptr;
+        if constexpr (MEAN == MEAN_TMEM) {
+          // the running sum of G_b comes out of tensor memory, 32 columns at a time
+          const uint32_t maddr = lane_base + (uint32_t)(MEAN_COL0 + h * COLS);
+#pragma unroll
+          for (int c = 0; c < COLS / 32; ++c) {
+            uint32_t m[32];
+            tmem_ld_32x32b_x32_wait(maddr + c * 32, m);
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              const int i = i_base + c * 32 + j;
+              if (mrow && i < p.d_in) {
+                if (p.nsplit == 1) *reinterpret_cast<float4*>(mrow + i) = make_float4(__uint_as_float(m[j]), __uint_as_float(m[j + 1]), __uint_as_float(m[j + 2]), __uint_as_float(m[j + 3]));
+                else red_add_f32x4(mrow + i, __uint_as_float(m[j]), __uint_as_float(m[j + 1]), __uint_as_float(m[j + 2]), __uint_as_float(m[j + 3]));
+              }
+            }
+          }
+          mrow = nullptr;
+        }
 #pragma unroll
         for (int j = 0; j < COLS; j += 4) {
           const int i = i_base + j;

@@ -87,6 +87,16 @@ def test_odd_batch_slices_and_long_sequences_single_output():
     assert pe.pe_get_async_status(DEV) == (0, 0)
 
 
+@pytest.mark.parametrize("B,T,d_in,d_out", [(5, 200, 136, 264), (40, 96, 384, 256), (3, 2000, 264, 520), (7, 128, 256, 512)])
+def test_register_mean_kernel_at_any_sequence_length(B, T, d_in, d_out):
+    """Long sequences normally keep sum_b G_b in tensor memory; the 256 x 128 kernel with both running
+    sums in registers must give the same statistics when forced."""
+    pe.pe_set_path(pe.PATH_TENSOR_NARROW)
+    li = inputs.gaussian_layer(B, T, d_in, d_out, seed=500 + T, device=DEV)
+    check_all(li, phis=("square", "sign"), token=False)
+    assert pe.pe_last_path() == pe.PATH_TENSOR
+
+
 def test_heavy_tailed_and_heterogeneous_small():
     check_all(inputs.heavy_tailed_layer(12, 128, 256, 384, seed=41, device=DEV))
     check_all(inputs.heterogeneous_layer(20, 64, 128, 256, seed=42, device=DEV))
