@@ -323,49 +323,52 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         }
       }
     }
+    // The tensor-memory loads below are warp-wide instructions: the condition around them is made
+    // uniform over the warp and they stay outside every per-lane condition.
+    ok = __all_sync(0xffffffffu, ok);
     if (ok && n_acc > 0) {
       const int o = tile_m * TC_TILE_M + q * 32 + lane;
       const int i_base = tile_n * NT + h * COLS;
-      if (o < p.d_out) {
-        float* mrow = ((KEEP_MEAN || MEAN == MEAN_TMEM) && p.out_mean) ? p.out_mean + (size_t)o * p.d_in : nullptr;
-        float* srow = p.out_stat ? p.out_stat + (size_t)o * p.d_in : nullptr;
-        if constexpr (MEAN == MEAN_TMEM) {
-          // the running sum of G_b comes out of tensor memory, 32 columns at a time
-          const uint32_t maddr = lane_base + (uint32_t)(MEAN_COL0 + h * COLS);
+      const bool row_ok = o < p.d_out;
+      float* mrow = ((KEEP_MEAN || MEAN == MEAN_TMEM) && p.out_mean && row_ok) ? p.out_mean + (size_t)o * p.d_in : nullptr;
+      float* srow = (p.out_stat && row_ok) ? p.out_stat + (size_t)o * p.d_in : nullptr;
+      if constexpr (MEAN == MEAN_TMEM) {
+        // the running sum of G_b comes out of tensor memory, 32 columns at a time
+        const uint32_t maddr = lane_base + (uint32_t)(MEAN_COL0 + h * COLS);
 #pragma unroll
-          for (int c = 0; c < COLS / 32; ++c) {
-            uint32_t m[32];
-            tmem_ld_32x32b_x32_wait(maddr + c * 32, m);
+        for (int c = 0; c < COLS / 32; ++c) {
+          uint32_t m[32];
+          tmem_ld_32x32b_x32_wait(maddr + c * 32, m);
 #pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-              const int i = i_base + c * 32 + j;
-              if (mrow && i < p.d_in) {
-                if (p.nsplit == 1) *reinterpret_cast<float4*>(mrow + i) = make_float4(__uint_as_float(m[j]), __uint_as_float(m[j + 1]), __uint_as_float(m[j + 2]), __uint_as_float(m[j + 3]));
-                else red_add_f32x4(mrow + i, __uint_as_float(m[j]), __uint_as_float(m[j + 1]), __uint_as_float(m[j + 2]), __uint_as_float(m[j + 3]));
-              }
+          for (int j = 0; j < 32; j += 4) {
+            const int i = i_base + c * 32 + j;
+            if (mrow && i < p.d_in) {
+              if (p.nsplit == 1) *reinterpret_cast<float4*>(mrow + i) = make_float4(__uint_as_float(m[j]), __uint_as_float(m[j + 1]), __uint_as_float(m[j + 2]), __uint_as_float(m[j + 3]));
+              else red_add_f32x4(mrow + i, __uint_as_float(m[j]), __uint_as_float(m[j + 1]), __uint_as_float(m[j + 2]), __uint_as_float(m[j + 3]));
             }
           }
-          mrow = nullptr;
         }
+        mrow = nullptr;
+      }
 #pragma unroll
-        for (int j = 0; j < COLS; j += 4) {
-          const int i = i_base + j;
-          if (i < p.d_in) {                                      // d_in % 8 == 0: a group of 4 is all in or all out
-            float4 vm = make_float4(0.f, 0.f, 0.f, 0.f), vs;
-            if (KEEP_MEAN) vm = make_float4(acc_mean[j], acc_mean[j + 1], acc_mean[j + 2], acc_mean[j + 3]);
-            if (PHI != 0) vs = make_float4(acc_stat[j], acc_stat[j + 1], acc_stat[j + 2], acc_stat[j + 3]);
-            else vs = vm;
-            if (p.nsplit == 1) {
-              if (mrow) *reinterpret_cast<float4*>(mrow + i) = vm;
-              if (srow) *reinterpret_cast<float4*>(srow + i) = vs;
-            } else {
-              if (mrow) red_add_f32x4(mrow + i, vm.x, vm.y, vm.z, vm.w);
-              if (srow) red_add_f32x4(srow + i, vs.x, vs.y, vs.z, vs.w);
-            }
+      for (int j = 0; j < COLS; j += 4) {
+        const int i = i_base + j;
+        if (i < p.d_in) {                                      // d_in % 8 == 0: a group of 4 is all in or all out
+          float4 vm = make_float4(0.f, 0.f, 0.f, 0.f), vs;
+          if (KEEP_MEAN) vm = make_float4(acc_mean[j], acc_mean[j + 1], acc_mean[j + 2], acc_mean[j + 3]);
+          if (PHI != 0) vs = make_float4(acc_stat[j], acc_stat[j + 1], acc_stat[j + 2], acc_stat[j + 3]);
+          else vs = vm;
+          if (p.nsplit == 1) {
+            if (mrow) *reinterpret_cast<float4*>(mrow + i) = vm;
+            if (srow) *reinterpret_cast<float4*>(srow + i) = vs;
+          } else {
+            if (mrow) red_add_f32x4(mrow + i, vm.x, vm.y, vm.z, vm.w);
+            if (srow) red_add_f32x4(srow + i, vs.x, vs.y, vs.z, vs.w);
           }
         }
       }
     }
+    __syncwarp();
   }
 
   // ---------------------------------------------------------------- teardown
