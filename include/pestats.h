@@ -48,7 +48,7 @@ typedef enum { PE_PHI_IDENTITY = 0, PE_PHI_SQUARE = 1, PE_PHI_SIGN = 2 } pe_phi_
 /* Which kernel family a call may use.  AUTO picks the tensor-core kernel whenever the shape allows
  * it (bf16 inputs, d_in % 8 == 0, d_out % 8 == 0) and the SIMT kernel otherwise.  TENSOR_NARROW is
  * TENSOR with the 256 x 128 tile that keeps both running sums in registers even for long sequences
- * (AUTO and TENSOR use it for T < 96 only and otherwise keep sum_b G_b in tensor memory beside a
+ * (AUTO and TENSOR use it for T < 2048 only and otherwise keep sum_b G_b in tensor memory beside a
  * 256 x 256 tile); it exists so that tests can reach that kernel at any T. */
 typedef enum { PE_PATH_AUTO = 0, PE_PATH_SIMT = 1, PE_PATH_TENSOR = 2, PE_PATH_TENSOR_NARROW = 3 } pe_path_t;
 

@@ -22,7 +22,7 @@ __device__ unsigned int g_dev_status = 0;   // first device-side wait that gave 
 static std::atomic<int> g_path{PE_PATH_AUTO};
 static std::atomic<int> g_last_path{PE_PATH_AUTO};
 static std::atomic<long long> g_launches{0};
-constexpr int TC_MEAN_TMEM_MIN_T = 96;
+constexpr int TC_MEAN_TMEM_MIN_T = 2048;
 
 constexpr int MAX_DEVICES = 64;
 struct DeviceInfo {

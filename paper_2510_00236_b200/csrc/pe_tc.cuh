@@ -105,6 +105,23 @@ __device__ __forceinline__ float phi_apply(float g) {
   return g;
 }
 
+// Walks the slots of the operand ring in the order the producers fill them.  With two issuers the
+// examples are taken two at a time and their stages interleaved: slot 2*kc of a pair of examples
+// belongs to its first example (issuer 0, even slots), slot 2*kc+1 to its second (issuer 1, odd
+// slots).  An unpaired last example leaves its partner's slots unused (used() is false there), so
+// that each slot is only ever consumed by the issuer of its own parity.
+template <int ISSUERS>
+struct StageWalk {
+  int nb, nk, e0, kc, x;
+  __device__ StageWalk(int nb_, int nk_) : nb(nb_), nk(nk_), e0(0), kc(0), x(0) {}
+  __device__ bool valid() const { return e0 < nb; }
+  __device__ bool used() const { return e0 + x < nb; }
+  __device__ int e() const { return e0 + x; }
+  __device__ void next() {
+    if (++x == ISSUERS) { x = 0; if (++kc == nk) { kc = 0; e0 += ISSUERS; } }
+  }
+};
+
 enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2 };   // where sum_b G_b is kept in per-example mode
 
 // gridDim = (2 * ceil(d_out / 256), ceil(d_in / NT), nsplit); blockIdx.x = 2 * pair row + rank in pair.
@@ -120,6 +137,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   constexpr int ISSUERS = (MEAN == MEAN_TMEM) ? 1 : 2;
   constexpr int ACC_BUFS = (MEAN == MEAN_TMEM) ? 1 : Op::ACC_BUFS;
   constexpr int BUFS_PER_ISSUER = ACC_BUFS / ISSUERS;     // 2 | 1
+  constexpr int PF_AHEAD = STAGES + 4;              // slots between an L2 prefetch and the load of the same boxes
   constexpr int MEAN_COL0 = 256;                    // first tensor-memory column of the MEAN_TMEM running sum
   constexpr int COLS = NT / 2;                      // accumulator columns per epilogue thread
   extern __shared__ uint8_t smem_raw[];
@@ -170,35 +188,34 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       // 2*kc+1 to its second (issuer 1, odd slots); the ring has an even number of slots.
       if (lane == 0) {
         const bool is_a = (warp == 0);
-        prefetch_tensormap(is_a ? &tmap_dy : &tmap_x);
+        const CUtensorMap* tmap = is_a ? &tmap_dy : &tmap_x;
+        const int c0 = is_a ? tile_m * TC_TILE_M : tile_n * NT + (int)rank * Op::B_FEATS;   // first feature of this warp's boxes
+        const int n_boxes = is_a ? Op::A_BOXES : Op::B_BOXES;
+        prefetch_tensormap(tmap);
+        // The ring holds what shared memory allows; the boxes of stages further ahead are requested
+        // into L2 so that the real load, when its slot frees up, does not wait on DRAM.
+        StageWalk<ISSUERS> pf(nb, nk);
+        for (int i = 0; i < PF_AHEAD && pf.valid(); ++i) {
+          if (i >= STAGES && pf.used())
+            for (int g = 0; g < n_boxes; ++g) tma_prefetch_3d(tmap, c0 + g * Op::BOX_FEATS, pf.kc * BK, b_begin + pf.e());
+          pf.next();
+        }
         int s = 0; uint32_t ph = 0;
-        bool ok = true;
-        for (int e0 = 0; e0 < nb && ok; e0 += ISSUERS) {
-          const int n_in_pair = (e0 + ISSUERS <= nb) ? ISSUERS : 1;
-          for (int kc = 0; kc < nk && ok; ++kc) {
-            for (int x = 0; x < n_in_pair; ++x) {
-              if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_EMPTY)) { ok = false; break; }
-              const int b = b_begin + e0 + x;
-              if (is_a && rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);     // both blocks' bytes
-              const uint32_t leader_full = map_to_cta(full_bar(s), 0);
-              const uint32_t a_dst = smem_base + s * STAGE_BYTES;
-              const uint32_t b_dst = a_dst + A_BYTES;
-              if (is_a) {
-#pragma unroll
-                for (int g = 0; g < Op::A_BOXES; ++g)
-                  tma_load_3d_pair(a_dst + g * BOX_BYTES, &tmap_dy, leader_full, tile_m * TC_TILE_M + g * Op::BOX_FEATS, kc * BK, b);
-              } else {
-#pragma unroll
-                for (int g = 0; g < Op::B_BOXES; ++g)
-                  tma_load_3d_pair(b_dst + g * BOX_BYTES, &tmap_x, leader_full,
-                                   tile_n * NT + (int)rank * Op::B_FEATS + g * Op::BOX_FEATS, kc * BK, b);
-              }
-              if (++s == STAGES) { s = 0; ph ^= 1u; }
-            }
-            // An unpaired last example leaves the second issuer's slot of every step unused, so
-            // that each slot is only ever consumed by the issuer of its own parity.
-            if (n_in_pair < ISSUERS) { if (++s == STAGES) { s = 0; ph ^= 1u; } }
+        for (StageWalk<ISSUERS> cur(nb, nk); cur.valid(); cur.next()) {
+          if (pf.valid()) {
+            if (pf.used())
+              for (int g = 0; g < n_boxes; ++g) tma_prefetch_3d(tmap, c0 + g * Op::BOX_FEATS, pf.kc * BK, b_begin + pf.e());
+            pf.next();
           }
+          if (cur.used()) {
+            if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_EMPTY)) break;
+            if (is_a && rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);     // both blocks' bytes
+            const uint32_t leader_full = map_to_cta(full_bar(s), 0);
+            const uint32_t dst = smem_base + s * STAGE_BYTES + (is_a ? 0 : A_BYTES);
+            for (int g = 0; g < n_boxes; ++g)
+              tma_load_3d_pair(dst + g * BOX_BYTES, tmap, leader_full, c0 + g * Op::BOX_FEATS, cur.kc * BK, b_begin + cur.e());
+          }
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
       }
       __syncwarp();
