@@ -137,7 +137,6 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   constexpr int ISSUERS = (MEAN == MEAN_TMEM) ? 1 : 2;
   constexpr int ACC_BUFS = (MEAN == MEAN_TMEM) ? 1 : Op::ACC_BUFS;
   constexpr int BUFS_PER_ISSUER = ACC_BUFS / ISSUERS;     // 2 | 1
-  constexpr int PF_AHEAD = STAGES + 4;              // slots between an L2 prefetch and the load of the same boxes
   constexpr int MEAN_COL0 = 256;                    // first tensor-memory column of the MEAN_TMEM running sum
   constexpr int COLS = NT / 2;                      // accumulator columns per epilogue thread
   extern __shared__ uint8_t smem_raw[];
@@ -192,21 +191,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         const int c0 = is_a ? tile_m * TC_TILE_M : tile_n * NT + (int)rank * Op::B_FEATS;   // first feature of this warp's boxes
         const int n_boxes = is_a ? Op::A_BOXES : Op::B_BOXES;
         prefetch_tensormap(tmap);
-        // The ring holds what shared memory allows; the boxes of stages further ahead are requested
-        // into L2 so that the real load, when its slot frees up, does not wait on DRAM.
-        StageWalk<ISSUERS> pf(nb, nk);
-        for (int i = 0; i < PF_AHEAD && pf.valid(); ++i) {
-          if (i >= STAGES && pf.used())
-            for (int g = 0; g < n_boxes; ++g) tma_prefetch_3d(tmap, c0 + g * Op::BOX_FEATS, pf.kc * BK, b_begin + pf.e());
-          pf.next();
-        }
         int s = 0; uint32_t ph = 0;
         for (StageWalk<ISSUERS> cur(nb, nk); cur.valid(); cur.next()) {
-          if (pf.valid()) {
-            if (pf.used())
-              for (int g = 0; g < n_boxes; ++g) tma_prefetch_3d(tmap, c0 + g * Op::BOX_FEATS, pf.kc * BK, b_begin + pf.e());
-            pf.next();
-          }
           if (cur.used()) {
             if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_EMPTY)) break;
             if (is_a && rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);     // both blocks' bytes
