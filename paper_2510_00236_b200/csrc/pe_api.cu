@@ -109,6 +109,20 @@ static pe_status_t make_operand_map(CUtensorMap* m, const void* base, int B, int
 // gain nothing from the tensor cores and take the SIMT kernel (fp32 squares).
 constexpr long long TOKEN_TC_MIN_ROWS = 256;
 
+// [d_out, d_in] fp32 output viewed as a 2-D tensor (d_in, d_out); one box = 32 columns (128 bytes,
+// 128-byte swizzled) x 32 rows, the piece one epilogue warp stages at a time.
+static pe_status_t make_output_map(CUtensorMap* m, float* base, int d_in, int d_out) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return PE_ERR_CUDA;
+  cuuint64_t dims[2] = {(cuuint64_t)d_in, (cuuint64_t)d_out};
+  cuuint64_t strides[1] = {(cuuint64_t)d_in * 4ull};
+  cuuint32_t box[2] = {32u, 32u};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? PE_OK : PE_ERR_CUDA;
+}
+
 static bool tc_shape_ok(int B, int T, int d_in, int d_out);
 static bool token_tc_ok(int B, int T, int d_in, int d_out) {
   return tc_shape_ok(B, T, d_in, d_out) && (long long)B * T >= TOKEN_TC_MIN_ROWS;
@@ -142,8 +156,8 @@ static pe_status_t zero_outputs(float* a, float* b, size_t bytes, cudaStream_t s
 }
 
 template <int PHI, bool TF32, int NT, int MEAN>
-static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& mx, const CUtensorMap& my, const TcParams& p,
-                                  dim3 grid, cudaStream_t st) {
+static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& mm,
+                                  const CUtensorMap& ms, const TcParams& p, dim3 grid, cudaStream_t st) {
   constexpr int smem = TcOperand<TF32, NT>::SMEM_BYTES;
   if (!di->tc_attr_set[slot]) {
     if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
@@ -152,7 +166,7 @@ static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& m
     }
     di->tc_attr_set[slot] = true;
   }
-  tc_stats_kernel<PHI, TF32, NT, MEAN><<<grid, TC_THREADS, smem, st>>>(mx, my, p);
+  tc_stats_kernel<PHI, TF32, NT, MEAN><<<grid, TC_THREADS, smem, st>>>(mx, my, mm, ms, p);
   return check_launch();
 }
 
@@ -173,6 +187,11 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   if (rc != PE_OK) return rc;
   rc = make_operand_map(&my, dY, B, T, d_out, tf32, box_feats, box_tokens);
   if (rc != PE_OK) return rc;
+  CUtensorMap mm, ms;       // an output that is not wanted gets the other one's map and is never used
+  rc = make_output_map(&mm, out_mean ? out_mean : out_stat, d_in, d_out);
+  if (rc != PE_OK) return rc;
+  rc = make_output_map(&ms, out_stat ? out_stat : out_mean, d_in, d_out);
+  if (rc != PE_OK) return rc;
   const int tiles_n = (d_in + nt - 1) / nt, pairs_m = (d_out + TC_PAIR_M - 1) / TC_PAIR_M;
   if (tiles_n > 65535 || pairs_m > (1 << 29)) return PE_ERR_DIM;
   const int ns = choose_nsplit((long long)tiles_n * pairs_m, B, T, di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 16);
@@ -184,18 +203,18 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = per_example;
   p.out_mean = out_mean; p.out_stat = out_stat; p.dev_status = di->status_ptr;
   dim3 grid(2 * pairs_m, tiles_n, ns);
-  if (tf32) return launch_tc_inst<0, true, 256, MEAN_NONE>(di, 5, mx, my, p, grid, st);
-  if (!per_example) return launch_tc_inst<0, false, 256, MEAN_NONE>(di, 4, mx, my, p, grid, st);
+  if (tf32) return launch_tc_inst<0, true, 256, MEAN_NONE>(di, 5, mx, my, mm, ms, p, grid, st);
+  if (!per_example) return launch_tc_inst<0, false, 256, MEAN_NONE>(di, 4, mx, my, mm, ms, p, grid, st);
   if (mean_regs) {
-    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, MEAN_REGS>(di, 0, mx, my, p, grid, st);
-    return launch_tc_inst<2, false, 128, MEAN_REGS>(di, 1, mx, my, p, grid, st);
+    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, MEAN_REGS>(di, 0, mx, my, mm, ms, p, grid, st);
+    return launch_tc_inst<2, false, 128, MEAN_REGS>(di, 1, mx, my, mm, ms, p, grid, st);
   }
   if (both) {
-    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, MEAN_TMEM>(di, 6, mx, my, p, grid, st);
-    return launch_tc_inst<2, false, 256, MEAN_TMEM>(di, 7, mx, my, p, grid, st);
+    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, MEAN_TMEM>(di, 6, mx, my, mm, ms, p, grid, st);
+    return launch_tc_inst<2, false, 256, MEAN_TMEM>(di, 7, mx, my, mm, ms, p, grid, st);
   }
-  if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, MEAN_NONE>(di, 2, mx, my, p, grid, st);
-  return launch_tc_inst<2, false, 256, MEAN_NONE>(di, 3, mx, my, p, grid, st);
+  if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, MEAN_NONE>(di, 2, mx, my, mm, ms, p, grid, st);
+  return launch_tc_inst<2, false, 256, MEAN_NONE>(di, 3, mx, my, mm, ms, p, grid, st);
 }
 
 template <typename TIn, int MODE>

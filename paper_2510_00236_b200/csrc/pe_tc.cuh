@@ -89,8 +89,8 @@ struct TcParams {
   int nsplit;          // batch slices (gridDim.z); > 1 => outputs pre-zeroed, partials added atomically
   int per_example;     // 1: reset the accumulator for every example and apply phi (statistics)
                        // 0: one accumulation over the whole slice (plain contraction, phi = identity)
-  float* out_mean;     // may be NULL
-  float* out_stat;     // may be NULL
+  float* out_mean;     // may be NULL; written through tmap_mean
+  float* out_stat;     // may be NULL; written through tmap_stat
   unsigned int* dev_status;
 };
 
@@ -127,7 +127,8 @@ enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2 };   // where sum_b G_b
 // gridDim = (2 * ceil(d_out / 256), ceil(d_in / NT), nsplit); blockIdx.x = 2 * pair row + rank in pair.
 template <int PHI, bool TF32, int NT, int MEAN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
-tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy, TcParams p) {
+tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
+                const __grid_constant__ CUtensorMap tmap_mean, const __grid_constant__ CUtensorMap tmap_stat, TcParams p) {
   using namespace sm100;
   using Op = TcOperand<TF32, NT>;
   static_assert(MEAN != MEAN_REGS || NT == 128, "two running sums only fit the registers at NT = 128");
@@ -326,50 +327,70 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         }
       }
     }
-    // The tensor-memory loads below are warp-wide instructions: the condition around them is made
-    // uniform over the warp and they stay outside every per-lane condition.
+    // Final write-out.  By now every MMA of this block has completed (the last accumulator was
+    // committed after them), so the operand ring is free: each warp stages its 32-row x COLS-column
+    // piece of an output there, 32 columns (one 128-byte-swizzled 4 KiB panel) at a time, and one lane
+    // hands the panels to TMA, which stores them (or, with a split batch, adds them) and drops
+    // whatever lies outside the matrix.  The tensor-memory loads are warp-wide instructions: the
+    // condition around them is made uniform over the warp.
     ok = __all_sync(0xffffffffu, ok);
     if (ok && n_acc > 0) {
-      const int o = tile_m * TC_TILE_M + q * 32 + lane;
-      const int i_base = tile_n * NT + h * COLS;
-      const bool row_ok = o < p.d_out;
-      float* mrow = ((KEEP_MEAN || MEAN == MEAN_TMEM) && p.out_mean && row_ok) ? p.out_mean + (size_t)o * p.d_in : nullptr;
-      float* srow = (p.out_stat && row_ok) ? p.out_stat + (size_t)o * p.d_in : nullptr;
-      if constexpr (MEAN == MEAN_TMEM) {
-        // the running sum of G_b comes out of tensor memory, 32 columns at a time
-        const uint32_t maddr = lane_base + (uint32_t)(MEAN_COL0 + h * COLS);
+      constexpr int PANELS = COLS / 32;
+      const uint32_t stage_base = smem_base + (uint32_t)(warp - 4) * (4u * 4096u);     // 16 KiB per epilogue warp
+      const int row0 = tile_m * TC_TILE_M + q * 32;
+      const int col0 = tile_n * NT + h * COLS;
+      auto put_panel = [&](uint32_t panel_addr, const float* v) {      // v: this lane's 32 consecutive columns
+        uint8_t* dst = smem_gen + (panel_addr - smem_base) + lane * 128;
 #pragma unroll
-        for (int c = 0; c < COLS / 32; ++c) {
-          uint32_t m[32];
-          tmem_ld_32x32b_x32_wait(maddr + c * 32, m);
-#pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const int i = i_base + c * 32 + j;
-            if (mrow && i < p.d_in) {
-              if (p.nsplit == 1) *reinterpret_cast<float4*>(mrow + i) = make_float4(__uint_as_float(m[j]), __uint_as_float(m[j + 1]), __uint_as_float(m[j + 2]), __uint_as_float(m[j + 3]));
-              else red_add_f32x4(mrow + i, __uint_as_float(m[j]), __uint_as_float(m[j + 1]), __uint_as_float(m[j + 2]), __uint_as_float(m[j + 3]));
+        for (int k = 0; k < 8; ++k)
+          *reinterpret_cast<float4*>(dst + ((k ^ (lane & 7)) << 4)) = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+      };
+      auto send = [&](const CUtensorMap* tm, uint32_t first_panel) {
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0 && row0 < p.d_out) {
+          for (int c = 0; c < PANELS; ++c) {
+            if (col0 + c * 32 < p.d_in) {
+              if (p.nsplit == 1) tma_store_2d<false>(tm, first_panel + c * 4096, col0 + c * 32, row0);
+              else tma_store_2d<true>(tm, first_panel + c * 4096, col0 + c * 32, row0);
             }
           }
+          bulk_commit_group();
         }
-        mrow = nullptr;
-      }
+      };
+      // sum_b phi(G_b), or the plain contraction when PHI == 0
+      if (p.out_stat) {
 #pragma unroll
-      for (int j = 0; j < COLS; j += 4) {
-        const int i = i_base + j;
-        if (i < p.d_in) {                                      // d_in % 8 == 0: a group of 4 is all in or all out
-          float4 vm = make_float4(0.f, 0.f, 0.f, 0.f), vs;
-          if (KEEP_MEAN) vm = make_float4(acc_mean[j], acc_mean[j + 1], acc_mean[j + 2], acc_mean[j + 3]);
-          if (PHI != 0) vs = make_float4(acc_stat[j], acc_stat[j + 1], acc_stat[j + 2], acc_stat[j + 3]);
-          else vs = vm;
-          if (p.nsplit == 1) {
-            if (mrow) *reinterpret_cast<float4*>(mrow + i) = vm;
-            if (srow) *reinterpret_cast<float4*>(srow + i) = vs;
-          } else {
-            if (mrow) red_add_f32x4(mrow + i, vm.x, vm.y, vm.z, vm.w);
-            if (srow) red_add_f32x4(srow + i, vs.x, vs.y, vs.z, vs.w);
-          }
-        }
+        for (int c = 0; c < PANELS; ++c) put_panel(stage_base + c * 4096, (PHI != 0) ? &acc_stat[c * 32] : &acc_mean[c * 32]);
+        send(&tmap_stat, stage_base);
       }
+      // sum_b G_b
+      if (p.out_mean && (KEEP_MEAN || MEAN == MEAN_TMEM)) {
+        uint32_t first = stage_base + PANELS * 4096;          // MEAN_REGS / PHI == 0: second half of the warp's 16 KiB
+        if constexpr (MEAN == MEAN_TMEM) {
+          // all 16 KiB are needed again: wait until TMA has read the first output out of them
+          if (lane == 0) bulk_wait_read_all();
+          __syncwarp();
+          first = stage_base;
+          const uint32_t maddr = lane_base + (uint32_t)(MEAN_COL0 + h * COLS);
+#pragma unroll
+          for (int c = 0; c < PANELS; ++c) {
+            uint32_t m[32];
+            tmem_ld_32x32b_x32_wait(maddr + c * 32, m);
+            put_panel(first + c * 4096, reinterpret_cast<const float*>(m));
+          }
+        } else if constexpr (KEEP_MEAN) {
+          if constexpr (PANELS * 2 * 4096 > 4 * 4096) {       // PHI == 0 at NT = 256: one output only ever
+            if (lane == 0) bulk_wait_read_all();
+            __syncwarp();
+            first = stage_base;
+          }
+#pragma unroll
+          for (int c = 0; c < PANELS; ++c) put_panel(first + c * 4096, &acc_mean[c * 32]);
+        }
+        send(&tmap_mean, first);
+      }
+      if (lane == 0) bulk_wait_read_all();       // shared memory must outlive TMA's reads
     }
     __syncwarp();
   }
