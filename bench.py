@@ -11,6 +11,7 @@ One step = one pass of the whole path over one batch of a transformer-MLP-shaped
 The metric is the contraction throughput of the step, 3 x 2*B*T*d_in*d_out flops per step, in TFLOP/s.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c4] [--impl ours|reference]
+  python bench.py --sweep          (single-layer shape sweep, one JSON line per point)
 
 With N > 1 (torchrun) every rank runs an independent replica of the same workload on its own GPU
 (the path has no exchange step); the reported value is the sum over ranks divided by the slowest
@@ -209,6 +210,46 @@ def context_numbers(torch, pe, st, li, peaks, dev):
     return extra
 
 
+def run_sweep(args):
+    """Shape sweep of a single bf16 layer (d_in = d_out): one JSON line per point with the time of
+    pe_linear_stats(square, both outputs), of the statistic alone, and of the cuBLAS batch
+    weight-gradient GEMM of the same shape."""
+    import torch
+    import paper_2510_00236_b200 as pe
+    from paper_2510_00236_b200 import inputs
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    pe.load_library()
+    peaks = measured_peaks()
+    for d in inputs.SWEEP_D:
+        for (B, T) in inputs.SWEEP_BT:
+            bytes_in = 2.0 * B * T * 2 * d
+            nsets = max(1, min(6, int(300e6 // bytes_in)))      # rotate input sets until they exceed L2
+            sets = [inputs.config5_point(B, T, d, dev, seed=inputs.BASE_SEED + 5 + 97 * k) for k in range(nsets)]
+            mean = torch.empty((d, d), device=dev)
+            stat = torch.empty((d, d), device=dev)
+            flops = 2.0 * B * T * d * d
+            med_b, best_b = time_each(torch, lambda i: pe.pe_linear_stats(sets[i % nsets].X, sets[i % nsets].dY, pe.PHI_SQUARE, mean, stat), iters=12)
+            med_s, best_s = time_each(torch, lambda i: pe.pe_linear_stats(sets[i % nsets].X, sets[i % nsets].dY, pe.PHI_SQUARE, None, stat), iters=12)
+            med_g, best_g = time_each(torch, lambda i: torch.matmul(sets[i % nsets].dY.view(B * T, d).t(), sets[i % nsets].X.view(B * T, d)), iters=12)
+            status, detail = pe.pe_get_async_status(dev)
+            assert status == 0, (status, detail)
+            # bounds per point: tensor pipe, the fp32 epilogue (2 ops per example and output entry on
+            # 128 lanes x 148 SMs, packed 2-wide at best), and HBM
+            t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
+            t_hbm = (bytes_in + 8.0 * d * d) / (peaks["hbm_gbs"] * 1e9)
+            print(json.dumps({
+                "sweep_point": {"B": B, "T": T, "d_in": d, "d_out": d}, "input_sets": nsets,
+                "both_outputs_us": med_b * 1e3, "both_outputs_tflops": flops / med_b / 1e9,
+                "both_outputs_frac_of_peak": flops / med_b / 1e9 / peaks["bf16_tflops"],
+                "stat_only_us": med_s * 1e3, "stat_only_tflops": flops / med_s / 1e9,
+                "cublas_gemm_us": med_g * 1e3, "cublas_gemm_tflops": flops / med_g / 1e9,
+                "overhead_both_vs_gemm": med_b / med_g, "overhead_stat_vs_gemm": med_s / med_g,
+                "bound_tensor_us": t_tensor * 1e6, "bound_hbm_us": t_hbm * 1e6, "peak_source": peaks["source"]}), flush=True)
+            del sets, mean, stat
+            torch.cuda.empty_cache()
+
+
 def oracle_sample(inputs, workload, n_rows, n_cols):
     """Column-gathered sub-layer of the workload for the CPU oracle (full B and T)."""
     import numpy as np
@@ -278,11 +319,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="shape sweep (B, T, d) instead of the step benchmark; one JSON line per point")
     ap.add_argument("--quick", action="store_true", help="timed region only: skip the per-kernel context numbers and the CPU baseline")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.sweep:
+        run_sweep(args)
         return
 
     import torch
