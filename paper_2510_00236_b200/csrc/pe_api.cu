@@ -23,6 +23,7 @@ static std::atomic<int> g_path{PE_PATH_AUTO};
 static std::atomic<int> g_last_path{PE_PATH_AUTO};
 static std::atomic<long long> g_launches{0};
 constexpr int TC_MEAN_TMEM_MIN_T = 2048;
+constexpr int TC_BAND = 8;          // pair rows per band of the tile order (8 x 256 rows of d_out)
 
 constexpr int MAX_DEVICES = 64;
 struct DeviceInfo {
@@ -193,7 +194,7 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   rc = make_output_map(&ms, out_stat ? out_stat : out_mean, d_in, d_out);
   if (rc != PE_OK) return rc;
   const int tiles_n = (d_in + nt - 1) / nt, pairs_m = (d_out + TC_PAIR_M - 1) / TC_PAIR_M;
-  if (tiles_n > 65535 || pairs_m > (1 << 29)) return PE_ERR_DIM;
+  if ((long long)tiles_n * pairs_m > (1ll << 29)) return PE_ERR_DIM;
   const int ns = choose_nsplit((long long)tiles_n * pairs_m, B, T, di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 16);
   if (ns > 1) {
     rc = zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
@@ -201,8 +202,9 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   }
   TcParams p;
   p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = per_example;
+  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
   p.out_mean = out_mean; p.out_stat = out_stat; p.dev_status = di->status_ptr;
-  dim3 grid(2 * pairs_m, tiles_n, ns);
+  dim3 grid(2 * pairs_m * tiles_n, 1, ns);
   if (tf32) return launch_tc_inst<0, true, 256, MEAN_NONE>(di, 5, mx, my, mm, ms, p, grid, st);
   if (!per_example) return launch_tc_inst<0, false, 256, MEAN_NONE>(di, 4, mx, my, mm, ms, p, grid, st);
   if (mean_regs) {

@@ -86,6 +86,7 @@ enum : int { TC_WAIT_EMPTY = 1, TC_WAIT_FULL = 2, TC_WAIT_ACC_EMPTY = 3, TC_WAIT
 
 struct TcParams {
   int B, T, d_in, d_out;
+  int pairs_m, tiles_n, band;   // tile grid: 256-row pair rows x NT-column tiles; pair rows per band of the tile order
   int nsplit;          // batch slices (gridDim.z); > 1 => outputs pre-zeroed, partials added atomically
   int per_example;     // 1: reset the accumulator for every example and apply phi (statistics)
                        // 0: one accumulation over the whole slice (plain contraction, phi = identity)
@@ -93,6 +94,19 @@ struct TcParams {
   float* out_stat;     // may be NULL; written through tmap_stat
   unsigned int* dev_status;
 };
+
+// Tile order.  Pairs that run at the same time should share operand panels in L2, so consecutive
+// pair indices sweep the d_in tiles inside a band of p.band pair rows before moving to the next band:
+// the ~74 resident pairs then touch about band*256 columns of dY and 74/band*NT columns of X per
+// example instead of all of dY.  Returns this block's 128-row tile of d_out and NT-column tile of d_in.
+__device__ __forceinline__ void tc_tile_of_block(const TcParams& p, uint32_t rank, int& tile_m, int& tile_n) {
+  const int pair_id = blockIdx.x >> 1;
+  const int per_band = p.band * p.tiles_n;
+  const int band = pair_id / per_band, r = pair_id - band * per_band;
+  const int rows = min(p.band, p.pairs_m - band * p.band);      // pair rows in this (possibly last, shorter) band
+  tile_n = r / rows;
+  tile_m = 2 * (band * p.band + (r - tile_n * rows)) + (int)rank;
+}
 
 template <int PHI>
 __device__ __forceinline__ float phi_apply(float g) {
@@ -124,7 +138,7 @@ struct StageWalk {
 
 enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2 };   // where sum_b G_b is kept in per-example mode
 
-// gridDim = (2 * ceil(d_out / 256), ceil(d_in / NT), nsplit); blockIdx.x = 2 * pair row + rank in pair.
+// gridDim = (2 * pairs_m * tiles_n, 1, nsplit); blockIdx.x = 2 * (pair index in the tile order) + rank in pair.
 template <int PHI, bool TF32, int NT, int MEAN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
@@ -155,8 +169,6 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair
-  const int tile_m = blockIdx.x;                    // 128-row tile of d_out (pair row = blockIdx.x / 2)
-  const int tile_n = blockIdx.y;                    // NT-column tile of d_in
   const int b_begin = (int)(((long long)p.B * blockIdx.z) / p.nsplit);
   const int b_end = (int)(((long long)p.B * (blockIdx.z + 1)) / p.nsplit);
   const int nb = b_end - b_begin;
@@ -188,6 +200,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       // 2*kc+1 to its second (issuer 1, odd slots); the ring has an even number of slots.
       if (lane == 0) {
         const bool is_a = (warp == 0);
+        int tile_m, tile_n;
+        tc_tile_of_block(p, rank, tile_m, tile_n);
         const CUtensorMap* tmap = is_a ? &tmap_dy : &tmap_x;
         const int c0 = is_a ? tile_m * TC_TILE_M : tile_n * NT + (int)rank * Op::B_FEATS;   // first feature of this warp's boxes
         const int n_boxes = is_a ? Op::A_BOXES : Op::B_BOXES;
@@ -336,6 +350,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     ok = __all_sync(0xffffffffu, ok);
     if (ok && n_acc > 0) {
       constexpr int PANELS = COLS / 32;
+      int tile_m, tile_n;
+      tc_tile_of_block(p, rank, tile_m, tile_n);
       const uint32_t stage_base = smem_base + (uint32_t)(warp - 4) * (4u * 4096u);     // 16 KiB per epilogue warp
       const int row0 = tile_m * TC_TILE_M + q * 32;
       const int col0 = tile_n * NT + h * COLS;
