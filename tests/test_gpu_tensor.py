@@ -41,6 +41,9 @@ def test_structured_single_tile_catches_layout_mistakes():
     (1, 1000, 256, 128),    # single example
     (70, 48, 8, 8),         # smallest widths the path takes, batch split across blocks
     (40, 96, 384, 256),
+    (130, 32, 264, 392),    # many short sequences: 32-token stages, batch split
+    (21, 64, 136, 520),     # two short stages per example
+    (11, 33, 128, 256),     # one full and one nearly empty short stage
 ])
 def test_tensor_small_shapes_full_comparison(B, T, d_in, d_out):
     li = inputs.gaussian_layer(B, T, d_in, d_out, seed=300 + 7 * B + T, device=DEV)
@@ -50,7 +53,7 @@ def test_tensor_small_shapes_full_comparison(B, T, d_in, d_out):
     assert pe.pe_last_path() == (pe.PATH_TENSOR if B * T >= 256 else pe.PATH_SIMT)
 
 
-@pytest.mark.parametrize("B,T,d_in,d_out", [(5, 200, 136, 264), (9, 16, 320, 192), (33, 300, 520, 264), (2, 1, 64, 72)])
+@pytest.mark.parametrize("B,T,d_in,d_out", [(5, 200, 136, 264), (9, 16, 320, 192), (33, 300, 520, 264), (2, 1, 64, 72), (75, 40, 520, 264)])
 def test_single_output_calls_use_the_wide_tile_and_match(B, T, d_in, d_out):
     """Asking for only sum_b phi(G_b) (or only sum_b G_b) takes the 256 x 256 pair tile (or the plain
     contraction); both must agree with the oracle like the two-output call does."""
