@@ -48,27 +48,20 @@ constexpr int TC_TMEM_COLS = 512;
 constexpr int TC_THREADS = 384;
 constexpr int TC_REGS_CONTROL = 64;     // setmaxnreg of warps 0..3
 constexpr int TC_REGS_EPILOGUE = 216;   // setmaxnreg of warps 4..11  (4*32*64 + 8*32*216 = 63488 <= 65536)
-constexpr int TC_BAR_BYTES = 512;    // up to 16 + 16 stage barriers, 4 + 4 accumulator barriers, two words
+constexpr int TC_BAR_BYTES = 512;
 constexpr int TC_SMEM_BUDGET = 200 * 1024;   // operand ring; leaves room for barriers and alignment slack
 
 // Operand element type of the MMA.  bf16 (kind::f16, 16 tokens per instruction) for the per-example
 // statistics; tf32 (kind::tf32, fp32 storage, 8 tokens per instruction) for the per-token statistic,
 // whose squared operands need more than bf16's 8 significant bits.  NT = d_in columns per pair tile.
-// Default tokens per pipeline stage: 128 for the 256 x 128 tile, 64 for the 256 x 256 tile, 32 for
-// tf32.  Short sequences (T <= 64) take 32-token stages instead: an example then occupies one or two
-// small slots, so many more examples are in flight in the same shared memory.
-__host__ __device__ constexpr int tc_default_bk(bool tf32, int nt) { return tf32 ? 32 : (nt == 128 ? 128 : 64); }
-constexpr int TC_SHORT_BK = 32;
-constexpr int TC_SHORT_T = 64;     // sequences up to this length use TC_SHORT_BK
-
-template <bool TF32, int NT, int BK_ = tc_default_bk(TF32, NT)>
+template <bool TF32, int NT>
 struct TcOperand {
   static constexpr int ELEM_BYTES = TF32 ? 4 : 2;
   static constexpr int BOX_FEATS = 128 / ELEM_BYTES;            // features per 128-byte swizzle row: 64 | 32
   // tokens per pipeline stage (one TMA box is BK tokens tall), chosen so that the ring has an EVEN
   // number of stages: with two MMA issuers taking alternate stages every slot then always belongs
   // to the same issuer (see the parity note at the issuer's wait).
-  static constexpr int BK = BK_;
+  static constexpr int BK = TF32 ? 32 : (NT == 128 ? 128 : 64);
   static constexpr int MMA_K = 32 / ELEM_BYTES;                 // tokens per MMA instruction: 16 | 8
   static constexpr int BOX_BYTES = 128 * BK;                    // one box: BK tokens x 128 bytes
   static constexpr int A_BOXES = TC_TILE_M / BOX_FEATS;         // this block's 128 rows of dY^T
@@ -77,7 +70,7 @@ struct TcOperand {
   static constexpr int A_BYTES = A_BOXES * BOX_BYTES;           // 32 KiB (NT = 128) | 16 KiB
   static constexpr int B_BYTES = B_BOXES * BOX_BYTES;           // 16 KiB
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;         // per block: 48 KiB | 32 KiB
-  static constexpr int STAGES = (TC_SMEM_BUDGET / STAGE_BYTES) & ~1;   // 4 | 6 (16 | 12 with 32-token stages)
+  static constexpr int STAGES = TC_SMEM_BUDGET / STAGE_BYTES;   // 4 | 6
   static_assert(STAGES % 2 == 0, "slots must alternate between the two issuers");
   static constexpr int K_STEP_BYTES = MMA_K * 128;              // smem advance per MMA: 2048 | 1024
   static constexpr int ACC_BUFS = TC_TMEM_COLS / NT;            // 4 | 2 accumulators in tensor memory
@@ -146,12 +139,12 @@ struct StageWalk {
 enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2 };   // where sum_b G_b is kept in per-example mode
 
 // gridDim = (2 * pairs_m * tiles_n, 1, nsplit); blockIdx.x = 2 * (pair index in the tile order) + rank in pair.
-template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT)>
+template <int PHI, bool TF32, int NT, int MEAN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
                 const __grid_constant__ CUtensorMap tmap_mean, const __grid_constant__ CUtensorMap tmap_stat, TcParams p) {
   using namespace sm100;
-  using Op = TcOperand<TF32, NT, BKT>;
+  using Op = TcOperand<TF32, NT>;
   static_assert(MEAN != MEAN_REGS || NT == 128, "two running sums only fit the registers at NT = 128");
   static_assert(MEAN != MEAN_TMEM || (NT == 256 && PHI != 0), "the tensor-memory mean sits beside one 256-column accumulator");
   constexpr int STAGES = Op::STAGES, BK = Op::BK;
@@ -331,22 +324,20 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         tmem_st_wait();
         continue;
       }
-      // 64 columns per tensor-memory read: every read is a round trip of a few hundred cycles that
-      // nothing else in this warp overlaps, so fewer and wider reads shorten the per-example chain.
 #pragma unroll
-      for (int c = 0; c < COLS / 64; ++c) {
-        uint32_t r[64];
-        tmem_ld_32x32b_x64_wait(taddr + c * 64, r);
-        if (c == COLS / 64 - 1) {
+      for (int c = 0; c < COLS / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32_wait(taddr + c * 32, r);
+        if (c == COLS / 32 - 1) {
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));   // buffer free for the issuer's next example
         }
 #pragma unroll
-        for (int j = 0; j < 64; ++j) {
+        for (int j = 0; j < 32; ++j) {
           const float g = __uint_as_float(r[j]);
-          if (KEEP_MEAN) acc_mean[c * 64 + j] += g;
-          if (PHI != 0) acc_stat[c * 64 + j] += phi_apply<PHI>(g);
+          if (KEEP_MEAN) acc_mean[c * 32 + j] += g;
+          if (PHI != 0) acc_stat[c * 32 + j] += phi_apply<PHI>(g);
         }
       }
     }
