@@ -5,7 +5,7 @@ One step = one pass of the whole path over one batch of a transformer-MLP-shaped
 (B=64, T=256, d_in=512, d_out=2048; X ~ N(0,1), dY ~ N(0,1/T) with 10% of sequences x5):
   pe_linear_stats(square)  -> sum_b G_b and sum_b G_b^2      (tcgen05 kernel)
   pe_linear_stats(sign)    -> sum_b sign(G_b)                (tcgen05 kernel)
-  pe_token_sqstats         -> sum_{b,t} dY^2 X^2             (square pre-pass + tcgen05 kernel)
+  pe_token_sqstats         -> sum_{b,t} dY^2 X^2             (squares on chip, tf32 tcgen05 kernel)
   microadam_step           on fp32 master weights (+ bf16 copy)
   microsignsgd_step        on a second set of master weights (+ bf16 copy)
 The metric is the contraction throughput of the step, 3 x 2*B*T*d_in*d_out flops per step, in TFLOP/s.
@@ -133,7 +133,6 @@ def make_state(pe, inputs, torch, name, dev, seed_offset=0):
         "shape": (B, T, d_in, d_out), "sets": sets,
         "mean": torch.empty((d_out, d_in), **f32), "sq": torch.empty((d_out, d_in), **f32),
         "sgn": torch.empty((d_out, d_in), **f32), "tok": torch.empty((d_out, d_in), **f32),
-        "ws": torch.empty(max(1, pe.pe_token_sqstats_workspace_bytes(B, T, d_in, d_out)), dtype=torch.uint8, device=dev),
         "theta": sets[0].W.clone(), "m": torch.zeros((d_out, d_in), **f32), "v": torch.zeros((d_out, d_in), **f32),
         "theta_lp": torch.empty((d_out, d_in), dtype=torch.bfloat16, device=dev),
         "theta2": sets[0].W.clone(), "m2": torch.zeros((d_out, d_in), **f32),
@@ -154,7 +153,7 @@ def run_step(pe, st, i, X=None, dY=None, ev=None):
     if ev is not None:
         ev[1].record()
     pe.pe_linear_stats(X, dY, pe.PHI_SIGN, None, st["sgn"])
-    pe.pe_token_sqstats(X, dY, st["tok"], st["ws"])
+    pe.pe_token_sqstats(X, dY, st["tok"])
     pe.microadam_step(st["theta"], st["m"], st["v"], st["mean"], st["sq"], B, step=i + 1, theta_lp=st["theta_lp"], **ADAM)
     pe.microsignsgd_step(st["theta2"], st["m2"], st["sgn"], B, theta_lp=st["theta2_lp"], **SIGN)
 
@@ -193,7 +192,7 @@ def context_numbers(torch, pe, st, li, peaks, dev):
     extra["pe_linear_stats_square_us"] = {"median": med * 1e3, "best": best * 1e3, "tflops_median": flops_one / med / 1e9}
     med_s, best_s = time_each(torch, lambda i: pe.pe_linear_stats(li.X, li.dY, pe.PHI_SIGN, None, st["sgn"]))
     extra["pe_linear_stats_sign_us"] = {"median": med_s * 1e3, "best": best_s * 1e3, "tflops_median": flops_one / med_s / 1e9}
-    med_t, best_t = time_each(torch, lambda i: pe.pe_token_sqstats(li.X, li.dY, st["tok"], st["ws"]))
+    med_t, best_t = time_each(torch, lambda i: pe.pe_token_sqstats(li.X, li.dY, st["tok"]))
     extra["pe_token_sqstats_us"] = {"median": med_t * 1e3, "best": best_t * 1e3, "tflops_median": flops_one / med_t / 1e9}
     A2, B2 = li.dY.view(B * T, d_out), li.X.view(B * T, d_in)
     med_g, best_g = time_each(torch, lambda i: torch.matmul(A2.t(), B2))

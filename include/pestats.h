@@ -78,37 +78,48 @@ pe_status_t pe_linear_stats_f32(const float* X, const float* dY, int B, int T, i
 /*
  * Per-token second moment (Section 2.3, the "per-token" alternative):
  *     out_stat[o,i] = sum_{b,t} dY[b,t,o]^2 * X[b,t,i]^2  =  ((dY o dY)^T (X o X))[o,i].
- * B and T only enter through the row count B*T.  bf16 inputs.  On the tensor-core path (taken when
- * the shape allows it and B*T >= 256) the squared operands are rounded to tf32 (11 significant bits,
- * so every entry is within about 1e-3 relative of the exact sum) and staged as fp32 in `workspace`
- * (device memory, 256-byte aligned, at least pe_token_sqstats_workspace_bytes() bytes, contents
- * undefined afterwards); the SIMT path squares in fp32 and ignores the workspace (it may then be
- * NULL).
+ * B and T only enter through the row count B*T.  bf16 inputs, 16-byte aligned; out_stat fp32
+ * [d_out, d_in], 16-byte aligned, overwritten.  On the tensor-core path (taken when the shape allows
+ * it and B*T >= 256) one kernel squares the operands on chip (exact in fp32), rounds each square to
+ * tf32 (11 significant bits, so every entry is within about 1e-3 relative of the exact sum) and
+ * contracts them; nothing is staged in global memory.  Otherwise the SIMT kernel squares in fp32.
  */
 pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_in, int d_out,
-                             float* out_stat, void* workspace, size_t workspace_bytes,
-                             pe_stream_t stream);
+                             float* out_stat, pe_stream_t stream);
 pe_status_t pe_token_sqstats_f32(const float* X, const float* dY, int B, int T, int d_in, int d_out,
                                  float* out_stat, pe_stream_t stream);
-/* Bytes of workspace pe_token_sqstats needs for this shape under the current path setting (0 when
- * the SIMT kernel will be used). */
-size_t pe_token_sqstats_workspace_bytes(int B, int T, int d_in, int d_out);
 
 /*
- * pe_token_sqstats for callers that have no device memory to give as workspace and no way to get
- * some.  (The paper has no counterpart; this is a convenience of this library.)  Typical cases: a
+ * The same statistic in two passes (Section 2.3): a streaming kernel writes the tf32-rounded squares
+ * as fp32 into `workspace` (device memory, 256-byte aligned, at least
+ * pe_token_sqstats_staged_workspace_bytes() bytes, contents undefined afterwards), then the plain
+ * tensor-core contraction reads them back.  Slower than pe_token_sqstats (it moves three times the
+ * bytes); kept as an independent second route to the same numbers and as the kernel behind
+ * pe_token_sqstats_static.  The SIMT path ignores the workspace (it may then be NULL).
+ */
+pe_status_t pe_token_sqstats_staged(const void* X, const void* dY, int B, int T, int d_in, int d_out,
+                                    float* out_stat, void* workspace, size_t workspace_bytes,
+                                    pe_stream_t stream);
+/* Bytes of workspace pe_token_sqstats_staged needs for this shape under the current path setting
+ * (0 when the SIMT kernel will be used). */
+size_t pe_token_sqstats_staged_workspace_bytes(int B, int T, int d_in, int d_out);
+
+/*
+ * pe_token_sqstats_staged for callers that have no device memory to give as workspace and no way to
+ * get some.  (The paper has no counterpart; this is a convenience of this library.)  Typical cases: a
  * plug-in that is handed input and output pointers but no allocator; a process whose framework
  * reserved all of the GPU's memory in its own pool at start-up, so that cudaMalloc would fail; a
  * latency-critical loop that must not pay cudaMalloc / cudaFree's device-wide synchronisation.
  *
- * Same arguments, result and path selection as pe_token_sqstats, minus the workspace: the fp32
+ * Same arguments, result and path selection as pe_token_sqstats_staged, minus the workspace: the fp32
  * staging of the squared operands lives in an array of PE_STATIC_SCRATCH_BYTES bytes that is part
  * of the library's device image, so every GPU on which the library is used holds that much memory
  * from module load until the process exits.  The call allocates and frees nothing, on the device or
  * through any library.
  *
- * Limit: shapes whose staging (pe_token_sqstats_workspace_bytes) exceeds PE_STATIC_SCRATCH_BYTES
- * are refused with PE_ERR_WORKSPACE and nothing is enqueued; use pe_token_sqstats with your own
+ * Limit: shapes whose staging (pe_token_sqstats_staged_workspace_bytes) exceeds
+ * PE_STATIC_SCRATCH_BYTES are refused with PE_ERR_WORKSPACE and nothing is enqueued; use
+ * pe_token_sqstats (which needs no workspace at all) or pe_token_sqstats_staged with your own
  * workspace for those.
  * First call on a device: looks up the array's device address (a host-side query, done once per
  * device with that device current) before enqueuing; make that first call outside any stream

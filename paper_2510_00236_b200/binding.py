@@ -14,8 +14,8 @@ import torch
 __all__ = [
     "PestatsError", "PHI_IDENTITY", "PHI_SQUARE", "PHI_SIGN", "PATH_AUTO", "PATH_SIMT", "PATH_TENSOR", "PATH_TENSOR_NARROW",
     "EXPORTED_SYMBOLS", "library_path", "load_library", "pe_linear_stats", "pe_linear_stats_f32",
-    "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_workspace_bytes", "microadam_step",
-    "microsignsgd_step", "pe_status_string", "pe_get_async_status", "pe_set_path", "pe_last_path",
+    "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_staged", "pe_token_sqstats_staged_workspace_bytes",
+    "microadam_step", "microsignsgd_step", "pe_status_string", "pe_get_async_status", "pe_set_path", "pe_last_path",
     "pe_launch_count", "pe_reset_launch_count", "pe_token_sqstats_static", "STATIC_SCRATCH_BYTES",
 ]
 
@@ -25,8 +25,8 @@ _PHI_NAMES = {"identity": PHI_IDENTITY, "square": PHI_SQUARE, "sign": PHI_SIGN}
 
 # every symbol include/pestats.h declares
 EXPORTED_SYMBOLS = [
-    "pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32",
-    "pe_token_sqstats_workspace_bytes", "microadam_step", "microsignsgd_step", "pe_status_string",
+    "pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_staged",
+    "pe_token_sqstats_staged_workspace_bytes", "microadam_step", "microsignsgd_step", "pe_status_string",
     "pe_get_async_status", "pe_set_path", "pe_last_path", "pe_launch_count", "pe_reset_launch_count",
     "pe_token_sqstats_static",
 ]
@@ -60,11 +60,12 @@ def load_library() -> ctypes.CDLL:
     vp, i, f, ll, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_longlong, ctypes.c_size_t
     lib.pe_linear_stats.argtypes = [vp, vp, i, i, i, i, i, vp, vp, vp]
     lib.pe_linear_stats_f32.argtypes = [vp, vp, i, i, i, i, i, vp, vp, vp]
-    lib.pe_token_sqstats.argtypes = [vp, vp, i, i, i, i, vp, vp, sz, vp]
+    lib.pe_token_sqstats.argtypes = [vp, vp, i, i, i, i, vp, vp]
+    lib.pe_token_sqstats_staged.argtypes = [vp, vp, i, i, i, i, vp, vp, sz, vp]
     lib.pe_token_sqstats_f32.argtypes = [vp, vp, i, i, i, i, vp, vp]
     lib.pe_token_sqstats_static.argtypes = [vp, vp, i, i, i, i, vp, vp]
-    lib.pe_token_sqstats_workspace_bytes.argtypes = [i, i, i, i]
-    lib.pe_token_sqstats_workspace_bytes.restype = sz
+    lib.pe_token_sqstats_staged_workspace_bytes.argtypes = [i, i, i, i]
+    lib.pe_token_sqstats_staged_workspace_bytes.restype = sz
     lib.microadam_step.argtypes = [vp, vp, vp, vp, vp, vp, ll, i, f, f, f, f, f, i, f, i, vp]
     lib.microsignsgd_step.argtypes = [vp, vp, vp, vp, ll, i, f, f, f, vp]
     lib.pe_status_string.argtypes = [i]
@@ -77,6 +78,7 @@ def load_library() -> ctypes.CDLL:
     lib.pe_reset_launch_count.argtypes = []
     lib.pe_reset_launch_count.restype = None
     for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_static",
+                 "pe_token_sqstats_staged",
                  "microadam_step", "microsignsgd_step", "pe_get_async_status", "pe_set_path", "pe_last_path"):
         getattr(lib, name).restype = i
     _lib = lib
@@ -155,23 +157,35 @@ def pe_linear_stats_f32(X, dY, phi, out_mean=None, out_stat=None):
     return out_mean, out_stat
 
 
-def pe_token_sqstats_workspace_bytes(B, T, d_in, d_out) -> int:
-    return int(load_library().pe_token_sqstats_workspace_bytes(int(B), int(T), int(d_in), int(d_out)))
-
-
-def pe_token_sqstats(X, dY, out_stat=None, workspace=None):
-    """Per-token second moment sum_{b,t} dY^2 X^2 (bf16 inputs).  ``workspace`` is a uint8 CUDA tensor of
-    at least pe_token_sqstats_workspace_bytes(...) bytes; allocated when omitted."""
+def pe_token_sqstats(X, dY, out_stat=None):
+    """Per-token second moment sum_{b,t} dY^2 X^2 (bf16 inputs), squared and contracted in one kernel."""
     B, T, d_in, d_out = _io_check(X, dY, torch.bfloat16)
     if out_stat is None:
         out_stat = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)
     _out_check("out_stat", out_stat, d_out, d_in)
-    need = pe_token_sqstats_workspace_bytes(B, T, d_in, d_out)
+    with _dev_ctx(X):
+        _check("pe_token_sqstats", load_library().pe_token_sqstats(
+            X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, out_stat.data_ptr(), _stream(X)))
+    return out_stat
+
+
+def pe_token_sqstats_staged_workspace_bytes(B, T, d_in, d_out) -> int:
+    return int(load_library().pe_token_sqstats_staged_workspace_bytes(int(B), int(T), int(d_in), int(d_out)))
+
+
+def pe_token_sqstats_staged(X, dY, out_stat=None, workspace=None):
+    """The same statistic in two passes through a workspace of fp32 squares.  ``workspace`` is a uint8
+    CUDA tensor of at least pe_token_sqstats_staged_workspace_bytes(...) bytes; allocated when omitted."""
+    B, T, d_in, d_out = _io_check(X, dY, torch.bfloat16)
+    if out_stat is None:
+        out_stat = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)
+    _out_check("out_stat", out_stat, d_out, d_in)
+    need = pe_token_sqstats_staged_workspace_bytes(B, T, d_in, d_out)
     if workspace is None and need > 0:
         workspace = torch.empty(need, dtype=torch.uint8, device=X.device)
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     with _dev_ctx(X):
-        _check("pe_token_sqstats", load_library().pe_token_sqstats(
+        _check("pe_token_sqstats_staged", load_library().pe_token_sqstats_staged(
             X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, out_stat.data_ptr(), _ptr(workspace), ws_bytes, _stream(X)))
     return out_stat
 

@@ -14,6 +14,7 @@
 #include "pe_optim.cuh"
 #include "pe_simt.cuh"
 #include "pe_tc.cuh"
+#include "pe_tok.cuh"
 
 namespace pe {
 
@@ -31,6 +32,7 @@ struct DeviceInfo {
   int cc_major = 0, sm_count = 0;
   unsigned int* status_ptr = nullptr;
   bool tc_attr_set[8] = {false, false, false, false, false, false, false, false};
+  bool tok_attr_set = false;
 };
 static DeviceInfo g_dev[MAX_DEVICES];
 
@@ -291,6 +293,46 @@ static int grid_for(long long work_items, int sm_count) {
   return (int)(blocks < cap ? blocks : cap);
 }
 
+// Fused per-token statistic: squares, rounds to tf32 and contracts inside one kernel.
+static pe_status_t launch_tok(DeviceInfo* di, const void* X, const void* dY, long long rows, int d_in, int d_out, float* out,
+                              cudaStream_t st) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return PE_ERR_CUDA;
+  CUtensorMap mx, my, mo;
+  auto operand_map = [&](CUtensorMap* m, const void* base, int d) {
+    cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)d * 2ull};
+    cuuint32_t box[2] = {64u, (cuuint32_t)TOK_BK};
+    cuuint32_t estr[2] = {1u, 1u};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  };
+  if (!operand_map(&mx, X, d_in) || !operand_map(&my, dY, d_out)) return PE_ERR_CUDA;
+  pe_status_t rc = make_output_map(&mo, out, d_in, d_out);
+  if (rc != PE_OK) return rc;
+  const int tiles_n = (d_in + TOK_NT - 1) / TOK_NT, pairs_m = (d_out + TC_PAIR_M - 1) / TC_PAIR_M;
+  if ((long long)tiles_n * pairs_m > (1ll << 29)) return PE_ERR_DIM;
+  const long long n_chunks = (rows + TOK_BK - 1) / TOK_BK;
+  const int units = n_chunks > (1 << 30) ? (1 << 30) : (int)n_chunks;
+  const int ns = choose_nsplit((long long)tiles_n * pairs_m, units, TOK_BK, di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 32);
+  if (ns > 1) {
+    rc = zero_outputs(out, nullptr, (size_t)d_in * d_out * sizeof(float), st);
+    if (rc != PE_OK) return rc;
+  }
+  if (!di->tok_attr_set) {
+    if (cudaFuncSetAttribute(tok_sqstats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TOK_SMEM_BYTES) != cudaSuccess) {
+      cudaGetLastError();
+      return PE_ERR_CUDA;
+    }
+    di->tok_attr_set = true;
+  }
+  TokParams p;
+  p.rows = rows; p.d_in = d_in; p.d_out = d_out; p.pairs_m = pairs_m; p.tiles_n = tiles_n;
+  p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND; p.nsplit = ns; p.dev_status = di->status_ptr;
+  tok_sqstats_kernel<<<dim3(2 * pairs_m * tiles_n, 1, ns), TC_THREADS, TOK_SMEM_BYTES, st>>>(mx, my, mo, p);
+  return check_launch();
+}
+
 }  // namespace pe
 
 using namespace pe;
@@ -308,14 +350,37 @@ pe_status_t pe_linear_stats_f32(const float* X, const float* dY, int B, int T, i
   return linear_stats_impl<float>(X, dY, B, T, d_in, d_out, phi, out_mean, out_stat, reinterpret_cast<cudaStream_t>(stream), false);
 }
 
-size_t pe_token_sqstats_workspace_bytes(int B, int T, int d_in, int d_out) {
+pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_stat,
+                             pe_stream_t stream) {
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (!out_stat) return PE_ERR_NULL;
+  pe_status_t rc = validate_stats(X, dY, B, T, d_in, d_out, out_stat, nullptr, false, 16);
+  if (rc != PE_OK) return rc;
+  DeviceInfo* di = nullptr;
+  rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  if (B == 0 || T == 0) return zero_outputs(out_stat, nullptr, (size_t)d_in * d_out * sizeof(float), st);
+  const int forced = g_path.load();
+  const long long rows = (long long)B * T;
+  const bool shape_ok = tc_shape_ok(B, T, d_in, d_out) && rows < (1ll << 31);
+  if ((forced == PE_PATH_TENSOR || forced == PE_PATH_TENSOR_NARROW) && !shape_ok) return PE_ERR_UNSUPPORTED_SHAPE;
+  if (shape_ok && rows >= TOKEN_TC_MIN_ROWS && forced != PE_PATH_SIMT) {
+    g_last_path.store(PE_PATH_TENSOR);
+    return launch_tok(di, X, dY, rows, d_in, d_out, out_stat, st);
+  }
+  g_last_path.store(PE_PATH_SIMT);
+  return launch_simt<__nv_bfloat16, MODE_TOKEN>(di, static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T,
+                                                d_in, d_out, 0, nullptr, out_stat, st);
+}
+
+size_t pe_token_sqstats_staged_workspace_bytes(int B, int T, int d_in, int d_out) {
   if (g_path.load() == PE_PATH_SIMT || !token_tc_ok(B, T, d_in, d_out)) return 0;
   const size_t rows = (size_t)B * (size_t)T;
   return align_up(rows * d_in * 4, 256) + align_up(rows * d_out * 4, 256);
 }
 
-pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_stat,
-                             void* workspace, size_t workspace_bytes, pe_stream_t stream) {
+pe_status_t pe_token_sqstats_staged(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_stat,
+                                    void* workspace, size_t workspace_bytes, pe_stream_t stream) {
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (!out_stat) return PE_ERR_NULL;
   pe_status_t rc = validate_stats(X, dY, B, T, d_in, d_out, out_stat, nullptr, false, 16);
@@ -385,7 +450,7 @@ pe_status_t pe_token_sqstats_static(const void* X, const void* dY, int B, int T,
   pe_status_t rc = validate_stats(X, dY, B, T, d_in, d_out, out_stat, nullptr, false, 16);
   if (rc != PE_OK) return rc;
   // Refuse what does not fit before touching the device.
-  if (pe_token_sqstats_workspace_bytes(B, T, d_in, d_out) > (size_t)PE_STATIC_SCRATCH_BYTES) return PE_ERR_WORKSPACE;
+  if (pe_token_sqstats_staged_workspace_bytes(B, T, d_in, d_out) > (size_t)PE_STATIC_SCRATCH_BYTES) return PE_ERR_WORKSPACE;
   DeviceInfo* di = nullptr;
   rc = device_info(&di);
   if (rc != PE_OK) return rc;
@@ -394,7 +459,7 @@ pe_status_t pe_token_sqstats_static(const void* X, const void* dY, int B, int T,
   if (rc != PE_OK) return rc;
   // Nothing in the array has to start at zero: the squaring pre-pass rewrites every element the
   // contraction reads.  Everything below only enqueues kernels and memsets on `stream`.
-  return pe_token_sqstats(X, dY, B, T, d_in, d_out, out_stat, scratch, (size_t)PE_STATIC_SCRATCH_BYTES, stream);
+  return pe_token_sqstats_staged(X, dY, B, T, d_in, d_out, out_stat, scratch, (size_t)PE_STATIC_SCRATCH_BYTES, stream);
 }
 
 pe_status_t pe_token_sqstats_f32(const float* X, const float* dY, int B, int T, int d_in, int d_out, float* out_stat,

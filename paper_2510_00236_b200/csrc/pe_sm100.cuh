@@ -111,6 +111,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* m, 
       : "memory");
 }
 
+// 2-D tiled load global -> this block's shared memory, completion counted in bytes on `bar`.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* m, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
 // 2-D tiled store shared -> global (rows / columns of the box outside the tensor are dropped).  c0 is
 // the innermost coordinate (16-byte rule) and neither coordinate may be negative.  ADD = true adds
 // the box to global memory (fp32) instead of overwriting it.  Completion is tracked by bulk groups.

@@ -100,6 +100,26 @@ def test_register_mean_kernel_at_any_sequence_length(B, T, d_in, d_out):
     assert pe.pe_last_path() == pe.PATH_TENSOR
 
 
+@pytest.mark.parametrize("B,T,d_in,d_out", [(5, 200, 136, 264), (64, 64, 512, 256), (3, 1000, 520, 776), (1, 257, 8, 8), (16, 512, 1024, 1024)])
+def test_token_stat_fused_staged_and_oracle_agree(B, T, d_in, d_out):
+    """The one-kernel per-token statistic, the two-pass one and the oracle give the same matrix; the two
+    GPU routes round the same tf32 squares, so they differ only by the order of the fp32 sums."""
+    from parity_util import FROB_TOL, oracle_on, rel_frob
+    li = inputs.heavy_tailed_layer(B, T, d_in, d_out, seed=1200 + B, device=DEV, with_weights=False)
+    fused = torch.full((d_out, d_in), float("nan"), device=DEV)
+    pe.pe_token_sqstats(li.X, li.dY, fused)
+    assert pe.pe_last_path() == pe.PATH_TENSOR
+    staged = pe.pe_token_sqstats_staged(li.X, li.dY)
+    torch.cuda.synchronize()
+    assert pe.pe_get_async_status(DEV) == (0, 0)
+    f, s_ = fused.cpu().numpy(), staged.cpu().numpy()
+    assert np.isfinite(f).all()
+    assert rel_frob(f, s_) <= 1e-5
+    if B * T * d_in * d_out <= 3e9:
+        _, tok = oracle_on(li)
+        assert rel_frob(f, tok) <= FROB_TOL
+
+
 def test_heavy_tailed_and_heterogeneous_small():
     check_all(inputs.heavy_tailed_layer(12, 128, 256, 384, seed=41, device=DEV))
     check_all(inputs.heterogeneous_layer(20, 64, 128, 256, seed=42, device=DEV))
@@ -141,9 +161,9 @@ def test_config5_points_sampled_outputs(B, T, d):
     torch.cuda.empty_cache()
 
 
-def test_token_stat_requires_workspace():
+def test_staged_token_stat_requires_workspace():
     li = inputs.gaussian_layer(4, 64, 64, 64, seed=44, device=DEV)
     out = torch.empty((64, 64), device=DEV)
     lib = pe.load_library()
-    st = lib.pe_token_sqstats(li.X.data_ptr(), li.dY.data_ptr(), 4, 64, 64, 64, out.data_ptr(), None, 0, None)
+    st = lib.pe_token_sqstats_staged(li.X.data_ptr(), li.dY.data_ptr(), 4, 64, 64, 64, out.data_ptr(), None, 0, None)
     assert st == 9      # PE_ERR_WORKSPACE

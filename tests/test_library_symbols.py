@@ -64,12 +64,12 @@ def test_host_side_validation_needs_no_gpu(lib):
 def test_workspace_size_formula(lib):
     prev = pe.pe_set_path(pe.PATH_AUTO)
     try:
-        assert pe.pe_token_sqstats_workspace_bytes(64, 256, 512, 2048) == 64 * 256 * (512 + 2048) * 4
-        assert pe.pe_token_sqstats_workspace_bytes(30, 10, 8, 8) == 9728 + 9728      # 9600 B rounded up to 256 B each
-        assert pe.pe_token_sqstats_workspace_bytes(3, 5, 8, 8) == 0                  # too few rows for bf16 squares
-        assert pe.pe_token_sqstats_workspace_bytes(3, 5, 7, 8) == 0                  # SIMT shape: no workspace
+        assert pe.pe_token_sqstats_staged_workspace_bytes(64, 256, 512, 2048) == 64 * 256 * (512 + 2048) * 4
+        assert pe.pe_token_sqstats_staged_workspace_bytes(30, 10, 8, 8) == 9728 + 9728      # 9600 B rounded up to 256 B each
+        assert pe.pe_token_sqstats_staged_workspace_bytes(3, 5, 8, 8) == 0                  # too few rows for bf16 squares
+        assert pe.pe_token_sqstats_staged_workspace_bytes(3, 5, 7, 8) == 0                  # SIMT shape: no workspace
         pe.pe_set_path(pe.PATH_SIMT)
-        assert pe.pe_token_sqstats_workspace_bytes(64, 256, 512, 2048) == 0
+        assert pe.pe_token_sqstats_staged_workspace_bytes(64, 256, 512, 2048) == 0
     finally:
         pe.pe_set_path(prev)
 

@@ -4,7 +4,7 @@ Some users of this library cannot hand it a workspace: they receive input and ou
 host application but no allocator, or their framework claimed the whole GPU at start-up, or they sit
 on a path where cudaMalloc's device-wide synchronisation is not acceptable.  For them the library
 carries a fixed 32 MiB device array and an entry point that stages the squared operands there.  This
-test drives that entry point through the C ABI and requires the same answer as pe_token_sqstats
+test drives that entry point through the C ABI and requires the same answer as pe_token_sqstats_staged
 with a caller-owned workspace, on two consecutive calls that share the array (the second one smaller,
 so anything stale from the first would show), and checks that a shape too large for the array is
 refused on the host.  The file name sorts last so every other test has already run when this one does.
@@ -30,10 +30,10 @@ def _auto_path():
 
 def _both_ways(li):
     B, T, d_in, d_out = li.shape
-    need = pe.pe_token_sqstats_workspace_bytes(B, T, d_in, d_out)
+    need = pe.pe_token_sqstats_staged_workspace_bytes(B, T, d_in, d_out)
     assert 0 < need <= pe.STATIC_SCRATCH_BYTES, "shape must take the staged (tensor-core) path and fit the array"
     want = torch.full((d_out, d_in), float("nan"), device=DEV)
-    pe.pe_token_sqstats(li.X, li.dY, want, torch.empty(need, dtype=torch.uint8, device=DEV))
+    pe.pe_token_sqstats_staged(li.X, li.dY, want, torch.empty(need, dtype=torch.uint8, device=DEV))
     got = torch.full((d_out, d_in), float("nan"), device=DEV)
     lib = pe.load_library()
     stream = torch.cuda.current_stream().cuda_stream
@@ -60,7 +60,7 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row():
 
 def test_static_scratch_refuses_shapes_beyond_its_size():
     B, T, d_in, d_out = 64, 256, 512, 2048                                       # needs 168 MB of staging
-    assert pe.pe_token_sqstats_workspace_bytes(B, T, d_in, d_out) > pe.STATIC_SCRATCH_BYTES
+    assert pe.pe_token_sqstats_staged_workspace_bytes(B, T, d_in, d_out) > pe.STATIC_SCRATCH_BYTES
     X = torch.zeros((B, T, d_in), dtype=torch.bfloat16, device=DEV)
     dY = torch.zeros((B, T, d_out), dtype=torch.bfloat16, device=DEV)
     out = torch.full((d_out, d_in), 7.0, device=DEV)
