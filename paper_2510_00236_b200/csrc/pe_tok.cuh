@@ -45,11 +45,13 @@ struct TokParams {
   unsigned int* dev_status;
 };
 
-// x -> x*x rounded to tf32 (10 explicit mantissa bits), as an fp32 bit pattern.  The square of a bf16
-// value is exact in fp32; it is positive, so adding half a tf32 ulp and clearing the 13 low bits
-// rounds to nearest (ties away from zero).
+// x -> x*x rounded to tf32 (10 explicit mantissa bits, round to nearest even), as an fp32 bit
+// pattern.  The square of a bf16 value is exact in fp32, so this rounding is the only error: at most
+// 2^-11 relative per operand, and unbiased.  (Squares of 8-bit significands hit exact ties often, so
+// rounding ties upward would bias the sums by about 1e-4.)
 __device__ __forceinline__ uint32_t tok_square_tf32(float v) {
-  return (__float_as_uint(v * v) + 0x1000u) & 0xFFFFE000u;
+  const uint32_t u = __float_as_uint(v * v);
+  return (u + 0xFFFu + ((u >> 13) & 1u)) & 0xFFFFE000u;
 }
 
 // gridDim = (2 * pairs_m * tiles_n, 1, nsplit); blockIdx.x = 2 * (pair index in the tile order) + rank in pair.
