@@ -45,13 +45,22 @@ struct TokParams {
   unsigned int* dev_status;
 };
 
-// x -> x*x rounded to tf32 (10 explicit mantissa bits, round to nearest even), as an fp32 bit
-// pattern.  The square of a bf16 value is exact in fp32, so this rounding is the only error: at most
-// 2^-11 relative per operand, and unbiased.  (Squares of 8-bit significands hit exact ties often, so
-// rounding ties upward would bias the sums by about 1e-4.)
-__device__ __forceinline__ uint32_t tok_square_tf32(float v) {
-  const uint32_t u = __float_as_uint(v * v);
-  return (u + 0xFFFu + ((u >> 13) & 1u)) & 0xFFFFE000u;
+// Two bf16 values (one 32-bit word) -> their squares rounded to tf32 (10 explicit mantissa bits,
+// round to nearest even), as two fp32 bit patterns in one 64-bit register.  A bf16 is the upper half
+// of an fp32 and its square is exact in fp32, so the rounding is the only error: at most 2^-11
+// relative per operand, and unbiased.  The rounding is Veltkamp's split: with s = RN(8193 x),
+// s - (s - x) is x rounded to 24 - 13 = 11 significant bits (nearest even; it equals the integer
+// formula (u + 0xFFF + ((u >> 13) & 1)) & ~0x1FFF on every square of an 8-bit significand, where exact
+// ties are frequent and rounding them upward would bias the sums by about 1e-4).  Four packed fp32
+// instructions per pair.  s is formed as fma(x, 8192, x): the assembler was seen to merge a separate
+// multiply by 8193 into the following subtraction, which skips the rounding of s that the split
+// relies on; a multiply by a power of two is exact, so this form gives the same s however it is merged.
+// Squares above 2^128 / 8193 come out as NaN instead of infinity.
+__device__ __forceinline__ uint64_t tok_square_tf32_pair(uint32_t two_bf16) {
+  const uint64_t v = sm100::f32x2_pack(__uint_as_float(two_bf16 << 16), __uint_as_float(two_bf16 & 0xFFFF0000u));
+  const uint64_t x = sm100::f32x2_mul(v, v);
+  const uint64_t s = sm100::f32x2_fma(x, sm100::f32x2_pack(8192.f, 8192.f), x);
+  return sm100::f32x2_sub(s, sm100::f32x2_sub(s, x));
 }
 
 // gridDim = (2 * pairs_m * tiles_n, 1, nsplit); blockIdx.x = 2 * (pair index in the tile order) + rank in pair.
@@ -169,16 +178,11 @@ tok_sqstats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
           const int g = (i * 8 + w) * 32 + lane;
           const int box = g >> 8, t = (g >> 3) & 31, c = g & 7;
           const uint4 v = *reinterpret_cast<const uint4*>(raw + box * TOK_BOX_BYTES + t * 128 + ((c ^ (t & 7)) << 4));
-          const uint32_t u[4] = {v.x, v.y, v.z, v.w};
-          uint32_t o[8];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {     // a bf16 is the upper half of an fp32
-            o[2 * j] = tok_square_tf32(__uint_as_float(u[j] << 16));
-            o[2 * j + 1] = tok_square_tf32(__uint_as_float(u[j] & 0xFFFF0000u));
-          }
+          const uint64_t o0 = tok_square_tf32_pair(v.x), o1 = tok_square_tf32_pair(v.y);
+          const uint64_t o2 = tok_square_tf32_pair(v.z), o3 = tok_square_tf32_pair(v.w);
           uint8_t* dst = cooked + (2 * box + (c >> 2)) * TOK_BOX_BYTES + t * 128 + (((c & 3) ^ (t & 3)) << 5);
-          *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
-          *reinterpret_cast<uint4*>(dst + 16) = make_uint4(o[4], o[5], o[6], o[7]);
+          *reinterpret_cast<ulonglong2*>(dst) = make_ulonglong2(o0, o1);
+          *reinterpret_cast<ulonglong2*>(dst + 16) = make_ulonglong2(o2, o3);
         }
         fence_async_smem();                 // the MMA reads these through the async proxy
         __syncwarp();
