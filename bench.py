@@ -116,6 +116,20 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def max_over_ranks(torch, dist, ms: float, device) -> float:
+    """Slowest rank's time (every rank gets the same answer); identity without a process group."""
+    if dist is None:
+        return float(ms)
+    tt = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def replica_throughput(world: int, flops_per_step: float, ms_per_step: float) -> float:
+    """Whole-job TFLOP/s of `world` independent replicas that all take the slowest rank's step time."""
+    return world * flops_per_step / (ms_per_step * 1e-3) / 1e12
+
+
 def make_state(pe, inputs, torch, name, dev, seed_offset=0):
     B, T, d_in, d_out, nsets = WORKLOADS[name]
     sets = []
@@ -380,12 +394,9 @@ def main():
     ms_total = t_start.elapsed_time(t_end)
     clocks = sampler.stop() if rank == 0 else None
     kernel_ms = statistics.fmean(a.elapsed_time(b) for a, b in kernel_events)
-    if dist is not None:
-        tt = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
+    ms_total = max_over_ranks(torch, dist, ms_total, dev)
     ms_step = ms_total / args.steps
-    value = world * flops_step / (ms_step * 1e-3) / 1e12
+    value = replica_throughput(world, flops_step, ms_step)
 
     # ------------------------------------------------------------ end to end: host buffers in, statistics out
     e2e_steps = max(3, min(20, args.steps // 5))
@@ -413,11 +424,8 @@ def main():
     eb.record()
     barrier()
     e2e_ms = ea.elapsed_time(eb)
-    if dist is not None:
-        tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt.item())
-    e2e_value = world * flops_step / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    e2e_ms = max_over_ranks(torch, dist, e2e_ms, dev)
+    e2e_value = replica_throughput(world, flops_step, e2e_ms / e2e_steps)
     h2d = hX.numel() * hX.element_size() + hdY.numel() * hdY.element_size()
     d2h = sum(o.numel() * o.element_size() for o in outs)
 
