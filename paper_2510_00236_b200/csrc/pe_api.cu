@@ -158,6 +158,31 @@ static pe_status_t zero_outputs(float* a, float* b, size_t bytes, cudaStream_t s
   return PE_OK;
 }
 
+// Zeroes one or two [d_out, d_in] outputs with a kernel that lets its successor start at once.
+static pe_status_t zero_for_split(DeviceInfo* di, float* a, float* b, size_t n, cudaStream_t st) {
+  float* first = a ? a : b;
+  float* second = a ? b : nullptr;
+  if (!first) return PE_OK;
+  const long long n4 = (long long)(n / 4);          // d_in % 8 == 0 on this path
+  long long blocks = (n4 + 255) / 256;
+  if (blocks > di->sm_count) blocks = di->sm_count;   // few blocks: the dependent kernel needs the SMs
+  zero_outputs_kernel<<<(int)(blocks < 1 ? 1 : blocks), 256, 0, st>>>(reinterpret_cast<float4*>(first), reinterpret_cast<float4*>(second), n4);
+  return check_launch();
+}
+
+// Launches `kernel`; as a programmatic dependent of the zeroing kernel when the batch is split.
+template <typename Kernel, typename... Args>
+static pe_status_t launch_pair_kernel(Kernel kernel, dim3 grid, int smem, cudaStream_t st, bool after_zeroing, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr; cfg.numAttrs = after_zeroing ? 1 : 0;
+  if (cudaLaunchKernelEx(&cfg, kernel, args...) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
+  return check_launch();
+}
+
 template <int PHI, bool TF32, int NT, int MEAN>
 static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& mm,
                                   const CUtensorMap& ms, const TcParams& p, dim3 grid, cudaStream_t st) {
@@ -169,8 +194,7 @@ static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& m
     }
     di->tc_attr_set[slot] = true;
   }
-  tc_stats_kernel<PHI, TF32, NT, MEAN><<<grid, TC_THREADS, smem, st>>>(mx, my, mm, ms, p);
-  return check_launch();
+  return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN>, grid, smem, st, p.nsplit > 1, mx, my, mm, ms, p);
 }
 
 // Tensor-core launch.  per_example = 0 runs the plain contraction over all B*T rows (its result goes
@@ -199,7 +223,7 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   if ((long long)tiles_n * pairs_m > (1ll << 29)) return PE_ERR_DIM;
   const int ns = choose_nsplit((long long)tiles_n * pairs_m, B, T, di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 16);
   if (ns > 1) {
-    rc = zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
+    rc = zero_for_split(di, out_mean, out_stat, (size_t)d_in * d_out, st);
     if (rc != PE_OK) return rc;
   }
   TcParams p;
@@ -316,7 +340,7 @@ static pe_status_t launch_tok(DeviceInfo* di, const void* X, const void* dY, lon
   const int units = n_chunks > (1 << 30) ? (1 << 30) : (int)n_chunks;
   const int ns = choose_nsplit((long long)tiles_n * pairs_m, units, TOK_BK, di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 32);
   if (ns > 1) {
-    rc = zero_outputs(out, nullptr, (size_t)d_in * d_out * sizeof(float), st);
+    rc = zero_for_split(di, out, nullptr, (size_t)d_in * d_out, st);
     if (rc != PE_OK) return rc;
   }
   if (!di->tok_attr_set) {
@@ -329,8 +353,7 @@ static pe_status_t launch_tok(DeviceInfo* di, const void* X, const void* dY, lon
   TokParams p;
   p.rows = rows; p.d_in = d_in; p.d_out = d_out; p.pairs_m = pairs_m; p.tiles_n = tiles_n;
   p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND; p.nsplit = ns; p.dev_status = di->status_ptr;
-  tok_sqstats_kernel<<<dim3(2 * pairs_m * tiles_n, 1, ns), TC_THREADS, TOK_SMEM_BYTES, st>>>(mx, my, mo, p);
-  return check_launch();
+  return launch_pair_kernel(tok_sqstats_kernel, dim3(2 * pairs_m * tiles_n, 1, ns), TOK_SMEM_BYTES, st, ns > 1, mx, my, mo, p);
 }
 
 }  // namespace pe

@@ -136,6 +136,20 @@ struct StageWalk {
   }
 };
 
+// Zeroes the outputs of a split-batch launch.  The statistics kernel that follows is launched as a
+// programmatic dependent: it starts right away (it only touches the outputs in its very last step,
+// behind griddepcontrol.wait), so the zeroing costs no time on the stream.  a, b: n4 float4 each; b may
+// be NULL.
+__global__ void __launch_bounds__(256) zero_outputs_kernel(float4* __restrict__ a, float4* __restrict__ b, long long n4) {
+  sm100::griddep_launch_dependents();
+  const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x; k < n4; k += stride) {
+    a[k] = z;
+    if (b) b[k] = z;
+  }
+}
+
 enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2 };   // where sum_b G_b is kept in per-example mode
 
 // gridDim = (2 * pairs_m * tiles_n, 1, nsplit); blockIdx.x = 2 * (pair index in the tile order) + rank in pair.
@@ -365,6 +379,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         fence_async_smem();
         __syncwarp();
         if (lane == 0 && row0 < p.d_out) {
+          if (p.nsplit > 1) griddep_wait();       // the kernel that zeroes the outputs may still be running
           for (int c = 0; c < PANELS; ++c) {
             if (col0 + c * 32 < p.d_in) {
               if (p.nsplit == 1) tma_store_2d<false>(tm, first_panel + c * 4096, col0 + c * 32, row0);

@@ -224,6 +224,7 @@ tok_sqstats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
       fence_async_smem();
       __syncwarp();
       if (lane == 0 && row0 < p.d_out) {
+        if (p.nsplit > 1) griddep_wait();         // the kernel that zeroes the output may still be running
         for (int c = 0; c < 4; ++c) {
           if (col0 + c * 32 < p.d_in) {
             if (p.nsplit == 1) tma_store_2d<false>(&tmap_out, stage_base + c * 4096, col0 + c * 32, row0);
