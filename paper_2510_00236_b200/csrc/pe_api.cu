@@ -31,7 +31,7 @@ struct DeviceInfo {
   std::atomic<int> state{0};     // 0 unknown, 1 ready, -1 failed
   int cc_major = 0, sm_count = 0;
   unsigned int* status_ptr = nullptr;
-  bool tc_attr_set[8] = {false, false, false, false, false, false, false, false};
+  bool tc_attr_set[10] = {};
   bool tok_attr_set = false;
 };
 static DeviceInfo g_dev[MAX_DEVICES];
@@ -183,18 +183,18 @@ static pe_status_t launch_pair_kernel(Kernel kernel, dim3 grid, int smem, cudaSt
   return check_launch();
 }
 
-template <int PHI, bool TF32, int NT, int MEAN>
+template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT)>
 static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& mm,
                                   const CUtensorMap& ms, const TcParams& p, dim3 grid, cudaStream_t st) {
-  constexpr int smem = TcOperand<TF32, NT>::SMEM_BYTES;
+  constexpr int smem = TcOperand<TF32, NT, BKT>::SMEM_BYTES;
   if (!di->tc_attr_set[slot]) {
-    if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+    if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
       cudaGetLastError();
       return PE_ERR_CUDA;
     }
     di->tc_attr_set[slot] = true;
   }
-  return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN>, grid, smem, st, p.nsplit > 1, mx, my, mm, ms, p);
+  return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT>, grid, smem, st, p.nsplit > 1, mx, my, mm, ms, p);
 }
 
 // Tensor-core launch.  per_example = 0 runs the plain contraction over all B*T rows (its result goes
@@ -208,7 +208,8 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   const bool mean_regs = both && (T < TC_MEAN_TMEM_MIN_T || g_path.load() == PE_PATH_TENSOR_NARROW);
   const int nt = mean_regs ? 128 : 256;
   const int box_feats = tf32 ? TcOperand<true, 256>::BOX_FEATS : TcOperand<false, 256>::BOX_FEATS;
-  const int box_tokens = tf32 ? TcOperand<true, 256>::BK : (mean_regs ? TcOperand<false, 128>::BK : TcOperand<false, 256>::BK);
+  const bool short_seq = mean_regs && T <= TC_SHORT_T;      // many short examples, both outputs: small stages
+  const int box_tokens = short_seq ? TC_SHORT_BK : tc_default_bk(tf32, nt);
   CUtensorMap mx, my;
   pe_status_t rc = make_operand_map(&mx, X, B, T, d_in, tf32, box_feats, box_tokens);
   if (rc != PE_OK) return rc;
@@ -233,6 +234,10 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   dim3 grid(2 * pairs_m * tiles_n, 1, ns);
   if (tf32) return launch_tc_inst<0, true, 256, MEAN_NONE>(di, 5, mx, my, mm, ms, p, grid, st);
   if (!per_example) return launch_tc_inst<0, false, 256, MEAN_NONE>(di, 4, mx, my, mm, ms, p, grid, st);
+  if (short_seq) {
+    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, MEAN_REGS, TC_SHORT_BK>(di, 8, mx, my, mm, ms, p, grid, st);
+    return launch_tc_inst<2, false, 128, MEAN_REGS, TC_SHORT_BK>(di, 9, mx, my, mm, ms, p, grid, st);
+  }
   if (mean_regs) {
     if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, MEAN_REGS>(di, 0, mx, my, mm, ms, p, grid, st);
     return launch_tc_inst<2, false, 128, MEAN_REGS>(di, 1, mx, my, mm, ms, p, grid, st);

@@ -54,14 +54,20 @@ constexpr int TC_SMEM_BUDGET = 200 * 1024;   // operand ring; leaves room for ba
 // Operand element type of the MMA.  bf16 (kind::f16, 16 tokens per instruction) for the per-example
 // statistics; tf32 (kind::tf32, fp32 storage, 8 tokens per instruction) for the per-token statistic,
 // whose squared operands need more than bf16's 8 significant bits.  NT = d_in columns per pair tile.
-template <bool TF32, int NT>
+// Default tokens per pipeline stage: 128 for the 256 x 128 tile, 64 for the 256 x 256 tile, 32 for
+// tf32.  With both outputs and short sequences (T <= 64) the 256 x 128 tile takes 32-token stages
+// instead: a 128-token box would be mostly zero fill, and 16 small slots keep more examples in flight.
+__host__ __device__ constexpr int tc_default_bk(bool tf32, int nt) { return tf32 ? 32 : (nt == 128 ? 128 : 64); }
+constexpr int TC_SHORT_BK = 32;
+constexpr int TC_SHORT_T = 64;
+template <bool TF32, int NT, int BK_ = tc_default_bk(TF32, NT)>
 struct TcOperand {
   static constexpr int ELEM_BYTES = TF32 ? 4 : 2;
   static constexpr int BOX_FEATS = 128 / ELEM_BYTES;            // features per 128-byte swizzle row: 64 | 32
   // tokens per pipeline stage (one TMA box is BK tokens tall), chosen so that the ring has an EVEN
   // number of stages: with two MMA issuers taking alternate stages every slot then always belongs
   // to the same issuer (see the parity note at the issuer's wait).
-  static constexpr int BK = TF32 ? 32 : (NT == 128 ? 128 : 64);
+  static constexpr int BK = BK_;
   static constexpr int MMA_K = 32 / ELEM_BYTES;                 // tokens per MMA instruction: 16 | 8
   static constexpr int BOX_BYTES = 128 * BK;                    // one box: BK tokens x 128 bytes
   static constexpr int A_BOXES = TC_TILE_M / BOX_FEATS;         // this block's 128 rows of dY^T
@@ -70,7 +76,7 @@ struct TcOperand {
   static constexpr int A_BYTES = A_BOXES * BOX_BYTES;           // 32 KiB (NT = 128) | 16 KiB
   static constexpr int B_BYTES = B_BOXES * BOX_BYTES;           // 16 KiB
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;         // per block: 48 KiB | 32 KiB
-  static constexpr int STAGES = TC_SMEM_BUDGET / STAGE_BYTES;   // 4 | 6
+  static constexpr int STAGES = (TC_SMEM_BUDGET / STAGE_BYTES) & ~1;   // 4 | 6 | 16 with 32-token stages
   static_assert(STAGES % 2 == 0, "slots must alternate between the two issuers");
   static constexpr int K_STEP_BYTES = MMA_K * 128;              // smem advance per MMA: 2048 | 1024
   static constexpr int ACC_BUFS = TC_TMEM_COLS / NT;            // 4 | 2 accumulators in tensor memory
@@ -153,12 +159,12 @@ __global__ void __launch_bounds__(256) zero_outputs_kernel(float4* __restrict__ 
 enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2 };   // where sum_b G_b is kept in per-example mode
 
 // gridDim = (2 * pairs_m * tiles_n, 1, nsplit); blockIdx.x = 2 * (pair index in the tile order) + rank in pair.
-template <int PHI, bool TF32, int NT, int MEAN>
+template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT)>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
                 const __grid_constant__ CUtensorMap tmap_mean, const __grid_constant__ CUtensorMap tmap_stat, TcParams p) {
   using namespace sm100;
-  using Op = TcOperand<TF32, NT>;
+  using Op = TcOperand<TF32, NT, BKT>;
   static_assert(MEAN != MEAN_REGS || NT == 128, "two running sums only fit the registers at NT = 128");
   static_assert(MEAN != MEAN_TMEM || (NT == 256 && PHI != 0), "the tensor-memory mean sits beside one 256-column accumulator");
   constexpr int STAGES = Op::STAGES, BK = Op::BK;
