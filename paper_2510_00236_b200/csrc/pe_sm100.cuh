@@ -121,8 +121,9 @@ __device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bu
 // Orders this thread's ordinary shared-memory writes before later accesses by TMA / the tensor core.
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// Same load issued by one block of a CTA pair: the data lands in the issuing block's shared memory,
-// the byte count is credited to `cluster_bar`, a cluster-window address that may lie in the peer.
+// 3-D tiled load (c0 innermost; c0 * element size must be a multiple of 16 bytes) issued by one block
+// of a CTA pair: the data lands in the issuing block's shared memory, the byte count is credited to
+// `cluster_bar`, a cluster-window address that may lie in the peer.
 __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* m, uint32_t cluster_bar, int c0, int c1, int c2) {
   asm volatile(
       "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"

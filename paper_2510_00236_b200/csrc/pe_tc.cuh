@@ -342,36 +342,36 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
           tmem_st_32x32b_x16(maddr + c * 16, r);
         }
         tmem_st_wait();
-        continue;
-      }
+      } else {
 #pragma unroll
-      for (int c = 0; c < COLS / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld_32x32b_x32_wait(taddr + c * 32, r);
-        if (c == COLS / 32 - 1) {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));   // buffer free for the issuer's next example
-        }
-        if constexpr (PHI == 2) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float g = __uint_as_float(r[j]);
-            if (KEEP_MEAN) acc_mean[c * 32 + j] += g;
-            acc_stat[c * 32 + j] += phi_apply<PHI>(g);
+        for (int c = 0; c < COLS / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld_32x32b_x32_wait(taddr + c * 32, r);
+          if (c == COLS / 32 - 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));   // buffer free for the issuer's next example
           }
-        } else {
-          // two columns per instruction: packed fp32 add for sum_b G_b, packed fma for sum_b G_b^2
+          if constexpr (PHI == 2) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const uint64_t g2 = f32x2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-            if (KEEP_MEAN) {
-              const uint64_t m2 = f32x2_add(f32x2_pack(acc_mean[c * 32 + j], acc_mean[c * 32 + j + 1]), g2);
-              f32x2_unpack(m2, acc_mean[c * 32 + j], acc_mean[c * 32 + j + 1]);
+            for (int j = 0; j < 32; ++j) {
+              const float g = __uint_as_float(r[j]);
+              if (KEEP_MEAN) acc_mean[c * 32 + j] += g;
+              acc_stat[c * 32 + j] += phi_apply<PHI>(g);
             }
-            if (PHI == 1) {
-              const uint64_t s2 = f32x2_fma(g2, g2, f32x2_pack(acc_stat[c * 32 + j], acc_stat[c * 32 + j + 1]));
-              f32x2_unpack(s2, acc_stat[c * 32 + j], acc_stat[c * 32 + j + 1]);
+          } else {
+            // two columns per instruction: packed fp32 add for sum_b G_b, packed fma for sum_b G_b^2
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+              const uint64_t g2 = f32x2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+              if (KEEP_MEAN) {
+                const uint64_t m2 = f32x2_add(f32x2_pack(acc_mean[c * 32 + j], acc_mean[c * 32 + j + 1]), g2);
+                f32x2_unpack(m2, acc_mean[c * 32 + j], acc_mean[c * 32 + j + 1]);
+              }
+              if (PHI == 1) {
+                const uint64_t s2 = f32x2_fma(g2, g2, f32x2_pack(acc_stat[c * 32 + j], acc_stat[c * 32 + j + 1]));
+                f32x2_unpack(s2, acc_stat[c * 32 + j], acc_stat[c * 32 + j + 1]);
+              }
             }
           }
         }
