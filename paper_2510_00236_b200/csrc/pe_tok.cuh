@@ -189,9 +189,12 @@ tok_sqstats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
           const uint4 v = *reinterpret_cast<const uint4*>(raw + box * TOK_BOX_BYTES + t * 128 + ((c ^ (t & 7)) << 4));
           const uint64_t o0 = tok_square_tf32_pair(v.x), o1 = tok_square_tf32_pair(v.y);
           const uint64_t o2 = tok_square_tf32_pair(v.z), o3 = tok_square_tf32_pair(v.w);
+          // Lanes with c >= 4 (the second of the two boxes) store their halves in the other order, so
+          // that each store instruction of the warp touches all eight 16-byte bank groups, not four.
           uint8_t* dst = cooked + (2 * box + (c >> 2)) * TOK_BOX_BYTES + t * 128 + (((c & 3) ^ (t & 3)) << 5);
-          *reinterpret_cast<ulonglong2*>(dst) = make_ulonglong2(o0, o1);
-          *reinterpret_cast<ulonglong2*>(dst + 16) = make_ulonglong2(o2, o3);
+          const bool swap = (c & 4) != 0;
+          *reinterpret_cast<ulonglong2*>(dst + (swap ? 16 : 0)) = swap ? make_ulonglong2(o2, o3) : make_ulonglong2(o0, o1);
+          *reinterpret_cast<ulonglong2*>(dst + (swap ? 0 : 16)) = swap ? make_ulonglong2(o0, o1) : make_ulonglong2(o2, o3);
         }
         fence_async_smem();                 // the MMA reads these through the async proxy
         __syncwarp();
