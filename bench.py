@@ -40,6 +40,7 @@ WORKLOADS = {
     "c4": (256, 1024, 2048, 8192, 1),
     "c4s": (16, 1024, 2048, 8192, 1),     # a 16-sequence slice of c4 (335 MB of inputs): small enough to profile
 }
+TOKEN_STAGED_MIN_ELEMS = 100_000_000
 ADAM = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8)
 SIGN = dict(lr=3.47e-3, beta=0.9)
 
@@ -53,13 +54,15 @@ def measured_peaks():
     return {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0, "source": "fallback"}
 
 
-def profile_traffic(workload: str):
-    """DRAM bytes per launch of the statistics kernel from the committed ncu summary, if present."""
+def profile_traffic(workload: str, kernel: str):
+    """DRAM bytes per launch of one kernel from the committed ncu summary of this workload, if present
+    (a line "dram_bytes_per_launch <kernel>: <bytes>")."""
     path = os.path.join(ROOT, "profiles", f"tc_stats_kernel_{workload}.txt")
+    key = f"dram_bytes_per_launch {kernel}:"
     try:
         for line in open(path):
-            if line.startswith("dram_bytes_per_launch:"):
-                return float(line.split(":")[1].split()[0])
+            if line.startswith(key):
+                return float(line[len(key):].split()[0])
     except OSError:
         pass
     return None
@@ -153,7 +156,21 @@ def make_state(pe, inputs, torch, name, dev, seed_offset=0):
         "theta2_lp": torch.empty((d_out, d_in), dtype=torch.bfloat16, device=dev),
         "n": n,
     }
+    # Per-token statistic: the one-kernel tf32 form on small layers; from about 1e8 input elements on, the
+    # two-pass form (half operands at the full 16-bit tensor rate) with a caller-owned workspace.
+    st["tok_ws"] = None
+    if B * T * (d_in + d_out) >= TOKEN_STAGED_MIN_ELEMS:
+        need = pe.pe_token_sqstats_staged_workspace_bytes(B, T, d_in, d_out)
+        if need > 0:
+            st["tok_ws"] = torch.empty(need, dtype=torch.uint8, device=dev)
     return st
+
+
+def token_stat(pe, st, X, dY):
+    if st["tok_ws"] is not None:
+        pe.pe_token_sqstats_staged(X, dY, st["tok"], st["tok_ws"])
+    else:
+        pe.pe_token_sqstats(X, dY, st["tok"])
 
 
 def run_step(pe, st, i, X=None, dY=None, ev=None):
@@ -167,7 +184,11 @@ def run_step(pe, st, i, X=None, dY=None, ev=None):
     if ev is not None:
         ev[1].record()
     pe.pe_linear_stats(X, dY, pe.PHI_SIGN, None, st["sgn"])
-    pe.pe_token_sqstats(X, dY, st["tok"])
+    if ev is not None:
+        ev[2].record()
+    token_stat(pe, st, X, dY)
+    if ev is not None:
+        ev[3].record()
     pe.microadam_step(st["theta"], st["m"], st["v"], st["mean"], st["sq"], B, step=i + 1, theta_lp=st["theta_lp"], **ADAM)
     pe.microsignsgd_step(st["theta2"], st["m2"], st["sgn"], B, theta_lp=st["theta2_lp"], **SIGN)
 
@@ -208,6 +229,13 @@ def context_numbers(torch, pe, st, li, peaks, dev):
     extra["pe_linear_stats_sign_us"] = {"median": med_s * 1e3, "best": best_s * 1e3, "tflops_median": flops_one / med_s / 1e9}
     med_t, best_t = time_each(torch, lambda i: pe.pe_token_sqstats(li.X, li.dY, st["tok"]))
     extra["pe_token_sqstats_us"] = {"median": med_t * 1e3, "best": best_t * 1e3, "tflops_median": flops_one / med_t / 1e9}
+    need = pe.pe_token_sqstats_staged_workspace_bytes(B, T, d_in, d_out)
+    if need > 0:
+        ws = st["tok_ws"] if st["tok_ws"] is not None else torch.empty(need, dtype=torch.uint8, device=dev)
+        med_t2, best_t2 = time_each(torch, lambda i: pe.pe_token_sqstats_staged(li.X, li.dY, st["tok"], ws))
+        extra["pe_token_sqstats_staged_us"] = {"median": med_t2 * 1e3, "best": best_t2 * 1e3, "tflops_median": flops_one / med_t2 / 1e9,
+                                               "workspace_bytes": need}
+        del ws
     A2, B2 = li.dY.view(B * T, d_out), li.X.view(B * T, d_in)
     med_g, best_g = time_each(torch, lambda i: torch.matmul(A2.t(), B2))
     extra["cublas_wgrad_gemm_us"] = {"median": med_g * 1e3, "best": best_g * 1e3, "tflops_median": flops_one / med_g / 1e9,
@@ -383,7 +411,7 @@ def main():
         time.sleep(0.25)
     barrier()
     pe.pe_reset_launch_count()
-    kernel_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    kernel_events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_start.record()
     for i in range(args.steps):
@@ -393,7 +421,8 @@ def main():
     launches = pe.pe_launch_count()
     ms_total = t_start.elapsed_time(t_end)
     clocks = sampler.stop() if rank == 0 else None
-    kernel_ms = statistics.fmean(a.elapsed_time(b) for a, b in kernel_events)
+    # average duration of each statistics call inside the timed steps (events on the launching stream)
+    call_ms = [statistics.fmean(ev[k].elapsed_time(ev[k + 1]) for ev in kernel_events) for k in range(3)]
     ms_total = max_over_ranks(torch, dist, ms_total, dev)
     ms_step = ms_total / args.steps
     value = replica_throughput(world, flops_step, ms_step)
@@ -439,12 +468,26 @@ def main():
     li = st["sets"][0]
     extra = {} if args.quick else context_numbers(torch, pe, st, li, peaks, dev)
 
-    achieved = flops_one / (kernel_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "tc_stats_kernel<square>", "achieved": achieved, "peak": peaks["bf16_tflops"],
-                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst)",
-                "traffic": profile_traffic(name), "avg_launch_ms": kernel_ms,
-                "algorithmic_flops_per_launch": flops_one,
-                "algorithmic_bytes_per_launch": 2.0 * B * T * (d_in + d_out) + 8.0 * d_in * d_out}
+    # One roofline entry per statistics kernel; the headline one is the kernel with the largest share
+    # of the timed step.  The per-token kernel contracts tf32 operands: its peak is the measured bf16
+    # peak times the nominal tf32 : bf16 ratio (1/2).
+    alg_bytes = 2.0 * B * T * (d_in + d_out)
+    specs = [("tc_stats_kernel<square, both outputs>", "square", peaks["bf16_tflops"], "bf16", alg_bytes + 8.0 * d_in * d_out),
+             ("tc_stats_kernel<sign, statistic only>", "sign", peaks["bf16_tflops"], "bf16", alg_bytes + 4.0 * d_in * d_out),
+             ("tok_sqstats_kernel", "token", 0.5 * peaks["bf16_tflops"], "tf32", alg_bytes + 4.0 * d_in * d_out)]
+    if st["tok_ws"] is not None:      # two-pass form: three streaming kernels around the half contraction
+        specs[2] = ("pe_token_sqstats_staged: column_max + square_to_half + tc_stats_kernel<identity, half> + unscale", "token_staged",
+                    peaks["bf16_tflops"], "f16", alg_bytes + 4.0 * d_in * d_out)
+    by_kernel = []
+    for (kname, key, peak, op_dtype, nbytes), ms in zip(specs, call_ms):
+        ach = flops_one / (ms * 1e-3) / 1e12
+        by_kernel.append({"bound": "tensor", "kernel": kname, "operand_dtype": op_dtype, "achieved": ach, "peak": peak,
+                          "unit": "TFLOP/s", "frac": ach / peak,
+                          "peak_source": peaks["source"] + (" bf16 (burst) x 0.5 nominal tf32 ratio" if op_dtype == "tf32" else " (burst)"),
+                          "traffic": profile_traffic(name, key), "avg_launch_ms": ms, "share_of_step": ms / ms_step,
+                          "algorithmic_flops_per_launch": flops_one, "algorithmic_bytes_per_launch": nbytes})
+    roofline = dict(max(by_kernel, key=lambda r: r["share_of_step"]))
+    roofline["by_kernel"] = by_kernel
 
     cpu_baseline = None
     if not args.no_cpu_baseline and not args.quick and world == 1:
@@ -464,7 +507,8 @@ def main():
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": name, "B": B, "T": T, "d_in": d_in, "d_out": d_out,
-                   "step": "pe_linear_stats(square)+pe_linear_stats(sign)+pe_token_sqstats+microadam_step+microsignsgd_step",
+                   "step": "pe_linear_stats(square)+pe_linear_stats(sign)+" + ("pe_token_sqstats_staged" if st["tok_ws"] is not None else "pe_token_sqstats")
+                           + "+microadam_step+microsignsgd_step",
                    "flops_per_step": flops_step, "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": f"{nsets} rotating input sets, {nsets * 2 * B * T * (d_in + d_out) / 1e6:.0f} MB in all (> 126 MB L2)"
                          if nsets > 1 else "inputs larger than L2"},

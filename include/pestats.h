@@ -90,12 +90,18 @@ pe_status_t pe_token_sqstats_f32(const float* X, const float* dY, int B, int T, 
                                  float* out_stat, pe_stream_t stream);
 
 /*
- * The same statistic in two passes (Section 2.3): a streaming kernel writes the tf32-rounded squares
- * as fp32 into `workspace` (device memory, 256-byte aligned, at least
- * pe_token_sqstats_staged_workspace_bytes() bytes, contents undefined afterwards), then the plain
- * tensor-core contraction reads them back.  Slower than pe_token_sqstats (it moves three times the
- * bytes); kept as an independent second route to the same numbers and as the kernel behind
- * pe_token_sqstats_static.  The SIMT path ignores the workspace (it may then be NULL).
+ * The same statistic in two passes (Section 2.3), for callers that can lend a workspace as large as
+ * the inputs.  Streaming kernels find the largest magnitude of every column of X and of dY and write
+ * the squares, each multiplied by a power of two chosen from its column's maximum so that it fits
+ * IEEE half, into `workspace` (device memory, 256-byte aligned, at least
+ * pe_token_sqstats_staged_workspace_bytes() bytes, contents undefined afterwards); the plain
+ * tensor-core contraction then runs on the half operands at the full 16-bit rate (the one-kernel
+ * pe_token_sqstats contracts tf32 at half that rate), and a last kernel undoes the scales.  Half keeps
+ * the same 11 significant bits as tf32, rounded to nearest even; within a column, entries more than
+ * 2^14 below the column's largest magnitude lose bits gradually and vanish 2^20 below it.  Faster
+ * than pe_token_sqstats once B*T*(d_in + d_out) reaches about 10^8 elements, slower below (six
+ * launches instead of one).  Also the kernel sequence behind pe_token_sqstats_static.  The SIMT path
+ * ignores the workspace (it may then be NULL).
  */
 pe_status_t pe_token_sqstats_staged(const void* X, const void* dY, int B, int T, int d_in, int d_out,
                                     float* out_stat, void* workspace, size_t workspace_bytes,
@@ -111,7 +117,7 @@ size_t pe_token_sqstats_staged_workspace_bytes(int B, int T, int d_in, int d_out
  * reserved all of the GPU's memory in its own pool at start-up, so that cudaMalloc would fail; a
  * latency-critical loop that must not pay cudaMalloc / cudaFree's device-wide synchronisation.
  *
- * Same arguments, result and path selection as pe_token_sqstats_staged, minus the workspace: the fp32
+ * Same arguments, result and path selection as pe_token_sqstats_staged, minus the workspace: the
  * staging of the squared operands lives in an array of PE_STATIC_SCRATCH_BYTES bytes that is part
  * of the library's device image, so every GPU on which the library is used holds that much memory
  * from module load until the process exits.  The call allocates and frees nothing, on the device or

@@ -174,8 +174,9 @@ def pe_token_sqstats_staged_workspace_bytes(B, T, d_in, d_out) -> int:
 
 
 def pe_token_sqstats_staged(X, dY, out_stat=None, workspace=None):
-    """The same statistic in two passes through a workspace of fp32 squares.  ``workspace`` is a uint8
-    CUDA tensor of at least pe_token_sqstats_staged_workspace_bytes(...) bytes; allocated when omitted."""
+    """The same statistic in two passes through a workspace holding the squares as column-scaled IEEE
+    half (as large as the inputs); the faster form on large layers.  ``workspace`` is a uint8 CUDA tensor
+    of at least pe_token_sqstats_staged_workspace_bytes(...) bytes; allocated when omitted."""
     B, T, d_in, d_out = _io_check(X, dY, torch.bfloat16)
     if out_stat is None:
         out_stat = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)

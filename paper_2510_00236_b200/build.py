@@ -12,7 +12,7 @@ import sys
 CSRC = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc")
 LIB = os.path.join(CSRC, "libpestats.so")
 SOURCES = ["pe_api.cu"]
-HEADERS = ["pe_optim.cuh", "pe_simt.cuh", "pe_tc.cuh", "pe_sm100.cuh", "../../include/pestats.h"]
+HEADERS = ["pe_optim.cuh", "pe_stage.cuh", "pe_simt.cuh", "pe_tc.cuh", "pe_tok.cuh", "pe_sm100.cuh", "../../include/pestats.h"]
 
 
 def _stale() -> bool:

@@ -12,6 +12,7 @@
 
 #include "../../include/pestats.h"
 #include "pe_optim.cuh"
+#include "pe_stage.cuh"
 #include "pe_simt.cuh"
 #include "pe_tc.cuh"
 #include "pe_tok.cuh"
@@ -107,8 +108,9 @@ static pe_status_t make_operand_map(CUtensorMap* m, const void* base, int B, int
   return r == CUDA_SUCCESS ? PE_OK : PE_ERR_CUDA;
 }
 
-// The tensor-core per-token statistic rounds each squared operand to tf32 (relative error at most
-// 2^-11 per factor, so at most ~1e-3 on any entry, all terms being non-negative).  Tiny problems
+// The tensor-core per-token statistic rounds each squared operand to 11 significant bits (tf32 in the
+// one-kernel form, column-scaled IEEE half in the two-pass form): relative error at most 2^-11 per
+// factor, so at most ~1e-3 on any entry, all terms being non-negative.  Tiny problems
 // gain nothing from the tensor cores and take the SIMT kernel (fp32 squares).
 constexpr long long TOKEN_TC_MIN_ROWS = 256;
 
@@ -201,19 +203,19 @@ static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& m
 // to whichever of out_mean / out_stat is not NULL).  With per_example = 1 and both outputs wanted the
 // pair tile is 256 x 128 (two running sums per thread); with only out_stat it is 256 x 256.
 static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int B, int T, int d_in, int d_out, int phi,
-                             int per_example, float* out_mean, float* out_stat, cudaStream_t st, bool tf32 = false) {
+                             int per_example, float* out_mean, float* out_stat, cudaStream_t st, bool half_ops = false) {
   const bool both = per_example && out_mean && out_stat;
   // Both outputs: sum_b G_b in tensor memory beside a 256-wide accumulator, unless the sequences are
   // so short that the per-example drain of that single accumulator would dominate.
   const bool mean_regs = both && (T < TC_MEAN_TMEM_MIN_T || g_path.load() == PE_PATH_TENSOR_NARROW);
   const int nt = mean_regs ? 128 : 256;
-  const int box_feats = tf32 ? TcOperand<true, 256>::BOX_FEATS : TcOperand<false, 256>::BOX_FEATS;
+  const int box_feats = TcOperand<false, 256>::BOX_FEATS;
   const bool short_seq = mean_regs && T <= TC_SHORT_T;      // many short examples, both outputs: small stages
-  const int box_tokens = short_seq ? TC_SHORT_BK : tc_default_bk(tf32, nt);
+  const int box_tokens = short_seq ? TC_SHORT_BK : tc_default_bk(false, nt);
   CUtensorMap mx, my;
-  pe_status_t rc = make_operand_map(&mx, X, B, T, d_in, tf32, box_feats, box_tokens);
+  pe_status_t rc = make_operand_map(&mx, X, B, T, d_in, false, box_feats, box_tokens);
   if (rc != PE_OK) return rc;
-  rc = make_operand_map(&my, dY, B, T, d_out, tf32, box_feats, box_tokens);
+  rc = make_operand_map(&my, dY, B, T, d_out, false, box_feats, box_tokens);
   if (rc != PE_OK) return rc;
   CUtensorMap mm, ms;       // an output that is not wanted gets the other one's map and is never used
   rc = make_output_map(&mm, out_mean ? out_mean : out_stat, d_in, d_out);
@@ -228,11 +230,10 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
     if (rc != PE_OK) return rc;
   }
   TcParams p;
-  p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = per_example;
+  p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = per_example; p.half_operands = half_ops ? 1 : 0;
   p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
   p.out_mean = out_mean; p.out_stat = out_stat; p.dev_status = di->status_ptr;
   dim3 grid(2 * pairs_m * tiles_n, 1, ns);
-  if (tf32) return launch_tc_inst<0, true, 256, MEAN_NONE>(di, 5, mx, my, mm, ms, p, grid, st);
   if (!per_example) return launch_tc_inst<0, false, 256, MEAN_NONE>(di, 4, mx, my, mm, ms, p, grid, st);
   if (short_seq) {
     if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, MEAN_REGS, TC_SHORT_BK>(di, 8, mx, my, mm, ms, p, grid, st);
@@ -401,10 +402,36 @@ pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_
                                                 d_in, d_out, 0, nullptr, out_stat, st);
 }
 
+// Workspace of the staged per-token statistic: the column maxima of X and dY (one 32-bit word per
+// column), then the scaled squares of X and of dY as IEEE half, each part 256-byte aligned.
+struct StagedLayout {
+  size_t max_bytes, x_bytes, y_bytes;
+  size_t total() const { return max_bytes + x_bytes + y_bytes; }
+};
+static StagedLayout staged_layout(int B, int T, int d_in, int d_out) {
+  const size_t rows = (size_t)B * (size_t)T;
+  StagedLayout l;
+  l.max_bytes = align_up(((size_t)d_in + (size_t)d_out) * 4, 256);
+  l.x_bytes = align_up(rows * d_in * 2, 256);
+  l.y_bytes = align_up(rows * d_out * 2, 256);
+  return l;
+}
+
 size_t pe_token_sqstats_staged_workspace_bytes(int B, int T, int d_in, int d_out) {
   if (g_path.load() == PE_PATH_SIMT || !token_tc_ok(B, T, d_in, d_out)) return 0;
-  const size_t rows = (size_t)B * (size_t)T;
-  return align_up(rows * d_in * 4, 256) + align_up(rows * d_out * 4, 256);
+  return staged_layout(B, T, d_in, d_out).total();
+}
+
+// Grid of the column-wise staging kernels: x covers the columns in groups of 256, y slices the rows
+// so that the whole grid is a few blocks per SM.
+static dim3 stage_grid(long long rows, int d, int sm_count) {
+  const int gx = (d + 255) / 256;
+  long long gy = ((long long)sm_count * 8 + gx - 1) / gx;
+  const long long max_gy = rows / 64 > 0 ? rows / 64 : 1;
+  if (gy > max_gy) gy = max_gy;
+  if (gy > 65535) gy = 65535;
+  if (gy < 1) gy = 1;
+  return dim3((unsigned)gx, (unsigned)gy, 1);
 }
 
 pe_status_t pe_token_sqstats_staged(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_stat,
@@ -421,24 +448,36 @@ pe_status_t pe_token_sqstats_staged(const void* X, const void* dY, int B, int T,
   const bool tc_ok = token_tc_ok(B, T, d_in, d_out);
   if ((forced == PE_PATH_TENSOR || forced == PE_PATH_TENSOR_NARROW) && !tc_shape_ok(B, T, d_in, d_out)) return PE_ERR_UNSUPPORTED_SHAPE;
   if (tc_ok && forced != PE_PATH_SIMT) {
-    const size_t rows = (size_t)B * (size_t)T;
-    const size_t x_bytes = align_up(rows * d_in * 4, 256), y_bytes = align_up(rows * d_out * 4, 256);
-    if (!workspace || workspace_bytes < x_bytes + y_bytes) return PE_ERR_WORKSPACE;
+    const long long rows = (long long)B * T;
+    const StagedLayout l = staged_layout(B, T, d_in, d_out);
+    if (!workspace || workspace_bytes < l.total()) return PE_ERR_WORKSPACE;
     if (!aligned(workspace, 256)) return PE_ERR_ALIGN;
-    float* x2 = static_cast<float*>(workspace);
-    float* y2 = reinterpret_cast<float*>(static_cast<char*>(workspace) + x_bytes);
-    const long long nx = (long long)rows * d_in, ny = (long long)rows * d_out;
-    square_to_tf32_kernel<<<grid_for(nx / 8 + 8, di->sm_count), OPT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(X), x2, nx);
+    uint32_t* max_x = static_cast<uint32_t*>(workspace);
+    uint32_t* max_y = max_x + d_in;
+    __half* x2 = reinterpret_cast<__half*>(static_cast<char*>(workspace) + l.max_bytes);
+    __half* y2 = reinterpret_cast<__half*>(static_cast<char*>(workspace) + l.max_bytes + l.x_bytes);
+    const uint16_t* Xb = static_cast<const uint16_t*>(X);
+    const uint16_t* Yb = static_cast<const uint16_t*>(dY);
+    if (cudaMemsetAsync(max_x, 0, ((size_t)d_in + (size_t)d_out) * 4, st) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
+    const dim3 gx = stage_grid(rows, d_in, di->sm_count), gy = stage_grid(rows, d_out, di->sm_count);
+    column_max_kernel<<<gx, STAGE_THREADS, 0, st>>>(Xb, rows, d_in, max_x);
     if ((rc = check_launch()) != PE_OK) return rc;
-    square_to_tf32_kernel<<<grid_for(ny / 8 + 8, di->sm_count), OPT_THREADS, 0, st>>>(static_cast<const __nv_bfloat16*>(dY), y2, ny);
+    column_max_kernel<<<gy, STAGE_THREADS, 0, st>>>(Yb, rows, d_out, max_y);
+    if ((rc = check_launch()) != PE_OK) return rc;
+    square_to_half_kernel<<<gx, STAGE_THREADS, 0, st>>>(Xb, x2, rows, d_in, max_x);
+    if ((rc = check_launch()) != PE_OK) return rc;
+    square_to_half_kernel<<<gy, STAGE_THREADS, 0, st>>>(Yb, y2, rows, d_out, max_y);
     if ((rc = check_launch()) != PE_OK) return rc;
     // B and T only enter through B*T: regroup the rows into two-stage "examples" when possible so
     // the batch split has many units to balance.
-    constexpr int REGROUP = 2 * TcOperand<true, 256>::BK;
+    constexpr int REGROUP = 2 * TcOperand<false, 256>::BK;
     int Bp = B, Tp = T;
-    if (T % REGROUP == 0 && rows / REGROUP < (size_t)(1u << 30)) { Bp = (int)(rows / REGROUP); Tp = REGROUP; }
+    if (T % REGROUP == 0 && rows / REGROUP < (1ll << 30)) { Bp = (int)(rows / REGROUP); Tp = REGROUP; }
     g_last_path.store(PE_PATH_TENSOR);
-    return launch_tc(di, x2, y2, Bp, Tp, d_in, d_out, PE_PHI_IDENTITY, 0, nullptr, out_stat, st, true);
+    rc = launch_tc(di, x2, y2, Bp, Tp, d_in, d_out, PE_PHI_IDENTITY, 0, nullptr, out_stat, st, true);
+    if (rc != PE_OK) return rc;
+    unscale_kernel<<<grid_for((long long)d_in * d_out / 4 + 4, di->sm_count), STAGE_THREADS, 0, st>>>(out_stat, d_out, d_in, max_x, max_y);
+    return check_launch();
   }
   g_last_path.store(PE_PATH_SIMT);
   return launch_simt<__nv_bfloat16, MODE_TOKEN>(di, static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T,

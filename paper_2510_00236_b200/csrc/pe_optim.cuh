@@ -115,36 +115,4 @@ microsignsgd_kernel(float* __restrict__ theta, __nv_bfloat16* __restrict__ theta
   }
 }
 
-// x -> x*x rounded to tf32 precision (10 explicit mantissa bits, round to nearest even), stored as
-// fp32.  The square of a bf16 value is exact in fp32, so this rounding is the only error: at most
-// 2^-11 relative per operand, and unbiased.
-__device__ __forceinline__ float square_to_tf32(float f) {
-  unsigned int u = __float_as_uint(f * f);
-  u += 0xFFFu + ((u >> 13) & 1u);
-  return __uint_as_float(u & 0xFFFFE000u);
-}
-
-// Operand staging for the tensor-core per-token statistic: dst[k] = tf32(src[k]^2), bf16 -> fp32.
-__global__ void __launch_bounds__(OPT_THREADS)
-square_to_tf32_kernel(const __nv_bfloat16* __restrict__ src, float* __restrict__ dst, long long n) {
-  const long long n8 = n >> 3;
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x; k < n8; k += stride) {
-    uint4 raw = __ldcs(reinterpret_cast<const uint4*>(src) + k);
-    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
-    float4 o[2];
-    float* of = reinterpret_cast<float*>(o);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      float2 f = __bfloat1622float2(h[j]);
-      of[2 * j] = square_to_tf32(f.x);
-      of[2 * j + 1] = square_to_tf32(f.y);
-    }
-    reinterpret_cast<float4*>(dst)[2 * k] = o[0];
-    reinterpret_cast<float4*>(dst)[2 * k + 1] = o[1];
-  }
-  long long k = (n8 << 3) + (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (k < n) dst[k] = square_to_tf32(__bfloat162float(src[k]));
-}
-
 }  // namespace pe

@@ -172,6 +172,10 @@ __host__ __device__ constexpr uint32_t make_idesc_mn_major(int M, int N, bool tf
          | ((uint32_t)(N >> 3) << 17)       // N / 8
          | ((uint32_t)(M >> 4) << 24);      // M / 16
 }
+// The same for kind::f16 with IEEE half A and B.
+__host__ __device__ constexpr uint32_t make_idesc_half_mn_major(int M, int N) {
+  return (1u << 4) | (1u << 15) | (1u << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);   // A, B format: F16 = 0
+}
 // CTA-pair MMA, issued by one thread of the pair's leader block: M rows are split between the two
 // blocks (each supplies its own A rows and receives its own accumulator rows), the N rows of B are
 // split too (each block's shared memory holds half of them at the same offset).

@@ -96,6 +96,7 @@ struct TcParams {
   int nsplit;          // batch slices (gridDim.z); > 1 => outputs pre-zeroed, partials added atomically
   int per_example;     // 1: reset the accumulator for every example and apply phi (statistics)
                        // 0: one accumulation over the whole slice (plain contraction, phi = identity)
+  int half_operands;   // 16-bit operands are IEEE half instead of bf16 (the staged per-token statistic)
   float* out_mean;     // may be NULL; written through tmap_mean
   float* out_stat;     // may be NULL; written through tmap_stat
   unsigned int* dev_status;
@@ -248,7 +249,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       // examples x, x+2, ... of the slice and TMEM buffers x*BUFS_PER_ISSUER .. +BUFS_PER_ISSUER-1.
       if (lane == 0) {
         const int x = (warp == 1) ? 0 : 1;
-        constexpr uint32_t idesc = make_idesc_mn_major(TC_PAIR_M, NT, TF32);
+        const uint32_t idesc = (!TF32 && p.half_operands) ? make_idesc_half_mn_major(TC_PAIR_M, NT) : make_idesc_mn_major(TC_PAIR_M, NT, TF32);
         bool ok = true;
         uint32_t accumulate = 0;
         int i_local = 0;                                   // examples this issuer has started

@@ -103,7 +103,8 @@ def test_register_mean_kernel_at_any_sequence_length(B, T, d_in, d_out):
 @pytest.mark.parametrize("B,T,d_in,d_out", [(5, 200, 136, 264), (64, 64, 512, 256), (3, 1000, 520, 776), (1, 257, 8, 8), (16, 512, 1024, 1024)])
 def test_token_stat_fused_staged_and_oracle_agree(B, T, d_in, d_out):
     """The one-kernel per-token statistic, the two-pass one and the oracle give the same matrix; the two
-    GPU routes round the same tf32 squares, so they differ only by the order of the fp32 sums."""
+    GPU routes round the squares to the same 11 significant bits (tf32 there, column-scaled half here),
+    so they differ only by the order of the fp32 sums."""
     from parity_util import FROB_TOL, oracle_on, rel_frob
     li = inputs.heavy_tailed_layer(B, T, d_in, d_out, seed=1200 + B, device=DEV, with_weights=False)
     fused = torch.full((d_out, d_in), float("nan"), device=DEV)
@@ -118,6 +119,28 @@ def test_token_stat_fused_staged_and_oracle_agree(B, T, d_in, d_out):
     if B * T * d_in * d_out <= 3e9:
         _, tok = oracle_on(li)
         assert rel_frob(f, tok) <= FROB_TOL
+
+
+def test_staged_token_stat_keeps_every_column_accurate_over_a_wide_range_of_magnitudes():
+    """The two-pass route stores the squares as IEEE half with one power-of-two scale per column.  Columns
+    whose magnitudes differ by up to 2^50 (far outside half's range without the scales) must each come
+    out right: the check is entry by entry, not a norm over the matrix."""
+    from parity_util import oracle_on
+    B, T, d_in, d_out = 6, 96, 136, 264
+    li = inputs.gaussian_layer(B, T, d_in, d_out, seed=1300, device=DEV, with_weights=False)
+    gen = torch.Generator().manual_seed(1301)
+    kx = torch.randint(-20, 21, (d_in,), generator=gen).to(DEV)
+    ky = torch.randint(-30, 11, (d_out,), generator=gen).to(DEV)
+    li.X.mul_(torch.pow(2.0, kx.float()).to(torch.bfloat16))          # powers of two: exact in bf16
+    li.dY.mul_(torch.pow(2.0, ky.float()).to(torch.bfloat16))
+    staged = pe.pe_token_sqstats_staged(li.X, li.dY)
+    assert pe.pe_last_path() == pe.PATH_TENSOR
+    torch.cuda.synchronize()
+    assert pe.pe_get_async_status(DEV) == (0, 0)
+    _, tok = oracle_on(li)
+    got = staged.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all() and (tok > 0).all()
+    assert np.max(np.abs(got - tok) / tok) <= 2e-3
 
 
 def test_heavy_tailed_and_heterogeneous_small():

@@ -64,8 +64,9 @@ def test_host_side_validation_needs_no_gpu(lib):
 def test_workspace_size_formula(lib):
     prev = pe.pe_set_path(pe.PATH_AUTO)
     try:
-        assert pe.pe_token_sqstats_staged_workspace_bytes(64, 256, 512, 2048) == 64 * 256 * (512 + 2048) * 4
-        assert pe.pe_token_sqstats_staged_workspace_bytes(30, 10, 8, 8) == 9728 + 9728      # 9600 B rounded up to 256 B each
+        # column maxima (4 B per column), then the squares as half (2 B each); every part a multiple of 256 B
+        assert pe.pe_token_sqstats_staged_workspace_bytes(64, 256, 512, 2048) == (512 + 2048) * 4 + 64 * 256 * (512 + 2048) * 2
+        assert pe.pe_token_sqstats_staged_workspace_bytes(30, 10, 8, 8) == 256 + 4864 + 4864   # 64 B and 4800 B rounded up
         assert pe.pe_token_sqstats_staged_workspace_bytes(3, 5, 8, 8) == 0                  # too few rows for bf16 squares
         assert pe.pe_token_sqstats_staged_workspace_bytes(3, 5, 7, 8) == 0                  # SIMT shape: no workspace
         pe.pe_set_path(pe.PATH_SIMT)
