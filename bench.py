@@ -55,10 +55,13 @@ def measured_peaks():
 
 
 def profile_traffic(workload: str, kernel: str):
-    """DRAM bytes per launch of one kernel from the committed ncu summary of this workload, if present
-    (a line "dram_bytes_per_launch <kernel>: <bytes>")."""
-    path = os.path.join(ROOT, "profiles", f"tc_stats_kernel_{workload}.txt")
-    key = f"dram_bytes_per_launch {kernel}:"
+    """DRAM bytes per launch of one kernel from the committed ncu summaries, if present (a line
+    "dram_bytes_per_launch <kernel>: <bytes>").  The full large layer is too big to capture; its figures are
+    the 16-sequence slice's, scaled by the examples processed (lines "dram_bytes_per_launch_c4 ...")."""
+    fname, tag = {"c2": ("c2", "dram_bytes_per_launch"), "c4s": ("c4_slice", "dram_bytes_per_launch"),
+                  "c4": ("c4_slice", "dram_bytes_per_launch_c4")}.get(workload, (workload, "dram_bytes_per_launch"))
+    path = os.path.join(ROOT, "profiles", f"tc_stats_kernel_{fname}.txt")
+    key = f"{tag} {kernel}:"
     try:
         for line in open(path):
             if line.startswith(key):

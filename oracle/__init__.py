@@ -57,6 +57,12 @@ def _load():
             ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double,
             ctypes.c_int, ctypes.c_double, ctypes.c_int,
         ]
+        lib.oracle_adam_family_step.restype = ctypes.c_int
+        lib.oracle_adam_family_step.argtypes = [
+            c_double_p, c_double_p, c_double_p, c_double_p, c_double_p, ctypes.c_longlong, ctypes.c_int, ctypes.c_int,
+            ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double,
+            ctypes.c_int, ctypes.c_double, ctypes.c_int,
+        ]
         lib.oracle_microsignsgd_step.restype = ctypes.c_int
         lib.oracle_microsignsgd_step.argtypes = [
             c_double_p, c_double_p, c_double_p, ctypes.c_longlong, ctypes.c_int, ctypes.c_double,
@@ -141,6 +147,30 @@ def microadam_step(theta, m, v, sum_g, sum_g2, B, *, grad_scale=1.0, lr, beta1, 
                                        float(eps), int(bool(eps_inside_sqrt)), float(weight_decay), int(step))
     if rc != 0:
         raise RuntimeError("oracle_microadam_step failed")
+    shp = np.shape(theta)
+    return th.reshape(shp), mm.reshape(shp), vv.reshape(shp)
+
+
+ADAM_VARIANTS = {"adam": 0, "microadam": 1, "microadam_var": 2, "microadam_msq": 3}
+
+
+def adam_family_step(theta, m, v, sum_g, sum_g2, B, variant, *, grad_scale=1.0, lr, beta1, beta2, eps,
+                     eps_inside_sqrt=False, weight_decay=0.0, step=1):
+    """One step of a member of the extended Adam family (Section 3.2.3; Algorithm 1 with the estimators of
+    Eq. (6)) in fp64.  variant: "adam", "microadam", "microadam_var", "microadam_msq".  Returns new (theta, m, v)."""
+    th = np.array(theta, np.float64).ravel().copy()
+    mm = np.array(m, np.float64).ravel().copy()
+    vv = np.array(v, np.float64).ravel().copy()
+    g = np.ascontiguousarray(np.asarray(sum_g, np.float64).ravel())
+    g2 = np.ascontiguousarray(np.asarray(sum_g2, np.float64).ravel())
+    n = th.size
+    if not (mm.size == vv.size == g.size == g2.size == n):
+        raise ValueError("size mismatch")
+    rc = _load().oracle_adam_family_step(_dp(th), _dp(mm), _dp(vv), _dp(g), _dp(g2), n, int(B), ADAM_VARIANTS[variant],
+                                         float(grad_scale), float(lr), float(beta1), float(beta2),
+                                         float(eps), int(bool(eps_inside_sqrt)), float(weight_decay), int(step))
+    if rc != 0:
+        raise RuntimeError("oracle_adam_family_step failed")
     shp = np.shape(theta)
     return th.reshape(shp), mm.reshape(shp), vv.reshape(shp)
 

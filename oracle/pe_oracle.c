@@ -169,6 +169,51 @@ int oracle_microadam_step(double* theta, double* m, double* v, const double* sum
 }
 
 /*
+ * One step of the extended Adam family (Section 3.2.3, "A new family of Adam methods"; Algorithm 1).
+ * All members share the first moment and differ in the preconditioner nu, built from
+ *   nu_adam  = mu^2               square of the average gradient
+ *   nu_micro = s^2 * sum_g2 / B   average of the per-example squares
+ * through the unbiased estimators of Eq. (6):
+ *   variant 0  Adam          nu = nu_adam
+ *   variant 1  MicroAdam     nu = nu_micro
+ *   variant 2  MicroAdamVar  nu = sigma2_hat = (nu_micro - nu_adam)     / (1 - 1/B)
+ *   variant 3  MicroAdamMSQ  nu = mu2_hat    = (nu_adam  - nu_micro/B)  / (1 - 1/B)
+ * (Algorithm 1 prints the factor of the last two as B/(1-B) and drops the 1/B inside MicroAdamMSQ; Eq. (6),
+ * which the text says these variants implement, is followed here.)  MicroAdamMSQ clamps the bias-corrected
+ * second moment at zero just before it is used (Algorithm 1; Section 3.2.3: the estimator itself stays unbiased).
+ * Everything else is as in oracle_microadam_step.  Variants 2 and 3 need B >= 2.
+ */
+int oracle_adam_family_step(double* theta, double* m, double* v, const double* sum_g, const double* sum_g2,
+                            long long n, int B, int variant, double grad_scale, double lr, double beta1,
+                            double beta2, double eps, int eps_inside_sqrt, double weight_decay, int step) {
+  if (!theta || !m || !v || !sum_g || !sum_g2 || n < 0 || B < 1 || step < 1) return 1;
+  if (variant < 0 || variant > 3 || (variant >= 2 && B < 2)) return 1;
+  double c1 = 1.0 - pow(beta1, (double)step);
+  double c2 = 1.0 - pow(beta2, (double)step);
+  double bessel = variant >= 2 ? 1.0 / (1.0 - 1.0 / (double)B) : 1.0;
+  for (long long k = 0; k < n; ++k) {
+    double mu = grad_scale * sum_g[k] / (double)B;
+    double nu_adam = mu * mu;
+    double nu_micro = grad_scale * grad_scale * sum_g2[k] / (double)B;
+    double nu;
+    switch (variant) {
+      case 0: nu = nu_adam; break;
+      case 1: nu = nu_micro; break;
+      case 2: nu = bessel * (nu_micro - nu_adam); break;
+      default: nu = bessel * (nu_adam - nu_micro / (double)B); break;
+    }
+    m[k] = beta1 * m[k] + (1.0 - beta1) * mu;
+    v[k] = beta2 * v[k] + (1.0 - beta2) * nu;
+    double mh = m[k] / c1;
+    double vh = v[k] / c2;
+    if (variant == 3 && vh < 0.0) vh = 0.0;
+    double u = eps_inside_sqrt ? mh / sqrt(eps + vh) : mh / (sqrt(vh) + eps);
+    theta[k] = theta[k] - lr * u - weight_decay * theta[k];
+  }
+  return 0;
+}
+
+/*
  * One MicroSignSGD step (Section 3.1: EMA o avg o sign):
  *   sbar = sum_sgn / B                       average of per-example signs
  *   m    = beta m + (1 - beta) sbar          plain EMA, no bias correction

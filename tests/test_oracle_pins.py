@@ -301,6 +301,79 @@ def test_microadam_bias_correction_uses_step_index():
     np.testing.assert_allclose(th, -u, rtol=1e-13)
 
 
+def test_adam_family_original_variant_is_adam_on_the_mean_gradient():
+    """Algorithm 1, "Original": nu = mu^2 at any batch size; torch's Adam fed the average gradient is the library check."""
+    n, B, steps = 23, 5, 3
+    lr, b1, b2, eps = 3e-3, 0.9, 0.99, 1e-8
+    rng = np.random.default_rng(31)
+    theta0 = rng.standard_normal(n)
+    p = torch.nn.Parameter(torch.tensor(theta0, dtype=torch.float64))
+    opt = torch.optim.Adam([p], lr=lr, betas=(b1, b2), eps=eps)
+    th, m, v = theta0.copy(), np.zeros(n), np.zeros(n)
+    for t in range(1, steps + 1):
+        g = rng.standard_normal((B, n))
+        p.grad = torch.tensor(g.mean(0), dtype=torch.float64)
+        opt.step()
+        th, m, v = oracle.adam_family_step(th, m, v, g.sum(0), (g * g).sum(0), B, "adam", lr=lr, beta1=b1, beta2=b2, eps=eps, step=t)
+        np.testing.assert_allclose(th, p.detach().numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_adam_family_preconditioners_are_the_textbook_unbiased_estimators():
+    """Eq. (6): sigma2_hat is the sample variance with Bessel's correction (numpy's var with ddof=1), mu2_hat is
+    mean^2 - var/B, and mu2_hat + sigma2_hat/B = nu_adam.  With beta2 = 0 the returned v IS the preconditioner."""
+    n, B = 41, 7
+    rng = np.random.default_rng(32)
+    g = rng.standard_normal((B, n)) * 0.7 + 0.3
+    kw = dict(lr=0.0, beta1=0.9, beta2=0.0, eps=1e-8, step=1)
+    zeros = np.zeros(n)
+    out = {k: oracle.adam_family_step(zeros, zeros, zeros, g.sum(0), (g * g).sum(0), B, k, **kw)[2] for k in oracle.ADAM_VARIANTS}
+    np.testing.assert_allclose(out["adam"], g.mean(0) ** 2, rtol=1e-13)
+    np.testing.assert_allclose(out["microadam"], (g * g).mean(0), rtol=1e-13)
+    np.testing.assert_allclose(out["microadam_var"], g.var(0, ddof=1), rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(out["microadam_msq"], g.mean(0) ** 2 - g.var(0, ddof=1) / B, rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(out["microadam_msq"] + out["microadam_var"] / B, out["adam"], rtol=1e-12, atol=1e-15)
+    # grad_scale s: sums of G_b = g_b / s give the same estimators
+    s = 4.0
+    v2 = oracle.adam_family_step(zeros, zeros, zeros, g.sum(0) / s, (g * g).sum(0) / s**2, B, "microadam_var", grad_scale=s, **kw)[2]
+    np.testing.assert_allclose(v2, out["microadam_var"], rtol=1e-12, atol=1e-15)
+
+
+def test_adam_family_estimators_are_unbiased_in_expectation():
+    """E[mu2_hat] = mu^2 and E[sigma2_hat] = sigma^2 (Eq. (6)); nu_adam and nu_micro are not (Eq. (5))."""
+    B, n, mu, sigma = 4, 200_000, 0.5, 2.0
+    rng = np.random.default_rng(33)
+    g = rng.standard_normal((B, n)) * sigma + mu
+    kw = dict(lr=0.0, beta1=0.0, beta2=0.0, eps=1e-8, step=1)
+    zeros = np.zeros(n)
+    est = {k: oracle.adam_family_step(zeros, zeros, zeros, g.sum(0), (g * g).sum(0), B, k, **kw)[2].mean() for k in oracle.ADAM_VARIANTS}
+    tol = 6 * 3 * sigma**2 / math.sqrt(n)
+    assert abs(est["microadam_msq"] - mu**2) < tol
+    assert abs(est["microadam_var"] - sigma**2) < tol
+    assert abs(est["adam"] - (mu**2 + sigma**2 / B)) < tol          # Eq. (5): nu_adam carries sigma^2 / B
+    assert abs(est["microadam"] - (mu**2 + sigma**2)) < tol          # nu_micro carries all of sigma^2
+
+
+def test_adam_family_msq_clamps_a_negative_second_moment_only_when_it_is_used():
+    # B = 2, g = {2, -1}: mu = 0.5, nu_adam = 0.25, nu_micro = 2.5, mu2_hat = 2 (0.25 - 1.25) = -2.
+    th, m, v = oracle.adam_family_step([1.0], [0.0], [0.0], [1.0], [5.0], 2, "microadam_msq",
+                                       lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-6, step=1)
+    np.testing.assert_allclose(v, [0.01 * -2.0], rtol=1e-14)          # the EMA keeps the negative value
+    np.testing.assert_allclose(m, [0.05], rtol=1e-14)
+    np.testing.assert_allclose(th, [1.0 - 1e-3 * 0.5 / 1e-6], rtol=1e-12)   # vh clamped to 0: u = mh / eps
+    th_in, _, _ = oracle.adam_family_step([1.0], [0.0], [0.0], [1.0], [5.0], 2, "microadam_msq",
+                                          lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-6, eps_inside_sqrt=True, step=1)
+    np.testing.assert_allclose(th_in, [1.0 - 1e-3 * 0.5 / 1e-3], rtol=1e-12)  # u = mh / sqrt(eps + 0)
+    # the variance needs two examples
+    for k in ("microadam_var", "microadam_msq"):
+        with pytest.raises(RuntimeError):
+            oracle.adam_family_step([1.0], [0.0], [0.0], [1.0], [1.0], 1, k, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8)
+    # and the MicroAdam member is the MicroAdam step
+    a = oracle.adam_family_step([1.0, 2.0], [0.1, 0.0], [0.2, 0.3], [3.0, -1.0], [5.0, 1.0], 2, "microadam", lr=0.1, beta1=0.9, beta2=0.99, eps=1e-8, step=3)
+    b = oracle.microadam_step([1.0, 2.0], [0.1, 0.0], [0.2, 0.3], [3.0, -1.0], [5.0, 1.0], 2, lr=0.1, beta1=0.9, beta2=0.99, eps=1e-8, step=3)
+    for x, y in zip(a, b):
+        np.testing.assert_array_equal(x, y)
+
+
 def test_microsignsgd_reductions():
     n = 20
     rng = np.random.default_rng(23)
