@@ -158,6 +158,25 @@ pe_status_t microadam_step(float* theta, void* theta_lp, float* m, float* v, con
                            float weight_decay, int step, pe_stream_t stream);
 
 /*
+ * One step of a member of the extended Adam family (Section 3.2.3, "A new family of Adam methods";
+ * Algorithm 1).  As microadam_step, except for what feeds the second-moment EMA:
+ *     nu_adam = mu^2,   nu_micro = s^2*sum_g2/B
+ *     PE_ADAM_ORIGINAL   nu = nu_adam                                   (Adam on the average gradient)
+ *     PE_ADAM_MICRO      nu = nu_micro                                  (microadam_step)
+ *     PE_ADAM_MICRO_VAR  nu = (nu_micro - nu_adam)   / (1 - 1/B)        (Eq. (6): unbiased variance)
+ *     PE_ADAM_MICRO_MSQ  nu = (nu_adam - nu_micro/B) / (1 - 1/B)        (Eq. (6): unbiased squared mean)
+ * Algorithm 1 prints the factor of the last two as B/(1-B); Eq. (6), which Section 3.2.3 says they
+ * implement, is followed.  PE_ADAM_MICRO_MSQ clamps vh at zero where it enters u (v itself keeps its
+ * sign, so the estimator stays unbiased); the paper runs it with eps = 1e-6.  The last two need
+ * B >= 2 (PE_ERR_DIM otherwise); an unknown variant is PE_ERR_PHI.
+ */
+typedef enum { PE_ADAM_ORIGINAL = 0, PE_ADAM_MICRO = 1, PE_ADAM_MICRO_VAR = 2, PE_ADAM_MICRO_MSQ = 3 } pe_adam_variant_t;
+pe_status_t microadam_family_step(float* theta, void* theta_lp, float* m, float* v, const float* sum_g,
+                                  const float* sum_g2, long long n, int B, pe_adam_variant_t variant,
+                                  float grad_scale, float lr, float beta1, float beta2, float eps,
+                                  int eps_inside_sqrt, float weight_decay, int step, pe_stream_t stream);
+
+/*
  * One MicroSignSGD step (Section 3.1: EMA o avg o sign):
  *     sbar = sum_sign/B;   m = beta*m + (1-beta)*sbar;   theta = theta - lr*m - weight_decay*theta
  * sum_sign: fp32 [n], the out_stat(sign) of pe_linear_stats.  No bias correction.

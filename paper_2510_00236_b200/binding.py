@@ -17,6 +17,7 @@ __all__ = [
     "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_staged", "pe_token_sqstats_staged_workspace_bytes",
     "microadam_step", "microsignsgd_step", "pe_status_string", "pe_get_async_status", "pe_set_path", "pe_last_path",
     "pe_launch_count", "pe_reset_launch_count", "pe_token_sqstats_static", "STATIC_SCRATCH_BYTES",
+    "microadam_family_step", "ADAM_VARIANTS",
 ]
 
 PHI_IDENTITY, PHI_SQUARE, PHI_SIGN = 0, 1, 2
@@ -28,8 +29,9 @@ EXPORTED_SYMBOLS = [
     "pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_staged",
     "pe_token_sqstats_staged_workspace_bytes", "microadam_step", "microsignsgd_step", "pe_status_string",
     "pe_get_async_status", "pe_set_path", "pe_last_path", "pe_launch_count", "pe_reset_launch_count",
-    "pe_token_sqstats_static",
+    "pe_token_sqstats_static", "microadam_family_step",
 ]
+ADAM_VARIANTS = {"adam": 0, "microadam": 1, "microadam_var": 2, "microadam_msq": 3}      # pe_adam_variant_t
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024      # PE_STATIC_SCRATCH_BYTES of pestats.h
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libpestats.so")
@@ -67,6 +69,7 @@ def load_library() -> ctypes.CDLL:
     lib.pe_token_sqstats_staged_workspace_bytes.argtypes = [i, i, i, i]
     lib.pe_token_sqstats_staged_workspace_bytes.restype = sz
     lib.microadam_step.argtypes = [vp, vp, vp, vp, vp, vp, ll, i, f, f, f, f, f, i, f, i, vp]
+    lib.microadam_family_step.argtypes = [vp, vp, vp, vp, vp, vp, ll, i, i, f, f, f, f, f, i, f, i, vp]
     lib.microsignsgd_step.argtypes = [vp, vp, vp, vp, ll, i, f, f, f, vp]
     lib.pe_status_string.argtypes = [i]
     lib.pe_status_string.restype = ctypes.c_char_p
@@ -79,7 +82,7 @@ def load_library() -> ctypes.CDLL:
     lib.pe_reset_launch_count.restype = None
     for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_static",
                  "pe_token_sqstats_staged",
-                 "microadam_step", "microsignsgd_step", "pe_get_async_status", "pe_set_path", "pe_last_path"):
+                 "microadam_step", "microadam_family_step", "microsignsgd_step", "pe_get_async_status", "pe_set_path", "pe_last_path"):
         getattr(lib, name).restype = i
     _lib = lib
     return lib
@@ -238,6 +241,23 @@ def microadam_step(theta, m, v, sum_g, sum_g2, B, *, lr, beta1, beta2, eps, step
     with _dev_ctx(theta):
         _check("microadam_step", load_library().microadam_step(
             theta.data_ptr(), _ptr(theta_lp), m.data_ptr(), v.data_ptr(), sum_g.data_ptr(), sum_g2.data_ptr(), n, int(B),
+            float(grad_scale), float(lr), float(beta1), float(beta2), float(eps), int(bool(eps_inside_sqrt)),
+            float(weight_decay), int(step), _stream(theta)))
+
+
+def microadam_family_step(theta, m, v, sum_g, sum_g2, B, variant, *, lr, beta1, beta2, eps, step, grad_scale=1.0,
+                          eps_inside_sqrt=False, weight_decay=0.0, theta_lp=None):
+    """In-place update by a member of the extended Adam family: variant is "adam", "microadam",
+    "microadam_var" or "microadam_msq" (or the integer code)."""
+    n = _flat_f32("theta", theta)
+    for name, t in (("m", m), ("v", v), ("sum_g", sum_g), ("sum_g2", sum_g2)):
+        _flat_f32(name, t, n)
+    if theta_lp is not None and (theta_lp.dtype != torch.bfloat16 or theta_lp.numel() != n or not theta_lp.is_contiguous()):
+        raise ValueError("theta_lp must be contiguous bfloat16 with theta's element count")
+    code = ADAM_VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    with _dev_ctx(theta):
+        _check("microadam_family_step", load_library().microadam_family_step(
+            theta.data_ptr(), _ptr(theta_lp), m.data_ptr(), v.data_ptr(), sum_g.data_ptr(), sum_g2.data_ptr(), n, int(B), code,
             float(grad_scale), float(lr), float(beta1), float(beta2), float(eps), int(bool(eps_inside_sqrt)),
             float(weight_decay), int(step), _stream(theta)))
 

@@ -543,11 +543,14 @@ pe_status_t pe_token_sqstats_f32(const float* X, const float* dY, int B, int T, 
   return launch_simt<float, MODE_TOKEN>(di, X, dY, B, T, d_in, d_out, 0, nullptr, out_stat, st);
 }
 
-pe_status_t microadam_step(float* theta, void* theta_lp, float* m, float* v, const float* sum_g, const float* sum_g2,
-                           long long n, int B, float grad_scale, float lr, float beta1, float beta2, float eps,
-                           int eps_inside_sqrt, float weight_decay, int step, pe_stream_t stream) {
+pe_status_t microadam_family_step(float* theta, void* theta_lp, float* m, float* v, const float* sum_g, const float* sum_g2,
+                                  long long n, int B, pe_adam_variant_t variant, float grad_scale, float lr, float beta1,
+                                  float beta2, float eps, int eps_inside_sqrt, float weight_decay, int step,
+                                  pe_stream_t stream) {
   if (!theta || !m || !v || !sum_g || !sum_g2) return PE_ERR_NULL;
   if (n < 0 || B < 1 || step < 1) return PE_ERR_DIM;
+  if ((int)variant < 0 || (int)variant > 3) return PE_ERR_PHI;
+  if (((int)variant == ADAM_MICRO_VAR || (int)variant == ADAM_MICRO_MSQ) && B < 2) return PE_ERR_DIM;   // a variance needs two examples
   if (!aligned(theta, 16) || !aligned(m, 16) || !aligned(v, 16) || !aligned(sum_g, 16) || !aligned(sum_g2, 16) ||
       (theta_lp && !aligned(theta_lp, 16)))
     return PE_ERR_ALIGN;
@@ -562,9 +565,25 @@ pe_status_t microadam_step(float* theta, void* theta_lp, float* m, float* v, con
   p.inv_c1 = (float)(1.0 / (1.0 - std::pow((double)beta1, (double)step)));
   p.inv_c2 = (float)(1.0 / (1.0 - std::pow((double)beta2, (double)step)));
   p.eps = eps; p.lr = lr; p.wd = weight_decay; p.eps_inside = eps_inside_sqrt ? 1 : 0;
-  microadam_kernel<<<grid_for(n / 4 + 4, di->sm_count), OPT_THREADS, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
-      theta, static_cast<__nv_bfloat16*>(theta_lp), m, v, sum_g, sum_g2, n, p);
+  p.inv_B = (float)(1.0 / (double)B);
+  p.bessel = B > 1 ? (float)(1.0 / (1.0 - 1.0 / (double)B)) : 1.f;
+  const int grid = grid_for(n / 4 + 4, di->sm_count);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  __nv_bfloat16* lp = static_cast<__nv_bfloat16*>(theta_lp);
+  switch ((int)variant) {
+    case ADAM_ORIGINAL: microadam_kernel<ADAM_ORIGINAL><<<grid, OPT_THREADS, 0, st>>>(theta, lp, m, v, sum_g, sum_g2, n, p); break;
+    case ADAM_MICRO: microadam_kernel<ADAM_MICRO><<<grid, OPT_THREADS, 0, st>>>(theta, lp, m, v, sum_g, sum_g2, n, p); break;
+    case ADAM_MICRO_VAR: microadam_kernel<ADAM_MICRO_VAR><<<grid, OPT_THREADS, 0, st>>>(theta, lp, m, v, sum_g, sum_g2, n, p); break;
+    default: microadam_kernel<ADAM_MICRO_MSQ><<<grid, OPT_THREADS, 0, st>>>(theta, lp, m, v, sum_g, sum_g2, n, p); break;
+  }
   return check_launch();
+}
+
+pe_status_t microadam_step(float* theta, void* theta_lp, float* m, float* v, const float* sum_g, const float* sum_g2,
+                           long long n, int B, float grad_scale, float lr, float beta1, float beta2, float eps,
+                           int eps_inside_sqrt, float weight_decay, int step, pe_stream_t stream) {
+  return microadam_family_step(theta, theta_lp, m, v, sum_g, sum_g2, n, B, PE_ADAM_MICRO, grad_scale, lr, beta1, beta2, eps,
+                               eps_inside_sqrt, weight_decay, step, stream);
 }
 
 pe_status_t microsignsgd_step(float* theta, void* theta_lp, float* m, const float* sum_sign, long long n, int B, float lr,

@@ -15,16 +15,30 @@ struct AdamParams {
   float inv_c1, inv_c2;   // 1/(1-beta1^t), 1/(1-beta2^t)
   float eps, lr, wd;
   int eps_inside;
+  float inv_B;       // 1 / B
+  float bessel;      // 1 / (1 - 1/B): the factor of the unbiased estimators of Eq. (6)
 };
 
-// Algorithm 1, MicroAdam branch, for one parameter.
+// Members of the extended Adam family (Section 3.2.3): what the second-moment EMA is fed.
+enum : int { ADAM_ORIGINAL = 0, ADAM_MICRO = 1, ADAM_MICRO_VAR = 2, ADAM_MICRO_MSQ = 3 };
+
+// Algorithm 1 for one parameter.  VARIANT picks the preconditioner: mu^2 (Adam), the average of the
+// per-example squares (MicroAdam), or the unbiased estimators of Eq. (6) built from the two
+// (MicroAdamVar: the variance; MicroAdamMSQ: the squared mean, clamped at zero only where it is used).
+template <int VARIANT>
 __device__ __forceinline__ void adam_one(float& th, float& m, float& v, float sg, float sg2, const AdamParams& p) {
   float mu = sg * p.mu_scale;
-  float nu = sg2 * p.nu_scale;
+  float nu_micro = sg2 * p.nu_scale;
+  float nu;
+  if (VARIANT == ADAM_ORIGINAL) nu = mu * mu;
+  else if (VARIANT == ADAM_MICRO) nu = nu_micro;
+  else if (VARIANT == ADAM_MICRO_VAR) nu = p.bessel * (nu_micro - mu * mu);
+  else nu = p.bessel * (mu * mu - nu_micro * p.inv_B);
   m = fmaf(p.beta1, m, (1.f - p.beta1) * mu);
   v = fmaf(p.beta2, v, (1.f - p.beta2) * nu);
   float mh = m * p.inv_c1;
   float vh = v * p.inv_c2;
+  if (VARIANT == ADAM_MICRO_MSQ) vh = fmaxf(vh, 0.f);
   float u = p.eps_inside ? mh / sqrtf(p.eps + vh) : mh / (sqrtf(vh) + p.eps);
   th = th - p.lr * u - p.wd * th;
 }
@@ -33,6 +47,7 @@ __device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p);
 
 constexpr int OPT_THREADS = 256;
 
+template <int VARIANT>
 __global__ void __launch_bounds__(OPT_THREADS)
 microadam_kernel(float* __restrict__ theta, __nv_bfloat16* __restrict__ theta_lp, float* __restrict__ m,
                  float* __restrict__ v, const float* __restrict__ sum_g, const float* __restrict__ sum_g2,
@@ -45,10 +60,10 @@ microadam_kernel(float* __restrict__ theta, __nv_bfloat16* __restrict__ theta_lp
     float4 vv = reinterpret_cast<float4*>(v)[k];
     float4 g = ld_stream(reinterpret_cast<const float4*>(sum_g) + k);
     float4 g2 = ld_stream(reinterpret_cast<const float4*>(sum_g2) + k);
-    adam_one(th.x, mm.x, vv.x, g.x, g2.x, p);
-    adam_one(th.y, mm.y, vv.y, g.y, g2.y, p);
-    adam_one(th.z, mm.z, vv.z, g.z, g2.z, p);
-    adam_one(th.w, mm.w, vv.w, g.w, g2.w, p);
+    adam_one<VARIANT>(th.x, mm.x, vv.x, g.x, g2.x, p);
+    adam_one<VARIANT>(th.y, mm.y, vv.y, g.y, g2.y, p);
+    adam_one<VARIANT>(th.z, mm.z, vv.z, g.z, g2.z, p);
+    adam_one<VARIANT>(th.w, mm.w, vv.w, g.w, g2.w, p);
     reinterpret_cast<float4*>(theta)[k] = th;
     reinterpret_cast<float4*>(m)[k] = mm;
     reinterpret_cast<float4*>(v)[k] = vv;
@@ -65,7 +80,7 @@ microadam_kernel(float* __restrict__ theta, __nv_bfloat16* __restrict__ theta_lp
   long long k = (n4 << 2) + (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (k < n) {
     float th = theta[k], mm = m[k], vv = v[k];
-    adam_one(th, mm, vv, sum_g[k], sum_g2[k], p);
+    adam_one<VARIANT>(th, mm, vv, sum_g[k], sum_g2[k], p);
     theta[k] = th; m[k] = mm; v[k] = vv;
     if (theta_lp) theta_lp[k] = __float2bfloat16_rn(th);
   }

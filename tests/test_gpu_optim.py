@@ -37,6 +37,48 @@ def test_microadam_matches_oracle(n, inside):
     assert torch.equal(lp, d[0].to(torch.bfloat16))
 
 
+@pytest.mark.parametrize("variant", ["adam", "microadam", "microadam_var", "microadam_msq"])
+@pytest.mark.parametrize("n,inside", [(3, False), (4099, False), ((1 << 19) + 1, True)])
+def test_adam_family_matches_oracle(variant, n, inside):
+    """Every member of the extended Adam family (Section 3.2.3) against the fp64 oracle.  The sums are built so
+    that the squared-mean estimator is clearly positive on even entries and clearly negative on odd ones (there
+    MicroAdamMSQ must clamp), never near zero where fp32 and fp64 could take different sides."""
+    g = torch.Generator().manual_seed(n + len(variant))
+    B = 8
+    theta = torch.randn(n, generator=g)
+    m = torch.randn(n, generator=g) * 0.1
+    sg = (torch.rand(n, generator=g) + 0.5) * torch.where(torch.rand(n, generator=g) < 0.5, -1.0, 1.0) * 3
+    odd = (torch.arange(n) % 2 == 1)
+    sg2 = torch.where(odd, 4 * sg * sg + 1, 0.25 * sg * sg)
+    if variant == "microadam_var":
+        sg2 = sg * sg / B * (1.5 + torch.rand(n, generator=g))         # a variance estimate is never negative
+    v = torch.zeros(n) if variant == "microadam_msq" else torch.rand(n, generator=g) * 0.1
+    kw = dict(lr=1e-2, beta1=0.9, beta2=0.95, eps=1e-6, step=2, grad_scale=0.5, weight_decay=1e-3, eps_inside_sqrt=inside)
+    ref = oracle.adam_family_step(theta.numpy(), m.numpy(), v.numpy(), sg.numpy(), sg2.numpy(), B, variant, **kw)
+    d = [t.to(DEV).contiguous() for t in (theta, m, v, sg, sg2)]
+    lp = torch.empty(n, dtype=torch.bfloat16, device=DEV)
+    pe.microadam_family_step(d[0], d[1], d[2], d[3], d[4], B, variant, theta_lp=lp, **kw)
+    torch.cuda.synchronize()
+    if variant == "microadam_msq" and n > 1:
+        assert (ref[2][1::2] < 0).all() and (ref[2][0::2] > 0).all()    # both branches of the clamp are exercised
+    for got, want in zip(d[:3], ref):
+        assert rel_frob(got.cpu().numpy(), want) <= 1e-5 <= FROB_TOL
+    assert rel_frob((d[0].cpu() - theta).numpy(), ref[0] - theta.numpy().astype(np.float64)) <= FROB_TOL
+    assert torch.equal(lp, d[0].to(torch.bfloat16))
+
+
+def test_adam_family_rejects_what_it_cannot_compute():
+    t = [torch.zeros(8, device=DEV) for _ in range(5)]
+    kw = dict(lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8, step=1)
+    for variant in ("microadam_var", "microadam_msq"):
+        with pytest.raises(pe.PestatsError) as e:
+            pe.microadam_family_step(*t, 1, variant, **kw)                 # a variance needs two examples
+        assert e.value.status == 2
+    with pytest.raises(pe.PestatsError) as e:
+        pe.microadam_family_step(*t, 4, 7, **kw)
+    assert e.value.status == 5
+
+
 def test_config1_statistics_then_microadam_step():
     li = inputs.config1(DEV)
     mean, stat = pe.pe_linear_stats_f32(li.X, li.dY, "square")
