@@ -48,7 +48,7 @@ typedef enum { PE_PHI_IDENTITY = 0, PE_PHI_SQUARE = 1, PE_PHI_SIGN = 2 } pe_phi_
 /* Which kernel family a call may use.  AUTO picks the tensor-core kernel whenever the shape allows
  * it (bf16 inputs, d_in % 8 == 0, d_out % 8 == 0) and the SIMT kernel otherwise.  TENSOR_NARROW is
  * TENSOR with the 256 x 128 tile that keeps both running sums in registers even for long sequences
- * (AUTO and TENSOR use it for T < 2048 only and otherwise keep sum_b G_b in tensor memory beside a
+ * (AUTO and TENSOR use it for T < 4096 only and otherwise keep sum_b G_b in tensor memory beside a
  * 256 x 256 tile); it exists so that tests can reach that kernel at any T. */
 typedef enum { PE_PATH_AUTO = 0, PE_PATH_SIMT = 1, PE_PATH_TENSOR = 2, PE_PATH_TENSOR_NARROW = 3 } pe_path_t;
 
@@ -74,6 +74,19 @@ pe_status_t pe_linear_stats(const void* X, const void* dY, int B, int T, int d_i
 /* Same for fp32 inputs (4-byte aligned suffices); always the SIMT kernel, fp32 FMA accumulation. */
 pe_status_t pe_linear_stats_f32(const float* X, const float* dY, int B, int T, int d_in, int d_out,
                                 pe_phi_t phi, float* out_mean, float* out_stat, pe_stream_t stream);
+
+/*
+ * The three statistics of pe_linear_stats in one pass over the examples (Eq. (2) with phi = identity,
+ * square and sign at once; Sections 2.1 and 3.1):
+ *     out_mean = sum_b G_b,   out_square = sum_b G_b^2,   out_sign = sum_b sign(G_b),   G_b = dY_b^T X_b.
+ * bf16 inputs as for pe_linear_stats; all three outputs [d_out, d_in] fp32, 16-byte aligned, non-NULL,
+ * overwritten.  Each G_b tile is formed once and feeds all three running sums (the sign sum is kept
+ * as a per-column count), so the call costs about one pe_linear_stats(square) instead of that plus a
+ * pe_linear_stats(sign).  Shapes the one-pass kernel does not take (sequences of at most 64 tokens,
+ * widths that are not multiples of 8, the SIMT path forced) are served by those two calls.
+ */
+pe_status_t pe_linear_stats_all(const void* X, const void* dY, int B, int T, int d_in, int d_out,
+                                float* out_mean, float* out_square, float* out_sign, pe_stream_t stream);
 
 /*
  * Per-token second moment (Section 2.3, the "per-token" alternative):

@@ -17,7 +17,7 @@ __all__ = [
     "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_staged", "pe_token_sqstats_staged_workspace_bytes",
     "microadam_step", "microsignsgd_step", "pe_status_string", "pe_get_async_status", "pe_set_path", "pe_last_path",
     "pe_launch_count", "pe_reset_launch_count", "pe_token_sqstats_static", "STATIC_SCRATCH_BYTES",
-    "microadam_family_step", "ADAM_VARIANTS",
+    "microadam_family_step", "ADAM_VARIANTS", "pe_linear_stats_all",
 ]
 
 PHI_IDENTITY, PHI_SQUARE, PHI_SIGN = 0, 1, 2
@@ -29,7 +29,7 @@ EXPORTED_SYMBOLS = [
     "pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_staged",
     "pe_token_sqstats_staged_workspace_bytes", "microadam_step", "microsignsgd_step", "pe_status_string",
     "pe_get_async_status", "pe_set_path", "pe_last_path", "pe_launch_count", "pe_reset_launch_count",
-    "pe_token_sqstats_static", "microadam_family_step",
+    "pe_token_sqstats_static", "microadam_family_step", "pe_linear_stats_all",
 ]
 ADAM_VARIANTS = {"adam": 0, "microadam": 1, "microadam_var": 2, "microadam_msq": 3}      # pe_adam_variant_t
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024      # PE_STATIC_SCRATCH_BYTES of pestats.h
@@ -62,6 +62,7 @@ def load_library() -> ctypes.CDLL:
     vp, i, f, ll, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_longlong, ctypes.c_size_t
     lib.pe_linear_stats.argtypes = [vp, vp, i, i, i, i, i, vp, vp, vp]
     lib.pe_linear_stats_f32.argtypes = [vp, vp, i, i, i, i, i, vp, vp, vp]
+    lib.pe_linear_stats_all.argtypes = [vp, vp, i, i, i, i, vp, vp, vp, vp]
     lib.pe_token_sqstats.argtypes = [vp, vp, i, i, i, i, vp, vp]
     lib.pe_token_sqstats_staged.argtypes = [vp, vp, i, i, i, i, vp, vp, sz, vp]
     lib.pe_token_sqstats_f32.argtypes = [vp, vp, i, i, i, i, vp, vp]
@@ -80,7 +81,7 @@ def load_library() -> ctypes.CDLL:
     lib.pe_launch_count.restype = ll
     lib.pe_reset_launch_count.argtypes = []
     lib.pe_reset_launch_count.restype = None
-    for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_static",
+    for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_linear_stats_all", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_static",
                  "pe_token_sqstats_staged",
                  "microadam_step", "microadam_family_step", "microsignsgd_step", "pe_get_async_status", "pe_set_path", "pe_last_path"):
         getattr(lib, name).restype = i
@@ -144,6 +145,22 @@ def pe_linear_stats(X, dY, phi, out_mean=None, out_stat=None):
         _check("pe_linear_stats", load_library().pe_linear_stats(
             X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, _phi(phi), _ptr(out_mean), _ptr(out_stat), _stream(X)))
     return out_mean, out_stat
+
+
+def pe_linear_stats_all(X, dY, out_mean=None, out_square=None, out_sign=None):
+    """sum_b G_b, sum_b G_b^2 and sum_b sign(G_b) in one pass (bf16 inputs); returns the three [d_out, d_in]
+    float32 tensors.  Missing outputs are allocated."""
+    B, T, d_in, d_out = _io_check(X, dY, torch.bfloat16)
+    outs = []
+    for name, t in (("out_mean", out_mean), ("out_square", out_square), ("out_sign", out_sign)):
+        if t is None:
+            t = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)
+        _out_check(name, t, d_out, d_in)
+        outs.append(t)
+    with _dev_ctx(X):
+        _check("pe_linear_stats_all", load_library().pe_linear_stats_all(
+            X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, outs[0].data_ptr(), outs[1].data_ptr(), outs[2].data_ptr(), _stream(X)))
+    return tuple(outs)
 
 
 def pe_linear_stats_f32(X, dY, phi, out_mean=None, out_stat=None):

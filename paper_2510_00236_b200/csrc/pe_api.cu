@@ -24,7 +24,9 @@ __device__ unsigned int g_dev_status = 0;   // first device-side wait that gave 
 static std::atomic<int> g_path{PE_PATH_AUTO};
 static std::atomic<int> g_last_path{PE_PATH_AUTO};
 static std::atomic<long long> g_launches{0};
-constexpr int TC_MEAN_TMEM_MIN_T = 2048;
+// Both outputs: from this sequence length on the running sum of G_b lives in tensor memory beside a
+// 256-column accumulator (measured: wins or ties at T = 4096, loses 16 % at T = 2048, 17 % at T = 1024).
+constexpr int TC_MEAN_TMEM_MIN_T = 4096;
 constexpr int TC_BAND = 8;          // pair rows per band of the tile order (8 x 256 rows of d_out)
 
 constexpr int MAX_DEVICES = 64;
@@ -32,7 +34,7 @@ struct DeviceInfo {
   std::atomic<int> state{0};     // 0 unknown, 1 ready, -1 failed
   int cc_major = 0, sm_count = 0;
   unsigned int* status_ptr = nullptr;
-  bool tc_attr_set[10] = {};
+  bool tc_attr_set[11] = {};
   bool tok_attr_set = false;
 };
 static DeviceInfo g_dev[MAX_DEVICES];
@@ -160,15 +162,16 @@ static pe_status_t zero_outputs(float* a, float* b, size_t bytes, cudaStream_t s
   return PE_OK;
 }
 
-// Zeroes one or two [d_out, d_in] outputs with a kernel that lets its successor start at once.
-static pe_status_t zero_for_split(DeviceInfo* di, float* a, float* b, size_t n, cudaStream_t st) {
+// Zeroes up to three [d_out, d_in] outputs with a kernel that lets its successor start at once.
+static pe_status_t zero_for_split(DeviceInfo* di, float* a, float* b, size_t n, cudaStream_t st, float* c = nullptr) {
   float* first = a ? a : b;
   float* second = a ? b : nullptr;
   if (!first) return PE_OK;
   const long long n4 = (long long)(n / 4);          // d_in % 8 == 0 on this path
   long long blocks = (n4 + 255) / 256;
   if (blocks > di->sm_count) blocks = di->sm_count;   // few blocks: the dependent kernel needs the SMs
-  zero_outputs_kernel<<<(int)(blocks < 1 ? 1 : blocks), 256, 0, st>>>(reinterpret_cast<float4*>(first), reinterpret_cast<float4*>(second), n4);
+  zero_outputs_kernel<<<(int)(blocks < 1 ? 1 : blocks), 256, 0, st>>>(reinterpret_cast<float4*>(first), reinterpret_cast<float4*>(second),
+                                                                            reinterpret_cast<float4*>(c), n4);
   return check_launch();
 }
 
@@ -187,7 +190,7 @@ static pe_status_t launch_pair_kernel(Kernel kernel, dim3 grid, int smem, cudaSt
 
 template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT)>
 static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& mm,
-                                  const CUtensorMap& ms, const TcParams& p, dim3 grid, cudaStream_t st) {
+                                  const CUtensorMap& ms, const CUtensorMap& msgn, const TcParams& p, dim3 grid, cudaStream_t st) {
   constexpr int smem = TcOperand<TF32, NT, BKT>::SMEM_BYTES;
   if (!di->tc_attr_set[slot]) {
     if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
@@ -196,21 +199,23 @@ static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& m
     }
     di->tc_attr_set[slot] = true;
   }
-  return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT>, grid, smem, st, p.nsplit > 1, mx, my, mm, ms, p);
+  return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT>, grid, smem, st, p.nsplit > 1, mx, my, mm, ms, msgn, p);
 }
 
 // Tensor-core launch.  per_example = 0 runs the plain contraction over all B*T rows (its result goes
 // to whichever of out_mean / out_stat is not NULL).  With per_example = 1 and both outputs wanted the
 // pair tile is 256 x 128 (two running sums per thread); with only out_stat it is 256 x 256.
 static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int B, int T, int d_in, int d_out, int phi,
-                             int per_example, float* out_mean, float* out_stat, cudaStream_t st, bool half_ops = false) {
+                             int per_example, float* out_mean, float* out_stat, cudaStream_t st, bool half_ops = false,
+                             float* out_sign = nullptr) {
+  const bool triple = out_sign != nullptr;       // mean + square + sign in one pass (phi = square, all three outputs given)
   const bool both = per_example && out_mean && out_stat;
   // Both outputs: sum_b G_b in tensor memory beside a 256-wide accumulator, unless the sequences are
   // so short that the per-example drain of that single accumulator would dominate.
-  const bool mean_regs = both && (T < TC_MEAN_TMEM_MIN_T || g_path.load() == PE_PATH_TENSOR_NARROW);
+  const bool mean_regs = both && (triple || T < TC_MEAN_TMEM_MIN_T || g_path.load() == PE_PATH_TENSOR_NARROW);
   const int nt = mean_regs ? 128 : 256;
   const int box_feats = TcOperand<false, 256>::BOX_FEATS;
-  const bool short_seq = mean_regs && T <= TC_SHORT_T;      // many short examples, both outputs: small stages
+  const bool short_seq = mean_regs && !triple && T <= TC_SHORT_T;      // many short examples, both outputs: small stages
   const int box_tokens = short_seq ? TC_SHORT_BK : tc_default_bk(false, nt);
   CUtensorMap mx, my;
   pe_status_t rc = make_operand_map(&mx, X, B, T, d_in, false, box_feats, box_tokens);
@@ -222,33 +227,37 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   if (rc != PE_OK) return rc;
   rc = make_output_map(&ms, out_stat ? out_stat : out_mean, d_in, d_out);
   if (rc != PE_OK) return rc;
+  CUtensorMap msgn = ms;
+  if (triple && (rc = make_output_map(&msgn, out_sign, d_in, d_out)) != PE_OK) return rc;
   const int tiles_n = (d_in + nt - 1) / nt, pairs_m = (d_out + TC_PAIR_M - 1) / TC_PAIR_M;
   if ((long long)tiles_n * pairs_m > (1ll << 29)) return PE_ERR_DIM;
-  const int ns = choose_nsplit((long long)tiles_n * pairs_m, B, T, di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 16);
+  int ns = choose_nsplit((long long)tiles_n * pairs_m, B, T, di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 16);
+  if (triple && (B + ns - 1) / ns > TC_SIGN_COUNT_MAX) ns = (B + TC_SIGN_COUNT_MAX - 1) / TC_SIGN_COUNT_MAX;   // 16-bit sign counters
   if (ns > 1) {
-    rc = zero_for_split(di, out_mean, out_stat, (size_t)d_in * d_out, st);
+    rc = zero_for_split(di, out_mean, out_stat, (size_t)d_in * d_out, st, out_sign);
     if (rc != PE_OK) return rc;
   }
   TcParams p;
   p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = per_example; p.half_operands = half_ops ? 1 : 0;
   p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
-  p.out_mean = out_mean; p.out_stat = out_stat; p.dev_status = di->status_ptr;
+  p.out_mean = out_mean; p.out_stat = out_stat; p.out_sign = out_sign; p.dev_status = di->status_ptr;
   dim3 grid(2 * pairs_m * tiles_n, 1, ns);
-  if (!per_example) return launch_tc_inst<0, false, 256, MEAN_NONE>(di, 4, mx, my, mm, ms, p, grid, st);
+  if (triple) return launch_tc_inst<1, false, 128, MEAN_REGS_SIGN>(di, 10, mx, my, mm, ms, msgn, p, grid, st);
+  if (!per_example) return launch_tc_inst<0, false, 256, MEAN_NONE>(di, 4, mx, my, mm, ms, msgn, p, grid, st);
   if (short_seq) {
-    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, MEAN_REGS, TC_SHORT_BK>(di, 8, mx, my, mm, ms, p, grid, st);
-    return launch_tc_inst<2, false, 128, MEAN_REGS, TC_SHORT_BK>(di, 9, mx, my, mm, ms, p, grid, st);
+    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, MEAN_REGS, TC_SHORT_BK>(di, 8, mx, my, mm, ms, msgn, p, grid, st);
+    return launch_tc_inst<2, false, 128, MEAN_REGS, TC_SHORT_BK>(di, 9, mx, my, mm, ms, msgn, p, grid, st);
   }
   if (mean_regs) {
-    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, MEAN_REGS>(di, 0, mx, my, mm, ms, p, grid, st);
-    return launch_tc_inst<2, false, 128, MEAN_REGS>(di, 1, mx, my, mm, ms, p, grid, st);
+    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, MEAN_REGS>(di, 0, mx, my, mm, ms, msgn, p, grid, st);
+    return launch_tc_inst<2, false, 128, MEAN_REGS>(di, 1, mx, my, mm, ms, msgn, p, grid, st);
   }
   if (both) {
-    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, MEAN_TMEM>(di, 6, mx, my, mm, ms, p, grid, st);
-    return launch_tc_inst<2, false, 256, MEAN_TMEM>(di, 7, mx, my, mm, ms, p, grid, st);
+    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, MEAN_TMEM>(di, 6, mx, my, mm, ms, msgn, p, grid, st);
+    return launch_tc_inst<2, false, 256, MEAN_TMEM>(di, 7, mx, my, mm, ms, msgn, p, grid, st);
   }
-  if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, MEAN_NONE>(di, 2, mx, my, mm, ms, p, grid, st);
-  return launch_tc_inst<2, false, 256, MEAN_NONE>(di, 3, mx, my, mm, ms, p, grid, st);
+  if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, MEAN_NONE>(di, 2, mx, my, mm, ms, msgn, p, grid, st);
+  return launch_tc_inst<2, false, 256, MEAN_NONE>(di, 3, mx, my, mm, ms, msgn, p, grid, st);
 }
 
 template <typename TIn, int MODE>
@@ -372,6 +381,30 @@ pe_status_t pe_linear_stats(const void* X, const void* dY, int B, int T, int d_i
                             float* out_mean, float* out_stat, pe_stream_t stream) {
   return linear_stats_impl<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T,
                                           d_in, d_out, phi, out_mean, out_stat, reinterpret_cast<cudaStream_t>(stream), true);
+}
+
+pe_status_t pe_linear_stats_all(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_mean,
+                                float* out_square, float* out_sign, pe_stream_t stream) {
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (!out_mean || !out_square || !out_sign) return PE_ERR_NULL;
+  pe_status_t rc = validate_stats(X, dY, B, T, d_in, d_out, out_mean, out_square, true, 16);
+  if (rc != PE_OK) return rc;
+  if (!aligned(out_sign, 16)) return PE_ERR_ALIGN;
+  DeviceInfo* di = nullptr;
+  rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  const int forced = g_path.load();
+  // One pass when the tensor-core kernel takes the shape and an example spans more than a short
+  // stage; otherwise the two calls this one stands for.
+  if (B > 0 && T > TC_SHORT_T && forced != PE_PATH_SIMT && tc_shape_ok(B, T, d_in, d_out)) {
+    g_last_path.store(PE_PATH_TENSOR);
+    return launch_tc(di, X, dY, B, T, d_in, d_out, PE_PHI_SQUARE, 1, out_mean, out_square, st, false, out_sign);
+  }
+  const __nv_bfloat16* Xb = static_cast<const __nv_bfloat16*>(X);
+  const __nv_bfloat16* Yb = static_cast<const __nv_bfloat16*>(dY);
+  rc = linear_stats_impl<__nv_bfloat16>(Xb, Yb, B, T, d_in, d_out, PE_PHI_SQUARE, out_mean, out_square, st, true);
+  if (rc != PE_OK) return rc;
+  return linear_stats_impl<__nv_bfloat16>(Xb, Yb, B, T, d_in, d_out, PE_PHI_SIGN, nullptr, out_sign, st, true);
 }
 
 pe_status_t pe_linear_stats_f32(const float* X, const float* dY, int B, int T, int d_in, int d_out, pe_phi_t phi,

@@ -11,6 +11,8 @@
 // 128 x 128 tile would need 128 B/clk at full tensor rate, a 256 x 128 pair 96, a 256 x 256 pair 64.
 //
 //   MEAN_REGS, NT = 128: two running sums per thread (64 + 64 registers)         -- both outputs, short sequences
+//   MEAN_REGS_SIGN, NT = 128: the same plus sum_b sign(G_b), counted in 16-bit halves
+//                        of 32 more registers                                      -- mean, square and sign in one pass
 //   MEAN_TMEM, NT = 256: sum_b phi(G_b) in 128 registers per thread, sum_b G_b in
 //                        tensor memory beside ONE per-example accumulator, one issuer -- both outputs
 //   MEAN_NONE, NT = 256: one running sum per thread (128 registers)               -- only sum_b phi(G_b) wanted
@@ -99,6 +101,7 @@ struct TcParams {
   int half_operands;   // 16-bit operands are IEEE half instead of bf16 (the staged per-token statistic)
   float* out_mean;     // may be NULL; written through tmap_mean
   float* out_stat;     // may be NULL; written through tmap_stat
+  float* out_sign;     // MEAN_REGS_SIGN only: sum_b sign(G_b), written through tmap_sign
   unsigned int* dev_status;
 };
 
@@ -145,28 +148,35 @@ struct StageWalk {
 
 // Zeroes the outputs of a split-batch launch.  The statistics kernel that follows is launched as a
 // programmatic dependent: it starts right away (it only touches the outputs in its very last step,
-// behind griddepcontrol.wait), so the zeroing costs no time on the stream.  a, b: n4 float4 each; b may
-// be NULL.
-__global__ void __launch_bounds__(256) zero_outputs_kernel(float4* __restrict__ a, float4* __restrict__ b, long long n4) {
+// behind griddepcontrol.wait), so the zeroing costs no time on the stream.  a, b, c: n4 float4 each; b and
+// c may be NULL.
+__global__ void __launch_bounds__(256) zero_outputs_kernel(float4* __restrict__ a, float4* __restrict__ b, float4* __restrict__ c,
+                                                           long long n4) {
   sm100::griddep_launch_dependents();
   const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x; k < n4; k += stride) {
     a[k] = z;
     if (b) b[k] = z;
+    if (c) c[k] = z;
   }
 }
 
-enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2 };   // where sum_b G_b is kept in per-example mode
+// where sum_b G_b is kept in per-example mode; MEAN_REGS_SIGN = MEAN_REGS with phi = square plus the sign statistic
+enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2, MEAN_REGS_SIGN = 3 };
+constexpr int TC_SIGN_COUNT_MAX = 32767;   // examples per block in MEAN_REGS_SIGN mode: 2 * count must fit 16 bits
 
 // gridDim = (2 * pairs_m * tiles_n, 1, nsplit); blockIdx.x = 2 * (pair index in the tile order) + rank in pair.
 template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT)>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
-                const __grid_constant__ CUtensorMap tmap_mean, const __grid_constant__ CUtensorMap tmap_stat, TcParams p) {
+                const __grid_constant__ CUtensorMap tmap_mean, const __grid_constant__ CUtensorMap tmap_stat,
+                const __grid_constant__ CUtensorMap tmap_sign, TcParams p) {
   using namespace sm100;
   using Op = TcOperand<TF32, NT, BKT>;
-  static_assert(MEAN != MEAN_REGS || NT == 128, "two running sums only fit the registers at NT = 128");
+  constexpr bool TRIPLE = (MEAN == MEAN_REGS_SIGN);
+  static_assert((MEAN != MEAN_REGS && !TRIPLE) || NT == 128, "two running sums only fit the registers at NT = 128");
+  static_assert(!TRIPLE || PHI == 1, "the three-statistic mode is mean + square + sign");
   static_assert(MEAN != MEAN_TMEM || (NT == 256 && PHI != 0), "the tensor-memory mean sits beside one 256-column accumulator");
   constexpr int STAGES = Op::STAGES, BK = Op::BK;
   constexpr int BOX_BYTES = Op::BOX_BYTES, A_BYTES = Op::A_BYTES, STAGE_BYTES = Op::STAGE_BYTES;
@@ -300,10 +310,16 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     setmaxnreg_inc<TC_REGS_EPILOGUE>();
     const int q = warp & 3;                 // TMEM lane quadrant this warp may access
     const int h = (warp - 4) >> 2;          // column half of the tile
-    constexpr bool KEEP_MEAN = MEAN == MEAN_REGS || PHI == 0;     // running sum of G_b in registers
+    constexpr bool KEEP_MEAN = MEAN == MEAN_REGS || TRIPLE || PHI == 0;     // running sum of G_b in registers
     constexpr int N_STAT = (PHI != 0) ? COLS : 1;
     constexpr int N_MEAN = KEEP_MEAN ? COLS : 1;
     float acc_stat[N_STAT], acc_mean[N_MEAN];
+    // TRIPLE: per column, sum_b (sign(G_b) + 1), a count in [0, 2 nb] that fits 16 bits; two columns per
+    // register, so the third statistic costs 32 registers instead of 64.  sum_b sign = count - nb.
+    constexpr int N_CNT = TRIPLE ? COLS / 2 : 1;
+    uint32_t acc_cnt[N_CNT];
+#pragma unroll
+    for (int j = 0; j < N_CNT; ++j) acc_cnt[j] = 0u;
 #pragma unroll
     for (int j = 0; j < N_STAT; ++j) acc_stat[j] = 0.f;
 #pragma unroll
@@ -372,6 +388,13 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
               if (PHI == 1) {
                 const uint64_t s2 = f32x2_fma(g2, g2, f32x2_pack(acc_stat[c * 32 + j], acc_stat[c * 32 + j + 1]));
                 f32x2_unpack(s2, acc_stat[c * 32 + j], acc_stat[c * 32 + j + 1]);
+              }
+              if (TRIPLE) {
+                const float g0 = __uint_as_float(r[j]), g1 = __uint_as_float(r[j + 1]);
+                // sign + 1 in {0, 1, 2}; +0 and -0 both give 1
+                const uint32_t c0 = 1u + (g0 > 0.f ? 1u : 0u) - (g0 < 0.f ? 1u : 0u);
+                const uint32_t c1 = 1u + (g1 > 0.f ? 1u : 0u) - (g1 < 0.f ? 1u : 0u);
+                acc_cnt[(c * 32 + j) >> 1] += c0 + (c1 << 16);
               }
             }
           }
@@ -443,6 +466,22 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
           for (int c = 0; c < PANELS; ++c) put_panel(first + c * 4096, &acc_mean[c * 32]);
         }
         send(&tmap_mean, first);
+      }
+      if constexpr (TRIPLE) {
+        // sum_b sign(G_b): the warp's 16 KiB are in use, so wait until TMA has read them
+        if (p.out_sign) {
+          if (lane == 0) bulk_wait_read_all();
+          __syncwarp();
+          const float nbf = (float)nb;
+#pragma unroll
+          for (int c = 0; c < PANELS; ++c) {
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = (float)((acc_cnt[(c * 32 + j) >> 1] >> (16 * (j & 1))) & 0xFFFFu) - nbf;
+            put_panel(stage_base + c * 4096, v);
+          }
+          send(&tmap_sign, stage_base);
+        }
       }
       if (lane == 0) bulk_wait_read_all();       // shared memory must outlive TMA's reads
     }

@@ -44,6 +44,7 @@ def test_structured_single_tile_catches_layout_mistakes():
     (130, 32, 264, 392),    # many short sequences: 32-token stages, batch split
     (21, 64, 136, 520),     # two short stages per example
     (11, 33, 128, 256),     # one full and one nearly empty short stage
+    (2, 4100, 136, 264),    # very long sequences: sum_b G_b kept in tensor memory when both outputs are wanted
 ])
 def test_tensor_small_shapes_full_comparison(B, T, d_in, d_out):
     li = inputs.gaussian_layer(B, T, d_in, d_out, seed=300 + 7 * B + T, device=DEV)
@@ -141,6 +142,55 @@ def test_staged_token_stat_keeps_every_column_accurate_over_a_wide_range_of_magn
     got = staged.cpu().numpy().astype(np.float64)
     assert np.isfinite(got).all() and (tok > 0).all()
     assert np.max(np.abs(got - tok) / tok) <= 2e-3
+
+
+@pytest.mark.parametrize("B,T,d_in,d_out,tensor_one_pass", [
+    (5, 200, 136, 264, True),      # ragged tiles, ragged T
+    (70, 96, 8, 8, True),          # one tile, batch split across blocks: partial sign counts are added
+    (33, 300, 520, 264, True),     # odd slices
+    (1, 1000, 256, 128, True),     # single example
+    (64, 256, 512, 2048, True),    # the benchmark layer, sampled below
+    (9, 16, 320, 192, False),      # short sequences: served by the two separate calls
+    (6, 40, 36, 20, False),        # widths the tensor-core path does not take
+])
+def test_three_statistics_in_one_pass(B, T, d_in, d_out, tensor_one_pass):
+    """pe_linear_stats_all: sum_b G_b, sum_b G_b^2 and sum_b sign(G_b) from one pass over the examples, against
+    the oracle (full comparison on the small shapes, sampled rows x columns on the benchmark layer)."""
+    from parity_util import FROB_TOL, boundary_and_random, check_sign, oracle_on, rel_frob
+    li = inputs.heterogeneous_layer(B, T, d_in, d_out, seed=1400 + B, device=DEV, with_weights=False)
+    outs = [torch.full((d_out, d_in), float("nan"), device=DEV) for _ in range(3)]
+    launches0 = pe.pe_launch_count()
+    pe.pe_linear_stats_all(li.X, li.dY, *outs)
+    torch.cuda.synchronize()
+    assert pe.pe_get_async_status(DEV) == (0, 0)
+    if tensor_one_pass:
+        assert pe.pe_last_path() == pe.PATH_TENSOR
+        assert pe.pe_launch_count() - launches0 <= 2            # the statistics kernel, plus the zeroing kernel when split
+    mean, sq, sgn = (o.cpu().numpy() for o in outs)
+    assert np.isfinite(mean).all() and np.isfinite(sq).all() and np.isfinite(sgn).all()
+    if B * T * d_in * d_out <= 3e9:
+        st, _ = oracle_on(li)
+    else:
+        rows, cols = boundary_and_random(d_out, 40, 11), boundary_and_random(d_in, 24, 12)
+        st, _ = oracle_on(inputs.gather_columns(li, rows, cols))
+        mean, sq, sgn = (a[np.asarray(rows)][:, np.asarray(cols)] for a in (mean, sq, sgn))
+    assert rel_frob(mean, st.sum_g) <= FROB_TOL
+    assert rel_frob(sq, st.sum_g2) <= FROB_TOL
+    check_sign(sgn, st)
+    # and the same numbers as the two calls it replaces (signs can differ only where an accumulator is within
+    # rounding of zero: the two kernels use different tile widths)
+    m2, s2 = pe.pe_linear_stats(li.X, li.dY, "square")
+    _, g2 = pe.pe_linear_stats(li.X, li.dY, "sign", None, torch.empty((d_out, d_in), device=DEV))
+    torch.cuda.synchronize()
+    assert float((g2 != outs[2]).float().mean()) <= 1e-3
+    assert rel_frob(outs[0].cpu().numpy(), m2.cpu().numpy()) <= 1e-5 and rel_frob(outs[1].cpu().numpy(), s2.cpu().numpy()) <= 1e-5
+
+
+def test_three_statistics_need_all_three_outputs():
+    li = inputs.gaussian_layer(2, 128, 64, 64, seed=1, device=DEV)
+    out = torch.empty((64, 64), device=DEV)
+    lib = pe.load_library()
+    assert lib.pe_linear_stats_all(li.X.data_ptr(), li.dY.data_ptr(), 2, 128, 64, 64, out.data_ptr(), out.data_ptr(), None, None) == 1
 
 
 def test_heavy_tailed_and_heterogeneous_small():
