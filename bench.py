@@ -183,15 +183,12 @@ def run_step(pe, st, i, X=None, dY=None, ev=None):
     dY = li.dY if dY is None else dY
     if ev is not None:
         ev[0].record()
-    pe.pe_linear_stats(X, dY, pe.PHI_SQUARE, st["mean"], st["sq"])
+    pe.pe_linear_stats_all(X, dY, st["mean"], st["sq"], st["sgn"])      # sum G_b, sum G_b^2 and sum sign(G_b) in one pass
     if ev is not None:
         ev[1].record()
-    pe.pe_linear_stats(X, dY, pe.PHI_SIGN, None, st["sgn"])
-    if ev is not None:
-        ev[2].record()
     token_stat(pe, st, X, dY)
     if ev is not None:
-        ev[3].record()
+        ev[2].record()
     pe.microadam_step(st["theta"], st["m"], st["v"], st["mean"], st["sq"], B, step=i + 1, theta_lp=st["theta_lp"], **ADAM)
     pe.microsignsgd_step(st["theta2"], st["m2"], st["sgn"], B, theta_lp=st["theta2_lp"], **SIGN)
 
@@ -230,6 +227,8 @@ def context_numbers(torch, pe, st, li, peaks, dev):
     extra["pe_linear_stats_square_us"] = {"median": med * 1e3, "best": best * 1e3, "tflops_median": flops_one / med / 1e9}
     med_s, best_s = time_each(torch, lambda i: pe.pe_linear_stats(li.X, li.dY, pe.PHI_SIGN, None, st["sgn"]))
     extra["pe_linear_stats_sign_us"] = {"median": med_s * 1e3, "best": best_s * 1e3, "tflops_median": flops_one / med_s / 1e9}
+    med_a3, best_a3 = time_each(torch, lambda i: pe.pe_linear_stats_all(li.X, li.dY, st["mean"], st["sq"], st["sgn"]))
+    extra["pe_linear_stats_all_us"] = {"median": med_a3 * 1e3, "best": best_a3 * 1e3, "tflops_median": flops_one / med_a3 / 1e9}
     med_t, best_t = time_each(torch, lambda i: pe.pe_token_sqstats(li.X, li.dY, st["tok"]))
     extra["pe_token_sqstats_us"] = {"median": med_t * 1e3, "best": best_t * 1e3, "tflops_median": flops_one / med_t / 1e9}
     need = pe.pe_token_sqstats_staged_workspace_bytes(B, T, d_in, d_out)
@@ -244,6 +243,7 @@ def context_numbers(torch, pe, st, li, peaks, dev):
     extra["cublas_wgrad_gemm_us"] = {"median": med_g * 1e3, "best": best_g * 1e3, "tflops_median": flops_one / med_g / 1e9,
                                      "note": "torch.matmul(dY_flat^T, X_flat), bf16 in and out"}
     extra["overhead_vs_gemm"] = med / med_g
+    extra["overhead_all_three_vs_gemm"] = med_a3 / med_g
     big = 1 << 26       # update kernels on a parameter count far larger than L2 (64 Mi parameters)
     bufs = [torch.zeros(big, device=dev) for _ in range(5)]
     lp = torch.empty(big, dtype=torch.bfloat16, device=dev)
@@ -394,7 +394,7 @@ def main():
     B, T, d_in, d_out, nsets = WORKLOADS[name]
     st = make_state(pe, inputs, torch, name, dev)
     flops_one = 2.0 * B * T * d_in * d_out
-    flops_step = 3.0 * flops_one
+    flops_step = 2.0 * flops_one      # two contractions per step: the per-example one (all three statistics) and the per-token one
 
     def barrier():
         torch.cuda.synchronize()
@@ -414,7 +414,7 @@ def main():
         time.sleep(0.25)
     barrier()
     pe.pe_reset_launch_count()
-    kernel_events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    kernel_events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_start.record()
     for i in range(args.steps):
@@ -425,7 +425,7 @@ def main():
     ms_total = t_start.elapsed_time(t_end)
     clocks = sampler.stop() if rank == 0 else None
     # average duration of each statistics call inside the timed steps (events on the launching stream)
-    call_ms = [statistics.fmean(ev[k].elapsed_time(ev[k + 1]) for ev in kernel_events) for k in range(3)]
+    call_ms = [statistics.fmean(ev[k].elapsed_time(ev[k + 1]) for ev in kernel_events) for k in range(2)]
     ms_total = max_over_ranks(torch, dist, ms_total, dev)
     ms_step = ms_total / args.steps
     value = replica_throughput(world, flops_step, ms_step)
@@ -475,11 +475,10 @@ def main():
     # of the timed step.  The per-token kernel contracts tf32 operands: its peak is the measured bf16
     # peak times the nominal tf32 : bf16 ratio (1/2).
     alg_bytes = 2.0 * B * T * (d_in + d_out)
-    specs = [("tc_stats_kernel<square, both outputs>", "square", peaks["bf16_tflops"], "bf16", alg_bytes + 8.0 * d_in * d_out),
-             ("tc_stats_kernel<sign, statistic only>", "sign", peaks["bf16_tflops"], "bf16", alg_bytes + 4.0 * d_in * d_out),
+    specs = [("tc_stats_kernel<mean + square + sign>", "all", peaks["bf16_tflops"], "bf16", alg_bytes + 12.0 * d_in * d_out),
              ("tok_sqstats_kernel", "token", 0.5 * peaks["bf16_tflops"], "tf32", alg_bytes + 4.0 * d_in * d_out)]
     if st["tok_ws"] is not None:      # two-pass form: three streaming kernels around the half contraction
-        specs[2] = ("pe_token_sqstats_staged: column_max + square_to_half + tc_stats_kernel<identity, half> + unscale", "token_staged",
+        specs[1] = ("pe_token_sqstats_staged: column_max + square_to_half + tc_stats_kernel<identity, half> + unscale", "token_staged",
                     peaks["bf16_tflops"], "f16", alg_bytes + 4.0 * d_in * d_out)
     by_kernel = []
     for (kname, key, peak, op_dtype, nbytes), ms in zip(specs, call_ms):
@@ -510,7 +509,7 @@ def main():
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": name, "B": B, "T": T, "d_in": d_in, "d_out": d_out,
-                   "step": "pe_linear_stats(square)+pe_linear_stats(sign)+" + ("pe_token_sqstats_staged" if st["tok_ws"] is not None else "pe_token_sqstats")
+                   "step": "pe_linear_stats_all(mean,square,sign)+" + ("pe_token_sqstats_staged" if st["tok_ws"] is not None else "pe_token_sqstats")
                            + "+microadam_step+microsignsgd_step",
                    "flops_per_step": flops_step, "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": f"{nsets} rotating input sets, {nsets * 2 * B * T * (d_in + d_out) / 1e6:.0f} MB in all (> 126 MB L2)"

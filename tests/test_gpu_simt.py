@@ -71,3 +71,16 @@ def test_only_one_output_requested():
     pe.pe_linear_stats_f32(li.X, li.dY, "square", mean, None)
     torch.cuda.synchronize()
     assert np.array_equal(stat.cpu().numpy(), stat_ref) and np.array_equal(mean.cpu().numpy(), mean_ref)
+
+
+def test_three_statistics_call_on_a_shape_the_tensor_cores_do_not_take():
+    """pe_linear_stats_all falls back to the two separate calls (here both on the SIMT kernel: widths that are
+    not multiples of 8)."""
+    from parity_util import FROB_TOL, check_sign, oracle_on, rel_frob
+    li = inputs.gaussian_layer(6, 40, 36, 20, seed=1500, device=DEV)
+    mean, sq, sgn = pe.pe_linear_stats_all(li.X, li.dY)
+    torch.cuda.synchronize()
+    assert pe.pe_last_path() == pe.PATH_SIMT
+    st, _ = oracle_on(li)
+    assert rel_frob(mean.cpu().numpy(), st.sum_g) <= FROB_TOL and rel_frob(sq.cpu().numpy(), st.sum_g2) <= FROB_TOL
+    check_sign(sgn.cpu().numpy(), st)

@@ -151,7 +151,7 @@ def test_staged_token_stat_keeps_every_column_accurate_over_a_wide_range_of_magn
     (1, 1000, 256, 128, True),     # single example
     (64, 256, 512, 2048, True),    # the benchmark layer, sampled below
     (9, 16, 320, 192, False),      # short sequences: served by the two separate calls
-    (6, 40, 36, 20, False),        # widths the tensor-core path does not take
+    (21, 64, 136, 520, False),     # exactly one short stage per example: still the two calls
 ])
 def test_three_statistics_in_one_pass(B, T, d_in, d_out, tensor_one_pass):
     """pe_linear_stats_all: sum_b G_b, sum_b G_b^2 and sum_b sign(G_b) from one pass over the examples, against
