@@ -129,6 +129,18 @@ __device__ __forceinline__ float phi_apply(float g) {
   return g;
 }
 
+// -1 if the fp32 value with these bits is > 0 (< 0), else 0; one instruction each.
+__device__ __forceinline__ int set_gt_zero(uint32_t bits) {
+  int d;
+  asm("set.gt.s32.f32 %0, %1, 0f00000000;" : "=r"(d) : "f"(__uint_as_float(bits)));
+  return d;
+}
+__device__ __forceinline__ int set_lt_zero(uint32_t bits) {
+  int d;
+  asm("set.lt.s32.f32 %0, %1, 0f00000000;" : "=r"(d) : "f"(__uint_as_float(bits)));
+  return d;
+}
+
 // Walks the slots of the operand ring in the order the producers fill them.  With two issuers the
 // examples are taken two at a time and their stages interleaved: slot 2*kc of a pair of examples
 // belongs to its first example (issuer 0, even slots), slot 2*kc+1 to its second (issuer 1, odd
@@ -314,8 +326,9 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     constexpr int N_STAT = (PHI != 0) ? COLS : 1;
     constexpr int N_MEAN = KEEP_MEAN ? COLS : 1;
     float acc_stat[N_STAT], acc_mean[N_MEAN];
-    // TRIPLE: per column, sum_b (sign(G_b) + 1), a count in [0, 2 nb] that fits 16 bits; two columns per
-    // register, so the third statistic costs 32 registers instead of 64.  sum_b sign = count - nb.
+    // TRIPLE: sum_b sign(G_b) of two neighbouring columns in one register, as signed 16-bit halves of
+    // one 32-bit two's-complement sum (low + 65536 * high; |sum| <= nb <= 32767 per half, so both are
+    // recovered exactly at the end).  The third statistic costs 32 registers instead of 64.
     constexpr int N_CNT = TRIPLE ? COLS / 2 : 1;
     uint32_t acc_cnt[N_CNT];
 #pragma unroll
@@ -390,11 +403,10 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 f32x2_unpack(s2, acc_stat[c * 32 + j], acc_stat[c * 32 + j + 1]);
               }
               if (TRIPLE) {
-                const float g0 = __uint_as_float(r[j]), g1 = __uint_as_float(r[j + 1]);
-                // sign + 1 in {0, 1, 2}; +0 and -0 both give 1
-                const uint32_t c0 = 1u + (g0 > 0.f ? 1u : 0u) - (g0 < 0.f ? 1u : 0u);
-                const uint32_t c1 = 1u + (g1 > 0.f ? 1u : 0u) - (g1 < 0.f ? 1u : 0u);
-                acc_cnt[(c * 32 + j) >> 1] += c0 + (c1 << 16);
+                // set.xx.s32.f32 gives -1 / 0, so sign(g) = (g < 0 ? -1 : 0) - (g > 0 ? -1 : 0); +-0 give 0
+                const int s0 = set_lt_zero(r[j]) - set_gt_zero(r[j]);
+                const int s1 = set_lt_zero(r[j + 1]) - set_gt_zero(r[j + 1]);
+                acc_cnt[(c * 32 + j) >> 1] += (uint32_t)(s0 + s1 * 65536);
               }
             }
           }
@@ -472,12 +484,16 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         if (p.out_sign) {
           if (lane == 0) bulk_wait_read_all();
           __syncwarp();
-          const float nbf = (float)nb;
 #pragma unroll
           for (int c = 0; c < PANELS; ++c) {
             float v[32];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = (float)((acc_cnt[(c * 32 + j) >> 1] >> (16 * (j & 1))) & 0xFFFFu) - nbf;
+            for (int j = 0; j < 32; j += 2) {
+              const int both = (int)acc_cnt[(c * 32 + j) >> 1];
+              const int low = (int)(short)(both & 0xFFFF);
+              v[j] = (float)low;
+              v[j + 1] = (float)((both - low) >> 16);
+            }
             put_panel(stage_base + c * 4096, v);
           }
           send(&tmap_sign, stage_base);
