@@ -76,6 +76,18 @@ pe_status_t pe_linear_stats_f32(const float* X, const float* dY, int B, int T, i
                                 pe_phi_t phi, float* out_mean, float* out_stat, pe_stream_t stream);
 
 /*
+ * pe_linear_stats for gradient accumulation over micro-batches: the statistics of this call's B
+ * examples are ADDED to what out_mean / out_stat already hold (both sums of Eq. (2) are additive over
+ * examples, so running this over the micro-batches of a batch, after zeroing the outputs once, gives
+ * the statistics of the whole batch; the caller divides by the total number of examples).  Same
+ * arguments and rules otherwise; an empty micro-batch leaves the outputs untouched.  Partial results
+ * are added with fp32 reduce operations, so the summation order over micro-batches is the call order
+ * but within a call it is unspecified.
+ */
+pe_status_t pe_linear_stats_accumulate(const void* X, const void* dY, int B, int T, int d_in, int d_out,
+                                       pe_phi_t phi, float* out_mean, float* out_stat, pe_stream_t stream);
+
+/*
  * The three statistics of pe_linear_stats in one pass over the examples (Eq. (2) with phi = identity,
  * square and sign at once; Sections 2.1 and 3.1):
  *     out_mean = sum_b G_b,   out_square = sum_b G_b^2,   out_sign = sum_b sign(G_b),   G_b = dY_b^T X_b.

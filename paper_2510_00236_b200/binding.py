@@ -17,7 +17,7 @@ __all__ = [
     "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_staged", "pe_token_sqstats_staged_workspace_bytes",
     "microadam_step", "microsignsgd_step", "pe_status_string", "pe_get_async_status", "pe_set_path", "pe_last_path",
     "pe_launch_count", "pe_reset_launch_count", "pe_token_sqstats_static", "STATIC_SCRATCH_BYTES",
-    "microadam_family_step", "ADAM_VARIANTS", "pe_linear_stats_all",
+    "microadam_family_step", "ADAM_VARIANTS", "pe_linear_stats_all", "pe_linear_stats_accumulate",
 ]
 
 PHI_IDENTITY, PHI_SQUARE, PHI_SIGN = 0, 1, 2
@@ -29,7 +29,7 @@ EXPORTED_SYMBOLS = [
     "pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_staged",
     "pe_token_sqstats_staged_workspace_bytes", "microadam_step", "microsignsgd_step", "pe_status_string",
     "pe_get_async_status", "pe_set_path", "pe_last_path", "pe_launch_count", "pe_reset_launch_count",
-    "pe_token_sqstats_static", "microadam_family_step", "pe_linear_stats_all",
+    "pe_token_sqstats_static", "microadam_family_step", "pe_linear_stats_all", "pe_linear_stats_accumulate",
 ]
 ADAM_VARIANTS = {"adam": 0, "microadam": 1, "microadam_var": 2, "microadam_msq": 3}      # pe_adam_variant_t
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024      # PE_STATIC_SCRATCH_BYTES of pestats.h
@@ -63,6 +63,7 @@ def load_library() -> ctypes.CDLL:
     lib.pe_linear_stats.argtypes = [vp, vp, i, i, i, i, i, vp, vp, vp]
     lib.pe_linear_stats_f32.argtypes = [vp, vp, i, i, i, i, i, vp, vp, vp]
     lib.pe_linear_stats_all.argtypes = [vp, vp, i, i, i, i, vp, vp, vp, vp]
+    lib.pe_linear_stats_accumulate.argtypes = [vp, vp, i, i, i, i, i, vp, vp, vp]
     lib.pe_token_sqstats.argtypes = [vp, vp, i, i, i, i, vp, vp]
     lib.pe_token_sqstats_staged.argtypes = [vp, vp, i, i, i, i, vp, vp, sz, vp]
     lib.pe_token_sqstats_f32.argtypes = [vp, vp, i, i, i, i, vp, vp]
@@ -81,7 +82,7 @@ def load_library() -> ctypes.CDLL:
     lib.pe_launch_count.restype = ll
     lib.pe_reset_launch_count.argtypes = []
     lib.pe_reset_launch_count.restype = None
-    for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_linear_stats_all", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_static",
+    for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_static",
                  "pe_token_sqstats_staged",
                  "microadam_step", "microadam_family_step", "microsignsgd_step", "pe_get_async_status", "pe_set_path", "pe_last_path"):
         getattr(lib, name).restype = i
@@ -143,6 +144,17 @@ def pe_linear_stats(X, dY, phi, out_mean=None, out_stat=None):
     _out_check("out_stat", out_stat, d_out, d_in)
     with _dev_ctx(X):
         _check("pe_linear_stats", load_library().pe_linear_stats(
+            X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, _phi(phi), _ptr(out_mean), _ptr(out_stat), _stream(X)))
+    return out_mean, out_stat
+
+
+def pe_linear_stats_accumulate(X, dY, phi, out_mean, out_stat):
+    """Adds this micro-batch's sum_b G_b / sum_b phi(G_b) to out_mean / out_stat (either may be None)."""
+    B, T, d_in, d_out = _io_check(X, dY, torch.bfloat16)
+    _out_check("out_mean", out_mean, d_out, d_in)
+    _out_check("out_stat", out_stat, d_out, d_in)
+    with _dev_ctx(X):
+        _check("pe_linear_stats_accumulate", load_library().pe_linear_stats_accumulate(
             X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, _phi(phi), _ptr(out_mean), _ptr(out_stat), _stream(X)))
     return out_mean, out_stat
 

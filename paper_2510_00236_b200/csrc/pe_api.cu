@@ -191,6 +191,7 @@ static pe_status_t launch_pair_kernel(Kernel kernel, dim3 grid, int smem, cudaSt
 template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT)>
 static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& mm,
                                   const CUtensorMap& ms, const CUtensorMap& msgn, const TcParams& p, dim3 grid, cudaStream_t st) {
+  const bool after_zeroing = p.nsplit > 1 && !p.accumulate;
   constexpr int smem = TcOperand<TF32, NT, BKT>::SMEM_BYTES;
   if (!di->tc_attr_set[slot]) {
     if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
@@ -199,7 +200,7 @@ static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& m
     }
     di->tc_attr_set[slot] = true;
   }
-  return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT>, grid, smem, st, p.nsplit > 1, mx, my, mm, ms, msgn, p);
+  return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT>, grid, smem, st, after_zeroing, mx, my, mm, ms, msgn, p);
 }
 
 // Tensor-core launch.  per_example = 0 runs the plain contraction over all B*T rows (its result goes
@@ -207,7 +208,7 @@ static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& m
 // pair tile is 256 x 128 (two running sums per thread); with only out_stat it is 256 x 256.
 static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int B, int T, int d_in, int d_out, int phi,
                              int per_example, float* out_mean, float* out_stat, cudaStream_t st, bool half_ops = false,
-                             float* out_sign = nullptr) {
+                             float* out_sign = nullptr, bool accumulate = false) {
   const bool triple = out_sign != nullptr;       // mean + square + sign in one pass (phi = square, all three outputs given)
   const bool both = per_example && out_mean && out_stat;
   // Both outputs: sum_b G_b in tensor memory beside a 256-wide accumulator, unless the sequences are
@@ -233,12 +234,13 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   if ((long long)tiles_n * pairs_m > (1ll << 29)) return PE_ERR_DIM;
   int ns = choose_nsplit((long long)tiles_n * pairs_m, B, T, di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 16);
   if (triple && (B + ns - 1) / ns > TC_SIGN_COUNT_MAX) ns = (B + TC_SIGN_COUNT_MAX - 1) / TC_SIGN_COUNT_MAX;   // 16-bit sign counters
-  if (ns > 1) {
+  if (ns > 1 && !accumulate) {
     rc = zero_for_split(di, out_mean, out_stat, (size_t)d_in * d_out, st, out_sign);
     if (rc != PE_OK) return rc;
   }
   TcParams p;
   p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = per_example; p.half_operands = half_ops ? 1 : 0;
+  p.accumulate = accumulate ? 1 : 0;
   p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
   p.out_mean = out_mean; p.out_stat = out_stat; p.out_sign = out_sign; p.dev_status = di->status_ptr;
   dim3 grid(2 * pairs_m * tiles_n, 1, ns);
@@ -262,15 +264,15 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
 
 template <typename TIn, int MODE>
 static pe_status_t launch_simt(DeviceInfo* di, const TIn* X, const TIn* dY, int B, int T, int d_in, int d_out, int phi,
-                               float* out_mean, float* out_stat, cudaStream_t st) {
+                               float* out_mean, float* out_stat, cudaStream_t st, bool accumulate = false) {
   const int tx = (d_in + SIMT_TILE - 1) / SIMT_TILE, ty = (d_out + SIMT_TILE - 1) / SIMT_TILE;
   if (ty > 65535) return PE_ERR_DIM;
   const int ns = choose_nsplit((long long)tx * ty, B, T, di->sm_count * 3, 64);
-  if (ns > 1) {
+  if (ns > 1 && !accumulate) {
     pe_status_t rc = zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
     if (rc != PE_OK) return rc;
   }
-  simt_stats_kernel<TIn, MODE><<<dim3(tx, ty, ns), SIMT_THREADS, 0, st>>>(X, dY, B, T, d_in, d_out, phi, out_mean, out_stat);
+  simt_stats_kernel<TIn, MODE><<<dim3(tx, ty, ns), SIMT_THREADS, 0, st>>>(X, dY, B, T, d_in, d_out, phi, out_mean, out_stat, accumulate ? 1 : 0);
   return check_launch();
 }
 
@@ -288,14 +290,14 @@ static pe_status_t validate_stats(const void* X, const void* dY, int B, int T, i
 
 template <typename TIn>
 static pe_status_t linear_stats_impl(const TIn* X, const TIn* dY, int B, int T, int d_in, int d_out, pe_phi_t phi,
-                                     float* out_mean, float* out_stat, cudaStream_t st, bool allow_tc) {
+                                     float* out_mean, float* out_stat, cudaStream_t st, bool allow_tc, bool accumulate = false) {
   pe_status_t rc = validate_stats(X, dY, B, T, d_in, d_out, out_mean, out_stat, true, allow_tc ? 16 : 4);
   if (rc != PE_OK) return rc;
   if (phi != PE_PHI_IDENTITY && phi != PE_PHI_SQUARE && phi != PE_PHI_SIGN) return PE_ERR_PHI;
   DeviceInfo* di = nullptr;
   rc = device_info(&di);
   if (rc != PE_OK) return rc;
-  if (B == 0 || T == 0) return zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
+  if (B == 0 || T == 0) return accumulate ? PE_OK : zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
   const int forced = g_path.load();
   const bool tc_ok = allow_tc && tc_shape_ok(B, T, d_in, d_out);
   if ((forced == PE_PATH_TENSOR || forced == PE_PATH_TENSOR_NARROW) && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
@@ -305,7 +307,9 @@ static pe_status_t linear_stats_impl(const TIn* X, const TIn* dY, int B, int T, 
       if (phi == PE_PHI_IDENTITY) {
         // phi = identity: both outputs are the plain contraction over all B*T rows.
         float* first = out_mean ? out_mean : out_stat;
-        rc = launch_tc(di, X, dY, B, T, d_in, d_out, phi, 0, first, nullptr, st);
+        rc = launch_tc(di, X, dY, B, T, d_in, d_out, phi, 0, first, nullptr, st, false, nullptr, accumulate);
+        if (rc == PE_OK && out_mean && out_stat && accumulate)      // a copy would overwrite: contract once more into the second
+          return launch_tc(di, X, dY, B, T, d_in, d_out, phi, 0, out_stat, nullptr, st, false, nullptr, true);
         if (rc == PE_OK && out_mean && out_stat) {
           if (cudaMemcpyAsync(out_stat, out_mean, (size_t)d_in * d_out * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
             cudaGetLastError();
@@ -315,12 +319,12 @@ static pe_status_t linear_stats_impl(const TIn* X, const TIn* dY, int B, int T, 
         return rc;
       }
       if (!out_stat)      // only sum_b G_b wanted: the plain contraction
-        return launch_tc(di, X, dY, B, T, d_in, d_out, phi, 0, out_mean, nullptr, st);
-      return launch_tc(di, X, dY, B, T, d_in, d_out, phi, 1, out_mean, out_stat, st);
+        return launch_tc(di, X, dY, B, T, d_in, d_out, phi, 0, out_mean, nullptr, st, false, nullptr, accumulate);
+      return launch_tc(di, X, dY, B, T, d_in, d_out, phi, 1, out_mean, out_stat, st, false, nullptr, accumulate);
     }
   }
   g_last_path.store(PE_PATH_SIMT);
-  return launch_simt<TIn, MODE_STATS>(di, X, dY, B, T, d_in, d_out, (int)phi, out_mean, out_stat, st);
+  return launch_simt<TIn, MODE_STATS>(di, X, dY, B, T, d_in, d_out, (int)phi, out_mean, out_stat, st, accumulate);
 }
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -381,6 +385,12 @@ pe_status_t pe_linear_stats(const void* X, const void* dY, int B, int T, int d_i
                             float* out_mean, float* out_stat, pe_stream_t stream) {
   return linear_stats_impl<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T,
                                           d_in, d_out, phi, out_mean, out_stat, reinterpret_cast<cudaStream_t>(stream), true);
+}
+
+pe_status_t pe_linear_stats_accumulate(const void* X, const void* dY, int B, int T, int d_in, int d_out, pe_phi_t phi,
+                                       float* out_mean, float* out_stat, pe_stream_t stream) {
+  return linear_stats_impl<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T,
+                                          d_in, d_out, phi, out_mean, out_stat, reinterpret_cast<cudaStream_t>(stream), true, true);
 }
 
 pe_status_t pe_linear_stats_all(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_mean,

@@ -27,11 +27,12 @@ __device__ __forceinline__ float apply_phi(float g, int phi) {
 // MODE_TOKEN: out_stat = sum_{b,t} dY^2 X^2; operands are squared as they are staged and the
 //             accumulator is never reset between examples             (Section 2.3, per-token form)
 // gridDim = (ceil(d_in/64), ceil(d_out/64), nsplit); block z handles examples [z*B/nsplit, (z+1)*B/nsplit).
-// With nsplit > 1 the outputs must be zero on entry and partial sums are added atomically.
+// With nsplit > 1 the outputs must be zero on entry and partial sums are added atomically; with
+// accumulate != 0 the results are added to whatever the outputs hold.
 template <typename TIn, int MODE>
 __global__ void __launch_bounds__(SIMT_THREADS)
 simt_stats_kernel(const TIn* __restrict__ X, const TIn* __restrict__ dY, int B, int T, int d_in, int d_out,
-                  int phi, float* __restrict__ out_mean, float* __restrict__ out_stat) {
+                  int phi, float* __restrict__ out_mean, float* __restrict__ out_stat, int accumulate) {
   __shared__ float sY[SIMT_TK][SIMT_TILE];
   __shared__ float sX[SIMT_TK][SIMT_TILE];
 
@@ -108,7 +109,7 @@ simt_stats_kernel(const TIn* __restrict__ X, const TIn* __restrict__ dY, int B, 
       if (i >= d_in) continue;
       size_t at = (size_t)o * d_in + i;
       float vs = (MODE == MODE_TOKEN) ? g[r][c] : acc_stat[r][c];
-      if (nsplit == 1) {
+      if (nsplit == 1 && !accumulate) {
         if (out_stat) out_stat[at] = vs;
         if (MODE == MODE_STATS && out_mean) out_mean[at] = acc_mean[r][c];
       } else {

@@ -99,6 +99,7 @@ struct TcParams {
   int per_example;     // 1: reset the accumulator for every example and apply phi (statistics)
                        // 0: one accumulation over the whole slice (plain contraction, phi = identity)
   int half_operands;   // 16-bit operands are IEEE half instead of bf16 (the staged per-token statistic)
+  int accumulate;      // add the results to what the outputs hold (no zeroing kernel runs before this one)
   float* out_mean;     // may be NULL; written through tmap_mean
   float* out_stat;     // may be NULL; written through tmap_stat
   float* out_sign;     // MEAN_REGS_SIGN only: sum_b sign(G_b), written through tmap_sign
@@ -437,10 +438,10 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         fence_async_smem();
         __syncwarp();
         if (lane == 0 && row0 < p.d_out) {
-          if (p.nsplit > 1) griddep_wait();       // the kernel that zeroes the outputs may still be running
+          if (p.nsplit > 1 && !p.accumulate) griddep_wait();       // the kernel that zeroes the outputs may still be running
           for (int c = 0; c < PANELS; ++c) {
             if (col0 + c * 32 < p.d_in) {
-              if (p.nsplit == 1) tma_store_2d<false>(tm, first_panel + c * 4096, col0 + c * 32, row0);
+              if (p.nsplit == 1 && !p.accumulate) tma_store_2d<false>(tm, first_panel + c * 4096, col0 + c * 32, row0);
               else tma_store_2d<true>(tm, first_panel + c * 4096, col0 + c * 32, row0);
             }
           }

@@ -70,7 +70,8 @@ def check_sign(gpu_sign: np.ndarray, st: oracle.LinearStats) -> int:
     return int((diff > 0).sum())
 
 
-def check_all(li_full: inputs.LayerInputs, rows=None, cols=None, phis=("square", "sign"), token=True, tol=FROB_TOL):
+def check_all(li_full: inputs.LayerInputs, rows=None, cols=None, phis=("square", "sign"), token=True, tol=FROB_TOL,
+              bench_calls=False):
     """Full comparison when rows/cols are None, otherwise on the sampled output rows x cols: the GPU runs
     the full layer, the oracle the column-gathered sub-layer (each output entry depends on one column
     of dY and one of X only)."""
@@ -100,6 +101,23 @@ def check_all(li_full: inputs.LayerInputs, rows=None, cols=None, phis=("square",
         e = rel_frob(t, tok)
         assert e <= tol, f"per-token statistic: rel. Frobenius error {e:.3e} > {tol}"
         report["token_err"] = e
+    if bench_calls:
+        # the calls the benchmark step makes: all three statistics in one pass, the two-pass per-token statistic
+        dev = li_full.X.device
+        B, T, d_in, d_out = li_full.shape
+        outs = [torch.full((d_out, d_in), float("nan"), device=dev) for _ in range(3)]
+        pe.pe_linear_stats_all(li_full.X, li_full.dY, *outs)
+        torch.cuda.synchronize()
+        mean, sq, sgn = (pick(o.cpu().numpy()) for o in outs)
+        del outs
+        assert np.isfinite(mean).all() and np.isfinite(sq).all() and np.isfinite(sgn).all()
+        report["one_pass_mean_err"], report["one_pass_square_err"] = rel_frob(mean, st.sum_g), rel_frob(sq, st.sum_g2)
+        assert report["one_pass_mean_err"] <= tol and report["one_pass_square_err"] <= tol
+        report["one_pass_sign_disagreements"] = check_sign(sgn, st)
+        t = pick(pe.pe_token_sqstats_staged(li_full.X, li_full.dY).cpu().numpy())
+        assert np.isfinite(t).all()
+        report["token_two_pass_err"] = rel_frob(t, tok)
+        assert report["token_two_pass_err"] <= tol
     status, detail = pe.pe_get_async_status(li_full.X.device)
     assert status == 0, f"device status {status} detail {detail}"
     return report

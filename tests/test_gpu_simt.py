@@ -84,3 +84,16 @@ def test_three_statistics_call_on_a_shape_the_tensor_cores_do_not_take():
     st, _ = oracle_on(li)
     assert rel_frob(mean.cpu().numpy(), st.sum_g) <= FROB_TOL and rel_frob(sq.cpu().numpy(), st.sum_g2) <= FROB_TOL
     check_sign(sgn.cpu().numpy(), st)
+
+
+def test_accumulate_on_the_simt_path():
+    from parity_util import FROB_TOL, oracle_on, rel_frob
+    li = inputs.gaussian_layer(7, 33, 36, 20, seed=1700, device=DEV)
+    mean = torch.zeros((20, 36), device=DEV)
+    stat = torch.zeros((20, 36), device=DEV)
+    for lo, hi in ((0, 3), (3, 7)):
+        pe.pe_linear_stats_accumulate(li.X[lo:hi].contiguous(), li.dY[lo:hi].contiguous(), "square", mean, stat)
+    torch.cuda.synchronize()
+    assert pe.pe_last_path() == pe.PATH_SIMT
+    st, _ = oracle_on(li)
+    assert rel_frob(mean.cpu().numpy(), st.sum_g) <= FROB_TOL and rel_frob(stat.cpu().numpy(), st.sum_g2) <= FROB_TOL

@@ -186,6 +186,48 @@ def test_three_statistics_in_one_pass(B, T, d_in, d_out, tensor_one_pass):
     assert rel_frob(outs[0].cpu().numpy(), m2.cpu().numpy()) <= 1e-5 and rel_frob(outs[1].cpu().numpy(), s2.cpu().numpy()) <= 1e-5
 
 
+@pytest.mark.parametrize("B,T,d_in,d_out,phi", [(11, 200, 136, 264, "square"), (70, 96, 8, 8, "sign"), (6, 4100, 136, 264, "square"),
+                                                  (9, 16, 320, 192, "sign"), (5, 300, 264, 136, "identity")])
+def test_accumulating_over_micro_batches_gives_the_statistics_of_the_batch(B, T, d_in, d_out, phi):
+    """pe_linear_stats_accumulate over three unequal micro-batches (one of them empty) into outputs zeroed once,
+    against the oracle on the whole batch."""
+    from parity_util import FROB_TOL, check_sign, oracle_on, rel_frob
+    li = inputs.gaussian_layer(B, T, d_in, d_out, seed=1600 + B, device=DEV)
+    mean = torch.zeros((d_out, d_in), device=DEV)
+    stat = torch.zeros((d_out, d_in), device=DEV)
+    cuts = [0, B // 3, B // 3, B - 2, B]                     # micro-batches of B//3, 0, B-2-B//3 and 2 examples
+    for lo, hi in zip(cuts[:-1], cuts[1:]):
+        pe.pe_linear_stats_accumulate(li.X[lo:hi].contiguous(), li.dY[lo:hi].contiguous(), phi, mean, stat)
+    torch.cuda.synchronize()
+    assert pe.pe_get_async_status(DEV) == (0, 0)
+    st, _ = oracle_on(li)
+    assert rel_frob(mean.cpu().numpy(), st.sum_g) <= FROB_TOL
+    if phi == "square":
+        assert rel_frob(stat.cpu().numpy(), st.sum_g2) <= FROB_TOL
+    elif phi == "sign":
+        check_sign(stat.cpu().numpy(), st)
+    else:
+        assert rel_frob(stat.cpu().numpy(), st.sum_g) <= FROB_TOL
+    # a single output works too, and what is already there is kept
+    only = torch.full((d_out, d_in), 3.0, device=DEV)
+    pe.pe_linear_stats_accumulate(li.X, li.dY, phi, None, only)
+    torch.cuda.synchronize()
+    ref = {"square": st.sum_g2, "sign": st.sum_sign, "identity": st.sum_g}[phi]
+    if phi == "sign":
+        check_sign(only.cpu().numpy() - 3.0, st)
+    else:
+        assert rel_frob(only.cpu().numpy().astype(np.float64) - 3.0, ref) <= FROB_TOL + 1e-4
+
+
+def test_three_statistics_of_an_empty_batch_are_zero():
+    outs = [torch.full((72, 64), float("nan"), device=DEV) for _ in range(3)]
+    X = torch.empty((0, 128, 64), dtype=torch.bfloat16, device=DEV)
+    dY = torch.empty((0, 128, 72), dtype=torch.bfloat16, device=DEV)
+    pe.pe_linear_stats_all(X, dY, *outs)
+    torch.cuda.synchronize()
+    assert all(bool((o == 0).all()) for o in outs)
+
+
 def test_three_statistics_need_all_three_outputs():
     li = inputs.gaussian_layer(2, 128, 64, 64, seed=1, device=DEV)
     out = torch.empty((64, 64), device=DEV)
@@ -209,7 +251,7 @@ def test_config2_full_size_sampled_outputs():
     li = inputs.config2(DEV)
     rows = boundary_and_random(2048, 40, 1)
     cols = boundary_and_random(512, 32, 2)
-    rep = check_all(li, rows, cols)
+    rep = check_all(li, rows, cols, bench_calls=True)
     assert pe.pe_last_path() == pe.PATH_TENSOR
     print("config2", rep)
 
@@ -218,7 +260,7 @@ def test_config4_full_size_sampled_outputs():
     li = inputs.config4(DEV)
     rows = boundary_and_random(8192, 24, 3)
     cols = boundary_and_random(2048, 24, 4)
-    rep = check_all(li, rows, cols)
+    rep = check_all(li, rows, cols, bench_calls=True)
     print("config4", rep)
     del li
     torch.cuda.empty_cache()
