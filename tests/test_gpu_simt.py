@@ -92,7 +92,7 @@ def test_accumulate_on_the_simt_path():
     mean = torch.zeros((20, 36), device=DEV)
     stat = torch.zeros((20, 36), device=DEV)
     for lo, hi in ((0, 3), (3, 7)):
-        pe.pe_linear_stats_accumulate(li.X[lo:hi].contiguous(), li.dY[lo:hi].contiguous(), "square", mean, stat)
+        pe.pe_linear_stats_accumulate(li.X[lo:hi].clone(), li.dY[lo:hi].clone(), "square", mean, stat)
     torch.cuda.synchronize()
     assert pe.pe_last_path() == pe.PATH_SIMT
     st, _ = oracle_on(li)

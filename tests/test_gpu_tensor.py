@@ -197,7 +197,7 @@ def test_accumulating_over_micro_batches_gives_the_statistics_of_the_batch(B, T,
     stat = torch.zeros((d_out, d_in), device=DEV)
     cuts = [0, B // 3, B // 3, B - 2, B]                     # micro-batches of B//3, 0, B-2-B//3 and 2 examples
     for lo, hi in zip(cuts[:-1], cuts[1:]):
-        pe.pe_linear_stats_accumulate(li.X[lo:hi].contiguous(), li.dY[lo:hi].contiguous(), phi, mean, stat)
+        pe.pe_linear_stats_accumulate(li.X[lo:hi].clone(), li.dY[lo:hi].clone(), phi, mean, stat)
     torch.cuda.synchronize()
     assert pe.pe_get_async_status(DEV) == (0, 0)
     st, _ = oracle_on(li)
