@@ -51,6 +51,11 @@ def _load():
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
             ctypes.c_int, c_double_p,
         ]
+        lib.oracle_example_sqnorms.restype = ctypes.c_int
+        lib.oracle_example_sqnorms.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+            ctypes.c_int, c_double_p,
+        ]
         lib.oracle_microadam_step.restype = ctypes.c_int
         lib.oracle_microadam_step.argtypes = [
             c_double_p, c_double_p, c_double_p, c_double_p, c_double_p, ctypes.c_longlong, ctypes.c_int,
@@ -128,6 +133,16 @@ def token_sqstats(X: np.ndarray, dY: np.ndarray) -> np.ndarray:
     rc = _load().oracle_token_sqstats(X.ctypes.data, dY.ctypes.data, is_bf16, B, T, d_in, d_out, _dp(out))
     if rc != 0:
         raise RuntimeError("oracle_token_sqstats failed")
+    return out
+
+
+def example_sqnorms(X: np.ndarray, dY: np.ndarray) -> np.ndarray:
+    """Per-example squared gradient norms N_b = ||dY_b^T X_b||_F^2 (Section 2.3), shape [B]."""
+    X, dY, is_bf16, B, T, d_in, d_out = _check_inputs(X, dY)
+    out = np.zeros((B,), np.float64)
+    rc = _load().oracle_example_sqnorms(X.ctypes.data, dY.ctypes.data, is_bf16, B, T, d_in, d_out, _dp(out))
+    if rc != 0:
+        raise RuntimeError("oracle_example_sqnorms failed")
     return out
 
 

@@ -109,6 +109,40 @@ int oracle_linear_stats(const void* X, const void* dY, int is_bf16, int B, int T
 }
 
 /*
+ * Per-example squared gradient norms (Section 2.3: the quantity N_b = ||grad_W f(theta; x_b)||_2^2 of the
+ * "ghost clipping" remark; what a clipping phi of Section 2.1 needs):
+ *     N_b = sum_{o,i} G_b[o,i]^2,     G_b[o,i] = sum_t dY[b,t,o] * X[b,t,i],
+ * computed the long way: the whole G_b is formed, then its entries are squared and summed.
+ */
+int oracle_example_sqnorms(const void* X, const void* dY, int is_bf16, int B, int T, int d_in, int d_out,
+                           double* norms) {
+  if (!X || !dY || !norms || B < 0 || T < 0 || d_in <= 0 || d_out <= 0) return 1;
+  double* row = (double*)malloc(sizeof(double) * (size_t)d_out);
+  double* xb = (double*)malloc(sizeof(double) * (size_t)((long long)(T > 0 ? T : 1) * d_in));
+  double* yb = (double*)malloc(sizeof(double) * (size_t)((long long)(T > 0 ? T : 1) * d_out));
+  if (!row || !xb || !yb) { free(row); free(xb); free(yb); return 1; }
+  for (int b = 0; b < B; ++b) {
+    widen_rows(X, is_bf16, (long long)b * T, T, d_in, xb);
+    widen_rows(dY, is_bf16, (long long)b * T, T, d_out, yb);
+#pragma omp parallel for schedule(static)
+    for (int o = 0; o < d_out; ++o) {
+      double acc = 0.0;
+      for (int i = 0; i < d_in; ++i) {
+        double g = 0.0;
+        for (int t = 0; t < T; ++t) g += yb[(long long)t * d_out + o] * xb[(long long)t * d_in + i];
+        acc += g * g;
+      }
+      row[o] = acc;
+    }
+    double nb = 0.0;
+    for (int o = 0; o < d_out; ++o) nb += row[o];
+    norms[b] = nb;
+  }
+  free(row); free(xb); free(yb);
+  return 0;
+}
+
+/*
  * Per-token second moment (Section 2.3, the "per-token" alternative):
  *     S'[o,i] = sum_{b,t} dY[b,t,o]^2 * X[b,t,i]^2 ,
  * one term per (example, token) row; B and T only enter as the row count.

@@ -229,6 +229,33 @@ def test_mean_sign_with_planted_mean_follows_2p_minus_1():
     assert abs(st.sum_sign.mean() / B - (2 * p - 1)) < 5 * se
 
 
+def test_example_norms_equal_the_gram_matrix_contraction_and_close_the_sum_of_squares():
+    """Per-example squared norms against three things the mathematics fixes: the "ghost" identity
+    ||dY_b^T X_b||_F^2 = sum_{t,t'} (X_b X_b^T)[t,t'] (dY_b dY_b^T)[t,t'] (Section 2.3's remark on norms from
+    Gram matrices; numpy's matmul, a different contraction order), the rank-one closed form ||x||^2 ||dy||^2 at
+    T = 1, and sum_b N_b = the sum of all entries of sum_b G_b^2."""
+    rng = np.random.default_rng(41)
+    B, T, d_in, d_out = 5, 7, 9, 6
+    X = rng.standard_normal((B, T, d_in)).astype(np.float32)
+    dY = rng.standard_normal((B, T, d_out)).astype(np.float32)
+    n = oracle.example_sqnorms(X, dY)
+    Xd, Yd = X.astype(np.float64), dY.astype(np.float64)
+    ghost = np.array([np.sum((Xd[b] @ Xd[b].T) * (Yd[b] @ Yd[b].T)) for b in range(B)])
+    np.testing.assert_allclose(n, ghost, rtol=1e-12)
+    np.testing.assert_allclose(n.sum(), oracle.linear_stats(X, dY).sum_g2.sum(), rtol=1e-12)
+    n1 = oracle.example_sqnorms(X[:, :1], dY[:, :1])
+    np.testing.assert_allclose(n1, (Xd[:, 0] ** 2).sum(1) * (Yd[:, 0] ** 2).sum(1), rtol=1e-12)
+    # bf16 bit patterns widen as everywhere else; scaling one example's cotangents by 3 scales its norm by 9
+    Xb = inputs.to_numpy_bits(torch.tensor(X).to(torch.bfloat16))
+    Yb = inputs.to_numpy_bits(torch.tensor(dY).to(torch.bfloat16))
+    nb = oracle.example_sqnorms(Xb, Yb)
+    Y3 = torch.tensor(dY).to(torch.bfloat16)
+    Y3[2] *= 2                                                    # exact in bf16
+    n3 = oracle.example_sqnorms(Xb, inputs.to_numpy_bits(Y3))
+    np.testing.assert_allclose(n3[2], 4 * nb[2], rtol=1e-12)
+    np.testing.assert_array_equal(np.delete(n3, 2), np.delete(nb, 2))
+
+
 # ----------------------------------------------------------------------------- optimizer steps
 
 def test_microadam_with_one_example_is_adam():
