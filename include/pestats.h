@@ -76,6 +76,19 @@ pe_status_t pe_linear_stats_f32(const float* X, const float* dY, int B, int T, i
                                 pe_phi_t phi, float* out_mean, float* out_stat, pe_stream_t stream);
 
 /*
+ * Per-example squared gradient norms (Section 2.3: N_b = ||grad_W f(theta; x_b)||_2^2, the quantity
+ * behind per-example clipping, one of the transformations phi of Section 2.1):
+ *     out_norms[b] = sum_{o,i} G_b[o,i]^2,     G_b = dY_b^T X_b.
+ * bf16 inputs as for pe_linear_stats; out_norms: fp32 [B], 4-byte aligned, overwritten (may be NULL
+ * only if B = 0).  Each G_b tile is formed on chip, squared and reduced there; every tile adds its
+ * share to out_norms[b] with an fp32 atomic, so the result is reproducible only to rounding.  A
+ * clipped batch gradient is then sum_b c_b G_b with c_b = min(1, C / sqrt(N_b)): scale the rows of dY
+ * by c_b and run the ordinary weight-gradient contraction (pe_linear_stats with phi = identity).
+ */
+pe_status_t pe_example_sqnorms(const void* X, const void* dY, int B, int T, int d_in, int d_out,
+                               float* out_norms, pe_stream_t stream);
+
+/*
  * pe_linear_stats for gradient accumulation over micro-batches: the statistics of this call's B
  * examples are ADDED to what out_mean / out_stat already hold (both sums of Eq. (2) are additive over
  * examples, so running this over the micro-batches of a batch, after zeroing the outputs once, gives

@@ -17,7 +17,7 @@ __all__ = [
     "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_staged", "pe_token_sqstats_staged_workspace_bytes",
     "microadam_step", "microsignsgd_step", "pe_status_string", "pe_get_async_status", "pe_set_path", "pe_last_path",
     "pe_launch_count", "pe_reset_launch_count", "pe_token_sqstats_static", "STATIC_SCRATCH_BYTES",
-    "microadam_family_step", "ADAM_VARIANTS", "pe_linear_stats_all", "pe_linear_stats_accumulate",
+    "microadam_family_step", "ADAM_VARIANTS", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms",
 ]
 
 PHI_IDENTITY, PHI_SQUARE, PHI_SIGN = 0, 1, 2
@@ -29,7 +29,7 @@ EXPORTED_SYMBOLS = [
     "pe_linear_stats", "pe_linear_stats_f32", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_staged",
     "pe_token_sqstats_staged_workspace_bytes", "microadam_step", "microsignsgd_step", "pe_status_string",
     "pe_get_async_status", "pe_set_path", "pe_last_path", "pe_launch_count", "pe_reset_launch_count",
-    "pe_token_sqstats_static", "microadam_family_step", "pe_linear_stats_all", "pe_linear_stats_accumulate",
+    "pe_token_sqstats_static", "microadam_family_step", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms",
 ]
 ADAM_VARIANTS = {"adam": 0, "microadam": 1, "microadam_var": 2, "microadam_msq": 3}      # pe_adam_variant_t
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024      # PE_STATIC_SCRATCH_BYTES of pestats.h
@@ -64,6 +64,7 @@ def load_library() -> ctypes.CDLL:
     lib.pe_linear_stats_f32.argtypes = [vp, vp, i, i, i, i, i, vp, vp, vp]
     lib.pe_linear_stats_all.argtypes = [vp, vp, i, i, i, i, vp, vp, vp, vp]
     lib.pe_linear_stats_accumulate.argtypes = [vp, vp, i, i, i, i, i, vp, vp, vp]
+    lib.pe_example_sqnorms.argtypes = [vp, vp, i, i, i, i, vp, vp]
     lib.pe_token_sqstats.argtypes = [vp, vp, i, i, i, i, vp, vp]
     lib.pe_token_sqstats_staged.argtypes = [vp, vp, i, i, i, i, vp, vp, sz, vp]
     lib.pe_token_sqstats_f32.argtypes = [vp, vp, i, i, i, i, vp, vp]
@@ -82,7 +83,7 @@ def load_library() -> ctypes.CDLL:
     lib.pe_launch_count.restype = ll
     lib.pe_reset_launch_count.argtypes = []
     lib.pe_reset_launch_count.restype = None
-    for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_static",
+    for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_static",
                  "pe_token_sqstats_staged",
                  "microadam_step", "microadam_family_step", "microsignsgd_step", "pe_get_async_status", "pe_set_path", "pe_last_path"):
         getattr(lib, name).restype = i
@@ -146,6 +147,19 @@ def pe_linear_stats(X, dY, phi, out_mean=None, out_stat=None):
         _check("pe_linear_stats", load_library().pe_linear_stats(
             X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, _phi(phi), _ptr(out_mean), _ptr(out_stat), _stream(X)))
     return out_mean, out_stat
+
+
+def pe_example_sqnorms(X, dY, out_norms=None):
+    """Per-example squared gradient norms ||dY_b^T X_b||_F^2 as a float32 [B] tensor (bf16 inputs)."""
+    B, T, d_in, d_out = _io_check(X, dY, torch.bfloat16)
+    if out_norms is None:
+        out_norms = torch.empty((B,), dtype=torch.float32, device=X.device)
+    if out_norms.dtype != torch.float32 or tuple(out_norms.shape) != (B,) or not out_norms.is_contiguous():
+        raise ValueError("out_norms must be a contiguous float32 [B] tensor")
+    with _dev_ctx(X):
+        _check("pe_example_sqnorms", load_library().pe_example_sqnorms(
+            X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, out_norms.data_ptr() if B > 0 else None, _stream(X)))
+    return out_norms
 
 
 def pe_linear_stats_accumulate(X, dY, phi, out_mean, out_stat):

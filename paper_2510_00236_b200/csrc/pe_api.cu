@@ -34,7 +34,7 @@ struct DeviceInfo {
   std::atomic<int> state{0};     // 0 unknown, 1 ready, -1 failed
   int cc_major = 0, sm_count = 0;
   unsigned int* status_ptr = nullptr;
-  bool tc_attr_set[11] = {};
+  bool tc_attr_set[12] = {};
   bool tok_attr_set = false;
 };
 static DeviceInfo g_dev[MAX_DEVICES];
@@ -242,7 +242,7 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = per_example; p.half_operands = half_ops ? 1 : 0;
   p.accumulate = accumulate ? 1 : 0;
   p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
-  p.out_mean = out_mean; p.out_stat = out_stat; p.out_sign = out_sign; p.dev_status = di->status_ptr;
+  p.out_mean = out_mean; p.out_stat = out_stat; p.out_sign = out_sign; p.out_norms = nullptr; p.dev_status = di->status_ptr;
   dim3 grid(2 * pairs_m * tiles_n, 1, ns);
   if (triple) return launch_tc_inst<1, false, 128, MEAN_REGS_SIGN>(di, 10, mx, my, mm, ms, msgn, p, grid, st);
   if (!per_example) return launch_tc_inst<0, false, 256, MEAN_NONE>(di, 4, mx, my, mm, ms, msgn, p, grid, st);
@@ -260,6 +260,28 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   }
   if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, MEAN_NONE>(di, 2, mx, my, mm, ms, msgn, p, grid, st);
   return launch_tc_inst<2, false, 256, MEAN_NONE>(di, 3, mx, my, mm, ms, msgn, p, grid, st);
+}
+
+// Per-example squared norms on the tensor cores: the statistic-only 256 x 256 schedule, but every
+// example's tile is reduced to one number and added to norms[b] (zeroed by the caller of this function).
+static pe_status_t launch_tc_norms(DeviceInfo* di, const void* X, const void* dY, int B, int T, int d_in, int d_out, float* norms,
+                                   cudaStream_t st) {
+  CUtensorMap mx, my;
+  const int box_feats = TcOperand<false, 256>::BOX_FEATS, box_tokens = tc_default_bk(false, 256);
+  pe_status_t rc = make_operand_map(&mx, X, B, T, d_in, false, box_feats, box_tokens);
+  if (rc != PE_OK) return rc;
+  rc = make_operand_map(&my, dY, B, T, d_out, false, box_feats, box_tokens);
+  if (rc != PE_OK) return rc;
+  const int tiles_n = (d_in + 255) / 256, pairs_m = (d_out + TC_PAIR_M - 1) / TC_PAIR_M;
+  if ((long long)tiles_n * pairs_m > (1ll << 29)) return PE_ERR_DIM;
+  const int ns = choose_nsplit((long long)tiles_n * pairs_m, B, T, di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 16);
+  TcParams p;
+  p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = 1; p.half_operands = 0;
+  p.accumulate = 1;       // nothing is zeroed by a preceding kernel and no matrix is written
+  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
+  p.out_mean = nullptr; p.out_stat = nullptr; p.out_sign = nullptr; p.out_norms = norms; p.dev_status = di->status_ptr;
+  // the three output maps are never used by this variant: any valid map will do
+  return launch_tc_inst<1, false, 256, MEAN_NORMS>(di, 11, mx, my, mx, mx, mx, p, dim3(2 * pairs_m * tiles_n, 1, ns), st);
 }
 
 template <typename TIn, int MODE>
@@ -385,6 +407,32 @@ pe_status_t pe_linear_stats(const void* X, const void* dY, int B, int T, int d_i
                             float* out_mean, float* out_stat, pe_stream_t stream) {
   return linear_stats_impl<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T,
                                           d_in, d_out, phi, out_mean, out_stat, reinterpret_cast<cudaStream_t>(stream), true);
+}
+
+pe_status_t pe_example_sqnorms(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_norms,
+                               pe_stream_t stream) {
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (!out_norms && B > 0) return PE_ERR_NULL;
+  pe_status_t rc = validate_stats(X, dY, B, T, d_in, d_out, nullptr, nullptr, false, 16);
+  if (rc != PE_OK) return rc;
+  if (out_norms && !aligned(out_norms, 4)) return PE_ERR_ALIGN;
+  DeviceInfo* di = nullptr;
+  rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  if (B == 0) return PE_OK;
+  if (cudaMemsetAsync(out_norms, 0, (size_t)B * sizeof(float), st) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
+  if (T == 0) return PE_OK;
+  const int forced = g_path.load();
+  const bool tc_ok = tc_shape_ok(B, T, d_in, d_out);
+  if ((forced == PE_PATH_TENSOR || forced == PE_PATH_TENSOR_NARROW) && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
+  if (tc_ok && forced != PE_PATH_SIMT) {
+    g_last_path.store(PE_PATH_TENSOR);
+    return launch_tc_norms(di, X, dY, B, T, d_in, d_out, out_norms, st);
+  }
+  g_last_path.store(PE_PATH_SIMT);
+  // every block handles whole examples of its slice and adds to out_norms[b]: "accumulate" keeps launch_simt from zeroing
+  return launch_simt<__nv_bfloat16, MODE_NORMS>(di, static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T,
+                                                d_in, d_out, 1, nullptr, out_norms, st, true);
 }
 
 pe_status_t pe_linear_stats_accumulate(const void* X, const void* dY, int B, int T, int d_in, int d_out, pe_phi_t phi,

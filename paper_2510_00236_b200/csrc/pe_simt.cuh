@@ -12,7 +12,7 @@ constexpr int SIMT_TILE = 64;   // output tile edge
 constexpr int SIMT_TK = 16;     // tokens staged per step
 constexpr int SIMT_THREADS = 256;
 
-enum : int { MODE_STATS = 0, MODE_TOKEN = 1 };
+enum : int { MODE_STATS = 0, MODE_TOKEN = 1, MODE_NORMS = 2 };
 
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
@@ -26,6 +26,8 @@ __device__ __forceinline__ float apply_phi(float g, int phi) {
 // MODE_STATS: out_mean = sum_b G_b, out_stat = sum_b phi(G_b)         (Section 2.3, Eq. (2))
 // MODE_TOKEN: out_stat = sum_{b,t} dY^2 X^2; operands are squared as they are staged and the
 //             accumulator is never reset between examples             (Section 2.3, per-token form)
+// MODE_NORMS: out_stat is a [B] array, zero on entry; every tile adds its share of ||G_b||_F^2 to
+//             out_stat[b] (Section 2.3, per-example squared norms); no [d_out, d_in] output
 // gridDim = (ceil(d_in/64), ceil(d_out/64), nsplit); block z handles examples [z*B/nsplit, (z+1)*B/nsplit).
 // With nsplit > 1 the outputs must be zero on entry and partial sums are added atomically; with
 // accumulate != 0 the results are added to whatever the outputs hold.
@@ -49,7 +51,7 @@ simt_stats_kernel(const TIn* __restrict__ X, const TIn* __restrict__ dY, int B, 
     for (int c = 0; c < 4; ++c) g[r][c] = acc_stat[r][c] = acc_mean[r][c] = 0.f;
 
   for (int b = b_begin; b < b_end; ++b) {
-    if (MODE == MODE_STATS) {
+    if (MODE == MODE_STATS || MODE == MODE_NORMS) {
 #pragma unroll
       for (int r = 0; r < 4; ++r)
 #pragma unroll
@@ -88,6 +90,16 @@ simt_stats_kernel(const TIn* __restrict__ X, const TIn* __restrict__ dY, int B, 
       }
       __syncthreads();
     }
+    if (MODE == MODE_NORMS) {
+      float s = 0.f;            // entries outside the matrix are exact zeros (their operands were zero-filled)
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) s = fmaf(g[r][c], g[r][c], s);
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+      if ((threadIdx.x & 31) == 0) atomicAdd(out_stat + b, s);
+    }
     if (MODE == MODE_STATS) {
 #pragma unroll
       for (int r = 0; r < 4; ++r)
@@ -99,22 +111,24 @@ simt_stats_kernel(const TIn* __restrict__ X, const TIn* __restrict__ dY, int B, 
     }
   }
 
+  if constexpr (MODE != MODE_NORMS) {       // MODE_NORMS has no [d_out, d_in] output
 #pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    int o = o0 + ty + 16 * r;
-    if (o >= d_out) continue;
+    for (int r = 0; r < 4; ++r) {
+      int o = o0 + ty + 16 * r;
+      if (o >= d_out) continue;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      int i = i0 + tx + 16 * c;
-      if (i >= d_in) continue;
-      size_t at = (size_t)o * d_in + i;
-      float vs = (MODE == MODE_TOKEN) ? g[r][c] : acc_stat[r][c];
-      if (nsplit == 1 && !accumulate) {
-        if (out_stat) out_stat[at] = vs;
-        if (MODE == MODE_STATS && out_mean) out_mean[at] = acc_mean[r][c];
-      } else {
-        if (out_stat) atomicAdd(out_stat + at, vs);
-        if (MODE == MODE_STATS && out_mean) atomicAdd(out_mean + at, acc_mean[r][c]);
+      for (int c = 0; c < 4; ++c) {
+        int i = i0 + tx + 16 * c;
+        if (i >= d_in) continue;
+        size_t at = (size_t)o * d_in + i;
+        float vs = (MODE == MODE_TOKEN) ? g[r][c] : acc_stat[r][c];
+        if (nsplit == 1 && !accumulate) {
+          if (out_stat) out_stat[at] = vs;
+          if (MODE == MODE_STATS && out_mean) out_mean[at] = acc_mean[r][c];
+        } else {
+          if (out_stat) atomicAdd(out_stat + at, vs);
+          if (MODE == MODE_STATS && out_mean) atomicAdd(out_mean + at, acc_mean[r][c]);
+        }
       }
     }
   }

@@ -16,6 +16,8 @@
 //   MEAN_TMEM, NT = 256: sum_b phi(G_b) in 128 registers per thread, sum_b G_b in
 //                        tensor memory beside ONE per-example accumulator, one issuer -- both outputs
 //   MEAN_NONE, NT = 256: one running sum per thread (128 registers)               -- only sum_b phi(G_b) wanted
+//   MEAN_NORMS, NT = 256: no running sums; every example's sum of squares over the
+//                        tile is reduced and added to out_norms[b]                 -- per-example squared norms
 //   PHI = 0,   NT = 256: no per-example reset (accumulate in tensor memory)        -- plain contraction over all rows
 //
 // Warp roles per block (12 warps): 0 = TMA producer of the dY boxes, 2 = TMEM allocator, then TMA
@@ -103,6 +105,7 @@ struct TcParams {
   float* out_mean;     // may be NULL; written through tmap_mean
   float* out_stat;     // may be NULL; written through tmap_stat
   float* out_sign;     // MEAN_REGS_SIGN only: sum_b sign(G_b), written through tmap_sign
+  float* out_norms;    // MEAN_NORMS only: [B], zero on entry; every tile adds its share of ||G_b||_F^2
   unsigned int* dev_status;
 };
 
@@ -176,7 +179,8 @@ __global__ void __launch_bounds__(256) zero_outputs_kernel(float4* __restrict__ 
 }
 
 // where sum_b G_b is kept in per-example mode; MEAN_REGS_SIGN = MEAN_REGS with phi = square plus the sign statistic
-enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2, MEAN_REGS_SIGN = 3 };
+// MEAN_NORMS keeps no [d_out, d_in] sums at all: it reduces each G_b tile to its sum of squares
+enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2, MEAN_REGS_SIGN = 3, MEAN_NORMS = 4 };
 constexpr int TC_SIGN_COUNT_MAX = 32767;   // examples per block in MEAN_REGS_SIGN mode: 2 * count must fit 16 bits
 
 // gridDim = (2 * pairs_m * tiles_n, 1, nsplit); blockIdx.x = 2 * (pair index in the tile order) + rank in pair.
@@ -190,6 +194,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   constexpr bool TRIPLE = (MEAN == MEAN_REGS_SIGN);
   static_assert((MEAN != MEAN_REGS && !TRIPLE) || NT == 128, "two running sums only fit the registers at NT = 128");
   static_assert(!TRIPLE || PHI == 1, "the three-statistic mode is mean + square + sign");
+  constexpr bool NORMS = (MEAN == MEAN_NORMS);
+  static_assert(!NORMS || (PHI == 1 && NT == 256), "per-example norms: squares on the 256 x 256 tile");
   static_assert(MEAN != MEAN_TMEM || (NT == 256 && PHI != 0), "the tensor-memory mean sits beside one 256-column accumulator");
   constexpr int STAGES = Op::STAGES, BK = Op::BK;
   constexpr int BOX_BYTES = Op::BOX_BYTES, A_BYTES = Op::A_BYTES, STAGE_BYTES = Op::STAGE_BYTES;
@@ -324,7 +330,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     const int q = warp & 3;                 // TMEM lane quadrant this warp may access
     const int h = (warp - 4) >> 2;          // column half of the tile
     constexpr bool KEEP_MEAN = MEAN == MEAN_REGS || TRIPLE || PHI == 0;     // running sum of G_b in registers
-    constexpr int N_STAT = (PHI != 0) ? COLS : 1;
+    constexpr int N_STAT = (PHI != 0 && !NORMS) ? COLS : 1;
     constexpr int N_MEAN = KEEP_MEAN ? COLS : 1;
     float acc_stat[N_STAT], acc_mean[N_MEAN];
     // TRIPLE: sum_b sign(G_b) of two neighbouring columns in one register, as signed 16-bit halves of
@@ -373,6 +379,33 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
           tmem_st_32x32b_x16(maddr + c * 16, r);
         }
         tmem_st_wait();
+      } else if constexpr (NORMS) {
+        // this thread's share of ||G_b||_F^2 (its row, its 128 columns; rows and columns outside the
+        // matrix are exact zeros), then the warp's, then one atomic per warp and example
+        uint64_t sa = f32x2_pack(0.f, 0.f), sb = sa;
+#pragma unroll
+        for (int c = 0; c < COLS / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld_32x32b_x32_wait(taddr + c * 32, r);
+          if (c == COLS / 32 - 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));
+          }
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const uint64_t g0 = f32x2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+            const uint64_t g1 = f32x2_pack(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+            sa = f32x2_fma(g0, g0, sa);
+            sb = f32x2_fma(g1, g1, sb);
+          }
+        }
+        float s0, s1;
+        f32x2_unpack(f32x2_add(sa, sb), s0, s1);
+        float s = s0 + s1;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+        if (lane == 0) atomicAdd(p.out_norms + b_begin + a, s);
       } else {
 #pragma unroll
         for (int c = 0; c < COLS / 32; ++c) {

@@ -97,3 +97,14 @@ def test_accumulate_on_the_simt_path():
     assert pe.pe_last_path() == pe.PATH_SIMT
     st, _ = oracle_on(li)
     assert rel_frob(mean.cpu().numpy(), st.sum_g) <= FROB_TOL and rel_frob(stat.cpu().numpy(), st.sum_g2) <= FROB_TOL
+
+
+def test_per_example_squared_norms_on_the_simt_path():
+    import oracle
+    li = inputs.gaussian_layer(9, 33, 36, 20, seed=1900, device=DEV)
+    norms = pe.pe_example_sqnorms(li.X, li.dY)
+    torch.cuda.synchronize()
+    assert pe.pe_last_path() == pe.PATH_SIMT
+    want = oracle.example_sqnorms(inputs.to_numpy_bits(li.X), inputs.to_numpy_bits(li.dY))
+    assert np.max(np.abs(norms.cpu().numpy() - want) / want) <= 2e-3
+    assert pe.pe_example_sqnorms(li.X[:0], li.dY[:0]).numel() == 0

@@ -4,6 +4,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2510_00236_b200 as pe
 from paper_2510_00236_b200 import inputs
 from parity_util import boundary_and_random, check_all, gpu_stats
@@ -217,6 +218,29 @@ def test_accumulating_over_micro_batches_gives_the_statistics_of_the_batch(B, T,
         check_sign(only.cpu().numpy() - 3.0, st)
     else:
         assert rel_frob(only.cpu().numpy().astype(np.float64) - 3.0, ref) <= FROB_TOL + 1e-4
+
+
+@pytest.mark.parametrize("B,T,d_in,d_out", [(5, 200, 136, 264), (70, 48, 8, 8), (33, 300, 520, 264), (9, 16, 320, 192),
+                                              (3, 2000, 264, 520), (64, 256, 512, 2048)])
+def test_per_example_squared_norms(B, T, d_in, d_out):
+    """pe_example_sqnorms against the oracle (on the benchmark layer: on a sample of the examples)."""
+    li = inputs.heterogeneous_layer(B, T, d_in, d_out, seed=1800 + B, device=DEV, with_weights=False)
+    norms = torch.full((B,), float("nan"), device=DEV)
+    pe.pe_example_sqnorms(li.X, li.dY, norms)
+    torch.cuda.synchronize()
+    assert pe.pe_last_path() == pe.PATH_TENSOR and pe.pe_get_async_status(DEV) == (0, 0)
+    got = norms.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    picked = list(range(B)) if B * T * d_in * d_out <= 3e9 else [0, 1, B // 2, B - 1]      # the oracle is slow: sample examples
+    want = oracle.example_sqnorms(inputs.to_numpy_bits(li.X[picked]), inputs.to_numpy_bits(li.dY[picked]))
+    assert np.max(np.abs(got[picked] - want) / want) <= 2e-3          # every example, not a norm over the batch
+    # the norms add up to the sum of all entries of sum_b G_b^2
+    _, sq = pe.pe_linear_stats(li.X, li.dY, "square")
+    assert abs(float(sq.double().sum()) - got.sum()) <= 1e-4 * got.sum()
+    # a second call overwrites, it does not add
+    pe.pe_example_sqnorms(li.X, li.dY, norms)
+    torch.cuda.synchronize()
+    assert np.max(np.abs(norms.cpu().numpy() - got) / got) <= 1e-5
 
 
 def test_three_statistics_of_an_empty_batch_are_zero():
