@@ -229,6 +229,9 @@ def context_numbers(torch, pe, st, li, peaks, dev):
     extra["pe_linear_stats_sign_us"] = {"median": med_s * 1e3, "best": best_s * 1e3, "tflops_median": flops_one / med_s / 1e9}
     med_a3, best_a3 = time_each(torch, lambda i: pe.pe_linear_stats_all(li.X, li.dY, st["mean"], st["sq"], st["sgn"]))
     extra["pe_linear_stats_all_us"] = {"median": med_a3 * 1e3, "best": best_a3 * 1e3, "tflops_median": flops_one / med_a3 / 1e9}
+    norms = torch.empty((B,), device=dev)
+    med_n, best_n = time_each(torch, lambda i: pe.pe_example_sqnorms(li.X, li.dY, norms))
+    extra["pe_example_sqnorms_us"] = {"median": med_n * 1e3, "best": best_n * 1e3, "tflops_median": flops_one / med_n / 1e9}
     med_t, best_t = time_each(torch, lambda i: pe.pe_token_sqstats(li.X, li.dY, st["tok"]))
     extra["pe_token_sqstats_us"] = {"median": med_t * 1e3, "best": best_t * 1e3, "tflops_median": flops_one / med_t / 1e9}
     need = pe.pe_token_sqstats_staged_workspace_bytes(B, T, d_in, d_out)
