@@ -182,11 +182,20 @@ tok_sqstats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         // A stage is 1024 16-byte chunks (4 boxes x 32 rows x 8 chunks of 8 features); chunk g of the
         // stage goes to lane g % 32 of warp (g / 32) % 4 of the group.  Eight neighbouring lanes read
         // one 128-byte row; its 64 features become two 128-byte rows of two neighbouring cooked boxes.
+        // All eight loads first: raw and cooked stages live in the same shared array, so a load written
+        // after a store would have to stay behind it and every iteration would pay the load latency.
+        uint4 vin[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int g = (i * 4 + wl) * 32 + lane;
           const int box = g >> 8, t = (g >> 3) & 31, c = g & 7;
-          const uint4 v = *reinterpret_cast<const uint4*>(raw + box * TOK_BOX_BYTES + t * 128 + ((c ^ (t & 7)) << 4));
+          vin[i] = *reinterpret_cast<const uint4*>(raw + box * TOK_BOX_BYTES + t * 128 + ((c ^ (t & 7)) << 4));
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int g = (i * 4 + wl) * 32 + lane;
+          const int box = g >> 8, t = (g >> 3) & 31, c = g & 7;
+          const uint4 v = vin[i];
           const uint64_t o0 = tok_square_tf32_pair(v.x), o1 = tok_square_tf32_pair(v.y);
           const uint64_t o2 = tok_square_tf32_pair(v.z), o3 = tok_square_tf32_pair(v.w);
           // Lanes with c >= 4 (the second of the two boxes) store their halves in the other order, so
