@@ -150,6 +150,7 @@ def test_staged_token_stat_keeps_every_column_accurate_over_a_wide_range_of_magn
     (70, 96, 8, 8, True),          # one tile, batch split across blocks: partial sign counts are added
     (33, 300, 520, 264, True),     # odd slices
     (1, 1000, 256, 128, True),     # single example
+    (2, 4100, 136, 264, True),     # very long sequences stay on the one-pass kernel
     (64, 256, 512, 2048, True),    # the benchmark layer, sampled below
     (9, 16, 320, 192, False),      # short sequences: served by the two separate calls
     (21, 64, 136, 520, False),     # exactly one short stage per example: still the two calls
