@@ -550,14 +550,14 @@ pe_status_t pe_token_sqstats_staged(const void* X, const void* dY, int B, int T,
     const uint16_t* Xb = static_cast<const uint16_t*>(X);
     const uint16_t* Yb = static_cast<const uint16_t*>(dY);
     if (cudaMemsetAsync(max_x, 0, ((size_t)d_in + (size_t)d_out) * 4, st) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
-    const dim3 gx = stage_grid(rows, d_in, di->sm_count), gy = stage_grid(rows, d_out, di->sm_count);
-    column_max_kernel<<<gx, STAGE_THREADS, 0, st>>>(Xb, rows, d_in, max_x);
+    // one launch per pass serves both tensors (gridDim.z picks X or dY; the grid is sized for the wider one)
+    dim3 grid = stage_grid(rows, d_in > d_out ? d_in : d_out, di->sm_count);
+    grid.y = (grid.y + 1) / 2;
+    grid.z = 2;
+    const StageTensor sx = {Xb, x2, max_x, d_in}, sy = {Yb, y2, max_y, d_out};
+    column_max_kernel<<<grid, STAGE_THREADS, 0, st>>>(sx, sy, rows);
     if ((rc = check_launch()) != PE_OK) return rc;
-    column_max_kernel<<<gy, STAGE_THREADS, 0, st>>>(Yb, rows, d_out, max_y);
-    if ((rc = check_launch()) != PE_OK) return rc;
-    square_to_half_kernel<<<gx, STAGE_THREADS, 0, st>>>(Xb, x2, rows, d_in, max_x);
-    if ((rc = check_launch()) != PE_OK) return rc;
-    square_to_half_kernel<<<gy, STAGE_THREADS, 0, st>>>(Yb, y2, rows, d_out, max_y);
+    square_to_half_kernel<<<grid, STAGE_THREADS, 0, st>>>(sx, sy, rows);
     if ((rc = check_launch()) != PE_OK) return rc;
     // B and T only enter through B*T: regroup the rows into two-stage "examples" when possible so
     // the batch split has many units to balance.

@@ -34,9 +34,21 @@ __device__ __forceinline__ float stage_inv_scale(int E) { return __uint_as_float
 
 // max_bits[c] = max over rows of |src[r, c]| as a bf16 bit pattern (which orders like the magnitude).
 // src: [rows, d] bf16, d a multiple of 8; max_bits: [d], zero on entry.  gridDim.x covers the columns
-// in groups of 256, gridDim.y slices the rows.
+// in groups of 256, gridDim.y slices the rows, gridDim.z = 2 picks the tensor (0: X, 1: dY), so one
+// launch serves both.
+struct StageTensor {
+  const uint16_t* src;     // [rows, d] bf16 bit patterns
+  __half* dst;             // [rows, d] scaled squares (square_to_half_kernel only)
+  uint32_t* max_bits;      // [d]
+  int d;
+};
 __global__ void __launch_bounds__(STAGE_THREADS)
-column_max_kernel(const uint16_t* __restrict__ src, long long rows, int d, uint32_t* __restrict__ max_bits) {
+column_max_kernel(StageTensor tx_, StageTensor ty_, long long rows) {
+  const StageTensor& tn = blockIdx.z == 0 ? tx_ : ty_;
+  const uint16_t* __restrict__ src = tn.src;
+  uint32_t* __restrict__ max_bits = tn.max_bits;
+  const int d = tn.d;
+  if (blockIdx.x * 256 >= d) return;          // the grid is sized for the wider tensor
   __shared__ uint32_t part[8][32][4];
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int col = (blockIdx.x * 32 + tx) * 8;
@@ -68,11 +80,15 @@ column_max_kernel(const uint16_t* __restrict__ src, long long rows, int d, uint3
   }
 }
 
-// dst[r, c] = half(src[r, c]^2 * scale(c)).  Same thread layout as column_max_kernel, so a thread's
-// eight columns, and with them its scales, never change.
+// dst[r, c] = half(src[r, c]^2 * scale(c)).  Same grid and thread layout as column_max_kernel, so a
+// thread's eight columns, and with them its scales, never change.
 __global__ void __launch_bounds__(STAGE_THREADS)
-square_to_half_kernel(const uint16_t* __restrict__ src, __half* __restrict__ dst, long long rows, int d,
-                      const uint32_t* __restrict__ max_bits) {
+square_to_half_kernel(StageTensor tx_, StageTensor ty_, long long rows) {
+  const StageTensor& tn = blockIdx.z == 0 ? tx_ : ty_;
+  const uint16_t* __restrict__ src = tn.src;
+  __half* __restrict__ dst = tn.dst;
+  const uint32_t* __restrict__ max_bits = tn.max_bits;
+  const int d = tn.d;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int col = (blockIdx.x * 32 + tx) * 8;
   if (col >= d) return;
