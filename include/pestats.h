@@ -137,7 +137,7 @@ pe_status_t pe_token_sqstats_f32(const float* X, const float* dY, int B, int T, 
  * pe_token_sqstats contracts tf32 at half that rate), and a last kernel undoes the scales.  Half keeps
  * the same 11 significant bits as tf32, rounded to nearest even; within a column, entries more than
  * 2^14 below the column's largest magnitude lose bits gradually and vanish 2^20 below it.  Faster
- * than pe_token_sqstats once B*T*(d_in + d_out) reaches about 10^8 elements, slower below (six
+ * than pe_token_sqstats once B*T*(d_in + d_out) reaches about 10^8 elements, slower below (several
  * launches instead of one).  Also the kernel sequence behind pe_token_sqstats_static.  The SIMT path
  * ignores the workspace (it may then be NULL).
  */
