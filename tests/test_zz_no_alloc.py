@@ -46,7 +46,7 @@ def _both_ways(li):
 
 
 def test_static_scratch_matches_workspace_version_twice_in_a_row():
-    first = inputs.gaussian_layer(12, 128, 264, 392, seed=901, device=DEV)        # 4 MB of staging, ragged tiles
+    first = inputs.gaussian_layer(12, 128, 264, 392, seed=901, device=DEV)        # 2 MB of staging, ragged tiles
     second = inputs.heavy_tailed_layer(5, 64, 136, 128, seed=902, device=DEV)     # smaller: reuses the array's front
     for li in (first, second):
         got, want = _both_ways(li)
@@ -59,7 +59,7 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row():
 
 
 def test_static_scratch_refuses_shapes_beyond_its_size():
-    B, T, d_in, d_out = 64, 256, 512, 2048                                       # needs 168 MB of staging
+    B, T, d_in, d_out = 64, 256, 512, 2048                                       # needs 84 MB of staging
     assert pe.pe_token_sqstats_staged_workspace_bytes(B, T, d_in, d_out) > pe.STATIC_SCRATCH_BYTES
     X = torch.zeros((B, T, d_in), dtype=torch.bfloat16, device=DEV)
     dY = torch.zeros((B, T, d_out), dtype=torch.bfloat16, device=DEV)
