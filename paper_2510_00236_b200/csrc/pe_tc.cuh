@@ -59,11 +59,11 @@ constexpr int TC_SMEM_BUDGET = 200 * 1024;   // operand ring; leaves room for ba
 // statistics; tf32 (kind::tf32, fp32 storage, 8 tokens per instruction) for the per-token statistic,
 // whose squared operands need more than bf16's 8 significant bits.  NT = d_in columns per pair tile.
 // Default tokens per pipeline stage: 128 for the 256 x 128 tile, 64 for the 256 x 256 tile, 32 for
-// tf32.  With both outputs and short sequences (T <= 64) the 256 x 128 tile takes 32-token stages
+// tf32.  With both outputs and short sequences (T <= 32) the 256 x 128 tile takes 32-token stages
 // instead: a 128-token box would be mostly zero fill, and 16 small slots keep more examples in flight.
 __host__ __device__ constexpr int tc_default_bk(bool tf32, int nt) { return tf32 ? 32 : (nt == 128 ? 128 : 64); }
 constexpr int TC_SHORT_BK = 32;
-constexpr int TC_SHORT_T = 64;
+constexpr int TC_SHORT_T = 32;
 template <bool TF32, int NT, int BK_ = tc_default_bk(TF32, NT)>
 struct TcOperand {
   static constexpr int ELEM_BYTES = TF32 ? 4 : 2;

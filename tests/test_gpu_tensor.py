@@ -43,8 +43,9 @@ def test_structured_single_tile_catches_layout_mistakes():
     (70, 48, 8, 8),         # smallest widths the path takes, batch split across blocks
     (40, 96, 384, 256),
     (130, 32, 264, 392),    # many short sequences: 32-token stages, batch split
-    (21, 64, 136, 520),     # two short stages per example
-    (11, 33, 128, 256),     # one full and one nearly empty short stage
+    (21, 64, 136, 520),     # half-filled stages
+    (11, 33, 128, 256),     # just above the short-stage limit
+    (13, 32, 264, 136),     # exactly one short stage per example
     (2, 4100, 136, 264),    # very long sequences: sum_b G_b kept in tensor memory when both outputs are wanted
 ])
 def test_tensor_small_shapes_full_comparison(B, T, d_in, d_out):
@@ -153,7 +154,8 @@ def test_staged_token_stat_keeps_every_column_accurate_over_a_wide_range_of_magn
     (2, 4100, 136, 264, True),     # very long sequences stay on the one-pass kernel
     (64, 256, 512, 2048, True),    # the benchmark layer, sampled below
     (9, 16, 320, 192, False),      # short sequences: served by the two separate calls
-    (21, 64, 136, 520, False),     # exactly one short stage per example: still the two calls
+    (21, 32, 136, 520, False),     # exactly one short stage per example: still the two calls
+    (21, 64, 136, 520, True),      # half-filled stages
 ])
 def test_three_statistics_in_one_pass(B, T, d_in, d_out, tensor_one_pass):
     """pe_linear_stats_all: sum_b G_b, sum_b G_b^2 and sum_b sign(G_b) from one pass over the examples, against
