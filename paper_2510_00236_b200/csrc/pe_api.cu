@@ -310,6 +310,14 @@ static pe_status_t validate_stats(const void* X, const void* dY, int B, int T, i
   return PE_OK;
 }
 
+// A plain contraction over all B*T rows does not care where one sequence ends: short sequences are
+// regrouped into full two-stage "examples" when the rows divide evenly (fewer, fuller pipeline stages).
+static void regroup_rows(int& B, int& T) {
+  constexpr int REGROUP = 2 * TcOperand<false, 256>::BK;
+  const long long rows = (long long)B * T;
+  if (T < REGROUP && rows % REGROUP == 0) { B = (int)(rows / REGROUP); T = REGROUP; }
+}
+
 template <typename TIn>
 static pe_status_t linear_stats_impl(const TIn* X, const TIn* dY, int B, int T, int d_in, int d_out, pe_phi_t phi,
                                      float* out_mean, float* out_stat, cudaStream_t st, bool allow_tc, bool accumulate = false) {
@@ -327,7 +335,9 @@ static pe_status_t linear_stats_impl(const TIn* X, const TIn* dY, int B, int T, 
     if constexpr (sizeof(TIn) == 2) {
       g_last_path.store(PE_PATH_TENSOR);
       if (phi == PE_PHI_IDENTITY) {
-        // phi = identity: both outputs are the plain contraction over all B*T rows.
+        // phi = identity: both outputs are the plain contraction over all B*T rows, and B and T only enter
+        // through B*T: regroup short sequences into full two-stage "examples" when the rows divide evenly.
+        regroup_rows(B, T);
         float* first = out_mean ? out_mean : out_stat;
         rc = launch_tc(di, X, dY, B, T, d_in, d_out, phi, 0, first, nullptr, st, false, nullptr, accumulate);
         if (rc == PE_OK && out_mean && out_stat && accumulate)      // a copy would overwrite: contract once more into the second
@@ -340,8 +350,10 @@ static pe_status_t linear_stats_impl(const TIn* X, const TIn* dY, int B, int T, 
         }
         return rc;
       }
-      if (!out_stat)      // only sum_b G_b wanted: the plain contraction
+      if (!out_stat) {    // only sum_b G_b wanted: the plain contraction
+        regroup_rows(B, T);
         return launch_tc(di, X, dY, B, T, d_in, d_out, phi, 0, out_mean, nullptr, st, false, nullptr, accumulate);
+      }
       return launch_tc(di, X, dY, B, T, d_in, d_out, phi, 1, out_mean, out_stat, st, false, nullptr, accumulate);
     }
   }
