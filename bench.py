@@ -278,6 +278,9 @@ def run_sweep(args):
             flops = 2.0 * B * T * d * d
             med_b, best_b = time_each(torch, lambda i: pe.pe_linear_stats(sets[i % nsets].X, sets[i % nsets].dY, pe.PHI_SQUARE, mean, stat), iters=12)
             med_s, best_s = time_each(torch, lambda i: pe.pe_linear_stats(sets[i % nsets].X, sets[i % nsets].dY, pe.PHI_SQUARE, None, stat), iters=12)
+            sgn = torch.empty((d, d), device=dev)
+            med_n, _ = time_each(torch, lambda i: pe.pe_linear_stats(sets[i % nsets].X, sets[i % nsets].dY, pe.PHI_SIGN, None, stat), iters=12)
+            med_a, _ = time_each(torch, lambda i: pe.pe_linear_stats_all(sets[i % nsets].X, sets[i % nsets].dY, mean, stat, sgn), iters=12)
             med_g, best_g = time_each(torch, lambda i: torch.matmul(sets[i % nsets].dY.view(B * T, d).t(), sets[i % nsets].X.view(B * T, d)), iters=12)
             status, detail = pe.pe_get_async_status(dev)
             assert status == 0, (status, detail)
@@ -285,15 +288,17 @@ def run_sweep(args):
             # 128 lanes x 148 SMs, packed 2-wide at best), and HBM
             t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
             t_hbm = (bytes_in + 8.0 * d * d) / (peaks["hbm_gbs"] * 1e9)
+            t_alu = 2.0 * B * d * d / (148 * 128 * 1.965e9)
             print(json.dumps({
                 "sweep_point": {"B": B, "T": T, "d_in": d, "d_out": d}, "input_sets": nsets,
                 "both_outputs_us": med_b * 1e3, "both_outputs_tflops": flops / med_b / 1e9,
                 "both_outputs_frac_of_peak": flops / med_b / 1e9 / peaks["bf16_tflops"],
                 "stat_only_us": med_s * 1e3, "stat_only_tflops": flops / med_s / 1e9,
+                "sign_only_us": med_n * 1e3, "all_three_us": med_a * 1e3, "overhead_all_three_vs_gemm": med_a / med_g,
                 "cublas_gemm_us": med_g * 1e3, "cublas_gemm_tflops": flops / med_g / 1e9,
                 "overhead_both_vs_gemm": med_b / med_g, "overhead_stat_vs_gemm": med_s / med_g,
-                "bound_tensor_us": t_tensor * 1e6, "bound_hbm_us": t_hbm * 1e6, "peak_source": peaks["source"]}), flush=True)
-            del sets, mean, stat
+                "bound_tensor_us": t_tensor * 1e6, "bound_hbm_us": t_hbm * 1e6, "bound_alu_us": t_alu * 1e6, "peak_source": peaks["source"]}), flush=True)
+            del sets, mean, stat, sgn
             torch.cuda.empty_cache()
 
 
