@@ -126,23 +126,11 @@ template <int PHI>
 __device__ __forceinline__ float phi_apply(float g) {
   if (PHI == 1) return g * g;
   if (PHI == 2) {
-    // sign(g) with sign(+-0) = 0: copy the sign bit onto 1.0f, then zero it when g == 0.
-    float s = __uint_as_float((__float_as_uint(g) & 0x80000000u) | 0x3f800000u);
-    return g != 0.f ? s : 0.f;
+    // sign(g) with sign(+-0) = 0: (g != 0) as 1.0f / 0.0f, then g's sign bit copied onto it (-0.0f adds nothing)
+    const float nz = (g != 0.f) ? 1.f : 0.f;
+    return __uint_as_float(__float_as_uint(nz) | (__float_as_uint(g) & 0x80000000u));
   }
   return g;
-}
-
-// -1 if the fp32 value with these bits is > 0 (< 0), else 0; one instruction each.
-__device__ __forceinline__ int set_gt_zero(uint32_t bits) {
-  int d;
-  asm("set.gt.s32.f32 %0, %1, 0f00000000;" : "=r"(d) : "f"(__uint_as_float(bits)));
-  return d;
-}
-__device__ __forceinline__ int set_lt_zero(uint32_t bits) {
-  int d;
-  asm("set.lt.s32.f32 %0, %1, 0f00000000;" : "=r"(d) : "f"(__uint_as_float(bits)));
-  return d;
 }
 
 // Walks the slots of the operand ring in the order the producers fill them.  With two issuers the
@@ -333,9 +321,9 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     constexpr int N_STAT = (PHI != 0 && !NORMS) ? COLS : 1;
     constexpr int N_MEAN = KEEP_MEAN ? COLS : 1;
     float acc_stat[N_STAT], acc_mean[N_MEAN];
-    // TRIPLE: sum_b sign(G_b) of two neighbouring columns in one register, as signed 16-bit halves of
-    // one 32-bit two's-complement sum (low + 65536 * high; |sum| <= nb <= 32767 per half, so both are
-    // recovered exactly at the end).  The third statistic costs 32 registers instead of 64.
+    // TRIPLE: sum_b (sign(G_b) + 1) of two neighbouring columns in one register, as unsigned 16-bit
+    // halves (each at most 2 nb <= 65534, so a plain 32-bit add never carries from one half into the
+    // other); sum_b sign = count - nb.  The third statistic costs 32 registers instead of 64.
     constexpr int N_CNT = TRIPLE ? COLS / 2 : 1;
     uint32_t acc_cnt[N_CNT];
 #pragma unroll
@@ -437,10 +425,11 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 f32x2_unpack(s2, acc_stat[c * 32 + j], acc_stat[c * 32 + j + 1]);
               }
               if (TRIPLE) {
-                // set.xx.s32.f32 gives -1 / 0, so sign(g) = (g < 0 ? -1 : 0) - (g > 0 ? -1 : 0); +-0 give 0
-                const int s0 = set_lt_zero(r[j]) - set_gt_zero(r[j]);
-                const int s1 = set_lt_zero(r[j + 1]) - set_gt_zero(r[j + 1]);
-                acc_cnt[(c * 32 + j) >> 1] += (uint32_t)(s0 + s1 * 65536);
+                // sign(g) as a float, plus 2^23 * 1.5 + 1: the low 16 bits of the sum's bit pattern are
+                // sign(g) + 1 in {0, 1, 2}; one byte permute packs the two columns' low halves
+                const float t0 = phi_apply<2>(__uint_as_float(r[j])) + 12582913.f;
+                const float t1 = phi_apply<2>(__uint_as_float(r[j + 1])) + 12582913.f;
+                acc_cnt[(c * 32 + j) >> 1] += __byte_perm(__float_as_uint(t0), __float_as_uint(t1), 0x5410);
               }
             }
           }
@@ -518,16 +507,12 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         if (p.out_sign) {
           if (lane == 0) bulk_wait_read_all();
           __syncwarp();
+          const float nbf = (float)nb;
 #pragma unroll
           for (int c = 0; c < PANELS; ++c) {
             float v[32];
 #pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-              const int both = (int)acc_cnt[(c * 32 + j) >> 1];
-              const int low = (int)(short)(both & 0xFFFF);
-              v[j] = (float)low;
-              v[j + 1] = (float)((both - low) >> 16);
-            }
+            for (int j = 0; j < 32; ++j) v[j] = (float)((acc_cnt[(c * 32 + j) >> 1] >> (16 * (j & 1))) & 0xFFFFu) - nbf;
             put_panel(stage_base + c * 4096, v);
           }
           send(&tmap_sign, stage_base);
