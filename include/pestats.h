@@ -2,9 +2,11 @@
  * pestats -- per-example gradient statistics for linear layers on NVIDIA B200 (sm_100a).
  *
  * C ABI.  Every pointer is a DEVICE pointer unless its name starts with "h_" or the comment says
- * "host".  The caller owns every buffer and the stream; the library allocates nothing, keeps no
- * state between calls apart from the process-wide path override below, and enqueues its work
- * asynchronously on `stream` (0 = the legacy default stream).  Functions return a pe_status_t and
+ * "host".  The caller owns every buffer and the stream; the library allocates nothing and enqueues
+ * its work asynchronously on `stream` (0 = the legacy default stream).  State kept between calls: the
+ * process-wide path override and wait limit below, and a per-device cache of device properties and
+ * kernel attributes that the first call on a device fills in (guarded by a mutex, so first calls
+ * from several host threads are safe).  Functions return a pe_status_t and
  * never throw.  Errors detected on the host (bad arguments, unsupported shape, CUDA launch
  * failure) are returned immediately and nothing is enqueued.  Errors detected on the device (a
  * bounded wait inside a kernel that ran out) are latched in a device status word that
@@ -46,11 +48,13 @@ typedef enum {
 typedef enum { PE_PHI_IDENTITY = 0, PE_PHI_SQUARE = 1, PE_PHI_SIGN = 2 } pe_phi_t;
 
 /* Which kernel family a call may use.  AUTO picks the tensor-core kernel whenever the shape allows
- * it (bf16 inputs, d_in % 8 == 0, d_out % 8 == 0) and the SIMT kernel otherwise.  TENSOR_NARROW is
- * TENSOR with the 256 x 128 tile that keeps both running sums in registers even for long sequences
- * (AUTO and TENSOR use it for T < 4096 only and otherwise keep sum_b G_b in tensor memory beside a
- * 256 x 256 tile); it exists so that tests can reach that kernel at any T. */
-typedef enum { PE_PATH_AUTO = 0, PE_PATH_SIMT = 1, PE_PATH_TENSOR = 2, PE_PATH_TENSOR_NARROW = 3 } pe_path_t;
+ * it (bf16 inputs, d_in % 8 == 0, d_out % 8 == 0) and the SIMT kernel otherwise.  When both outputs
+ * are wanted AUTO and TENSOR keep both running sums in registers on a 256 x 128 tile for T < 256, on a
+ * 256 x 192 tile for 256 <= T < 4096 (unless d_in pads badly to multiples of 192), and from T = 4096 on
+ * keep sum_b G_b in tensor memory beside a 256 x 256 tile.  TENSOR_NARROW is TENSOR with the 256 x 128
+ * tile and TENSOR_WIDE is TENSOR with the 256 x 192 tile, both at any T; they exist so that tests can
+ * reach those kernels on every shape. */
+typedef enum { PE_PATH_AUTO = 0, PE_PATH_SIMT = 1, PE_PATH_TENSOR = 2, PE_PATH_TENSOR_NARROW = 3, PE_PATH_TENSOR_WIDE = 4 } pe_path_t;
 
 typedef struct CUstream_st* pe_stream_t; /* a cudaStream_t */
 
@@ -64,9 +68,10 @@ typedef struct CUstream_st* pe_stream_t; /* a cudaStream_t */
  * X, dY: bf16, 16-byte aligned.  out_mean, out_stat: fp32 [d_out, d_in], 16-byte aligned, OVERWRITTEN;
  * either may be NULL to skip it (not both).  Products are exact in fp32 and accumulated in fp32.
  * B, T >= 0 (B == 0 or T == 0 writes zeros, and X, dY may then be NULL); d_in, d_out >= 1; B*T*max(d_in,d_out) < 2^40.
- * When the batch is split across thread blocks the partial sums are combined with fp32 atomic
- * adds, so the low bits of out_mean / the square statistic may differ between runs; the sign
- * statistic is always exact-integer valued.
+ * When the batch is split across thread blocks the outputs are zeroed first and every block adds its
+ * partial tile with fp32 reduce-add bulk stores (the SIMT kernel: fp32 atomic adds), so the low bits
+ * of out_mean / the square statistic may differ between runs; the sign statistic is always
+ * exact-integer valued.
  */
 pe_status_t pe_linear_stats(const void* X, const void* dY, int B, int T, int d_in, int d_out,
                             pe_phi_t phi, float* out_mean, float* out_stat, pe_stream_t stream);

@@ -12,7 +12,7 @@ import os
 import torch
 
 __all__ = [
-    "PestatsError", "PHI_IDENTITY", "PHI_SQUARE", "PHI_SIGN", "PATH_AUTO", "PATH_SIMT", "PATH_TENSOR", "PATH_TENSOR_NARROW",
+    "PestatsError", "PHI_IDENTITY", "PHI_SQUARE", "PHI_SIGN", "PATH_AUTO", "PATH_SIMT", "PATH_TENSOR", "PATH_TENSOR_NARROW", "PATH_TENSOR_WIDE",
     "EXPORTED_SYMBOLS", "library_path", "load_library", "pe_linear_stats", "pe_linear_stats_f32",
     "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_staged", "pe_token_sqstats_staged_workspace_bytes",
     "microadam_step", "microsignsgd_step", "pe_status_string", "pe_get_async_status", "pe_set_path", "pe_last_path",
@@ -21,7 +21,7 @@ __all__ = [
 ]
 
 PHI_IDENTITY, PHI_SQUARE, PHI_SIGN = 0, 1, 2
-PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_NARROW = 0, 1, 2, 3
+PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_NARROW, PATH_TENSOR_WIDE = 0, 1, 2, 3, 4
 _PHI_NAMES = {"identity": PHI_IDENTITY, "square": PHI_SQUARE, "sign": PHI_SIGN}
 
 # every symbol include/pestats.h declares

@@ -5,6 +5,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <cmath>
+#include <mutex>
 
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -27,6 +28,9 @@ static std::atomic<long long> g_launches{0};
 // Both outputs: from this sequence length on the running sum of G_b lives in tensor memory beside a
 // 256-column accumulator (measured: wins or ties at T = 4096, loses 16 % at T = 2048, 17 % at T = 1024).
 constexpr int TC_MEAN_TMEM_MIN_T = 4096;
+// Both outputs, phi = square or sign: from this sequence length on (and below TC_MEAN_TMEM_MIN_T) the pair
+// tile is 256 x 192 instead of 256 x 128, unless d_in is so narrow that the wider tile's padding eats the gain.
+constexpr int TC_WIDE_MIN_T = 256;
 constexpr int TC_BAND = 8;          // pair rows per band of the tile order (8 x 256 rows of d_out)
 
 constexpr int MAX_DEVICES = 64;
@@ -34,10 +38,11 @@ struct DeviceInfo {
   std::atomic<int> state{0};     // 0 unknown, 1 ready, -1 failed
   int cc_major = 0, sm_count = 0;
   unsigned int* status_ptr = nullptr;
-  bool tc_attr_set[12] = {};
+  bool tc_attr_set[16] = {};
   bool tok_attr_set = false;
 };
 static DeviceInfo g_dev[MAX_DEVICES];
+static std::mutex g_dev_mutex;      // guards the lazily filled per-device state (first calls from several host threads)
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -48,7 +53,9 @@ static pe_status_t device_info(DeviceInfo** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) { cudaGetLastError(); return PE_ERR_CUDA; }
   DeviceInfo& d = g_dev[dev];
-  if (d.state.load() == 0) {
+  if (d.state.load(std::memory_order_acquire) == 0) {
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    if (d.state.load(std::memory_order_relaxed) != 0) { *out = &d; return d.cc_major == 10 ? PE_OK : PE_ERR_ARCH; }
     int major = 0, sms = 0;
     void* sp = nullptr;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
@@ -62,7 +69,7 @@ static pe_status_t device_info(DeviceInfo** out) {
       if (cudaGetSymbolAddress(&sp, g_dev_status) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
       d.status_ptr = static_cast<unsigned int*>(sp);
     }
-    d.state.store(1);
+    d.state.store(1, std::memory_order_release);
   }
   *out = &d;
   return d.cc_major == 10 ? PE_OK : PE_ERR_ARCH;
@@ -94,8 +101,10 @@ static pe_status_t check_launch() {
 
 // [B, T, d] row-major (bf16, or fp32 read as tf32) viewed as a 3-D tensor (d, T, B); one box = 128
 // bytes of features x one pipeline stage of tokens of one example, 128-byte swizzled (16-byte chunks for bf16, 32-byte
-// chunks for fp32: the MN-major tf32 MMA accepts no other layout).  Tokens past T and features past d read as zero.
-static pe_status_t make_operand_map(CUtensorMap* m, const void* base, int B, int T, int d, bool f32, int box_feats, int box_tokens) {
+// chunks for fp32: the MN-major tf32 MMA accepts no other layout).  rows64: 64 bytes of features per box row with
+// the 64-byte swizzle (X of the 256 x 192 tile).  Tokens past T and features past d read as zero.
+static pe_status_t make_operand_map(CUtensorMap* m, const void* base, int B, int T, int d, bool f32, int box_feats, int box_tokens,
+                                    bool rows64 = false) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return PE_ERR_CUDA;
   const cuuint64_t es = f32 ? 4ull : 2ull;
@@ -104,7 +113,8 @@ static pe_status_t make_operand_map(CUtensorMap* m, const void* base, int B, int
   cuuint32_t box[3] = {(cuuint32_t)box_feats, (cuuint32_t)box_tokens, 1u};
   cuuint32_t estr[3] = {1u, 1u, 1u};
   CUresult r = enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, f32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   f32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : (rows64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B),
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? PE_OK : PE_ERR_CUDA;
@@ -193,12 +203,15 @@ static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& m
                                   const CUtensorMap& ms, const CUtensorMap& msgn, const TcParams& p, dim3 grid, cudaStream_t st) {
   const bool after_zeroing = p.nsplit > 1 && !p.accumulate;
   constexpr int smem = TcOperand<TF32, NT, BKT>::SMEM_BYTES;
-  if (!di->tc_attr_set[slot]) {
-    if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
-      cudaGetLastError();
-      return PE_ERR_CUDA;
+  {
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    if (!di->tc_attr_set[slot]) {
+      if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+        cudaGetLastError();
+        return PE_ERR_CUDA;
+      }
+      di->tc_attr_set[slot] = true;
     }
-    di->tc_attr_set[slot] = true;
   }
   return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT>, grid, smem, st, after_zeroing, mx, my, mm, ms, msgn, p);
 }
@@ -213,13 +226,19 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   const bool both = per_example && out_mean && out_stat;
   // Both outputs: sum_b G_b in tensor memory beside a 256-wide accumulator, unless the sequences are
   // so short that the per-example drain of that single accumulator would dominate.
-  const bool mean_regs = both && (triple || T < TC_MEAN_TMEM_MIN_T || g_path.load() == PE_PATH_TENSOR_NARROW);
-  const int nt = mean_regs ? 128 : 256;
+  const int forced = g_path.load();
+  const bool mean_regs = both && (triple || T < TC_MEAN_TMEM_MIN_T || forced == PE_PATH_TENSOR_NARROW || forced == PE_PATH_TENSOR_WIDE);
+  // 256 x 192 tile: a third less operand traffic per flop than 256 x 128; its column padding must stay below ~7 %
+  const long long pad192 = (long long)((d_in + 191) / 192) * 192, pad128 = (long long)((d_in + 127) / 128) * 128;
+  const bool wide = mean_regs && !triple && forced != PE_PATH_TENSOR_NARROW &&
+                    (forced == PE_PATH_TENSOR_WIDE || (T >= TC_WIDE_MIN_T && pad192 * 100 <= pad128 * 107));
+  const int nt = mean_regs ? (wide ? 192 : 128) : 256;
   const int box_feats = TcOperand<false, 256>::BOX_FEATS;
-  const bool short_seq = mean_regs && !triple && T <= TC_SHORT_T;      // many short examples, both outputs: small stages
+  const bool short_seq = mean_regs && !wide && !triple && T <= TC_SHORT_T;      // many short examples, both outputs: small stages
   const int box_tokens = short_seq ? TC_SHORT_BK : tc_default_bk(false, nt);
   CUtensorMap mx, my;
-  pe_status_t rc = make_operand_map(&mx, X, B, T, d_in, false, box_feats, box_tokens);
+  pe_status_t rc = wide ? make_operand_map(&mx, X, B, T, d_in, false, TcOperand<false, 192>::B_BOX_FEATS, box_tokens, true)
+                        : make_operand_map(&mx, X, B, T, d_in, false, box_feats, box_tokens);
   if (rc != PE_OK) return rc;
   rc = make_operand_map(&my, dY, B, T, d_out, false, box_feats, box_tokens);
   if (rc != PE_OK) return rc;
@@ -249,6 +268,10 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   if (short_seq) {
     if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, MEAN_REGS, TC_SHORT_BK>(di, 8, mx, my, mm, ms, msgn, p, grid, st);
     return launch_tc_inst<2, false, 128, MEAN_REGS, TC_SHORT_BK>(di, 9, mx, my, mm, ms, msgn, p, grid, st);
+  }
+  if (wide) {
+    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 192, MEAN_REGS>(di, 12, mx, my, mm, ms, msgn, p, grid, st);
+    return launch_tc_inst<2, false, 192, MEAN_REGS>(di, 13, mx, my, mm, ms, msgn, p, grid, st);
   }
   if (mean_regs) {
     if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 128, MEAN_REGS>(di, 0, mx, my, mm, ms, msgn, p, grid, st);
@@ -330,7 +353,7 @@ static pe_status_t linear_stats_impl(const TIn* X, const TIn* dY, int B, int T, 
   if (B == 0 || T == 0) return accumulate ? PE_OK : zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
   const int forced = g_path.load();
   const bool tc_ok = allow_tc && tc_shape_ok(B, T, d_in, d_out);
-  if ((forced == PE_PATH_TENSOR || forced == PE_PATH_TENSOR_NARROW) && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
+  if (forced >= PE_PATH_TENSOR && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
   if (tc_ok && forced != PE_PATH_SIMT) {
     if constexpr (sizeof(TIn) == 2) {
       g_last_path.store(PE_PATH_TENSOR);
@@ -396,12 +419,15 @@ static pe_status_t launch_tok(DeviceInfo* di, const void* X, const void* dY, lon
     rc = zero_for_split(di, out, nullptr, (size_t)d_in * d_out, st);
     if (rc != PE_OK) return rc;
   }
-  if (!di->tok_attr_set) {
-    if (cudaFuncSetAttribute(tok_sqstats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TOK_SMEM_BYTES) != cudaSuccess) {
-      cudaGetLastError();
-      return PE_ERR_CUDA;
+  {
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    if (!di->tok_attr_set) {
+      if (cudaFuncSetAttribute(tok_sqstats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TOK_SMEM_BYTES) != cudaSuccess) {
+        cudaGetLastError();
+        return PE_ERR_CUDA;
+      }
+      di->tok_attr_set = true;
     }
-    di->tok_attr_set = true;
   }
   TokParams p;
   p.rows = rows; p.d_in = d_in; p.d_out = d_out; p.pairs_m = pairs_m; p.tiles_n = tiles_n;
@@ -436,7 +462,7 @@ pe_status_t pe_example_sqnorms(const void* X, const void* dY, int B, int T, int 
   if (T == 0) return PE_OK;
   const int forced = g_path.load();
   const bool tc_ok = tc_shape_ok(B, T, d_in, d_out);
-  if ((forced == PE_PATH_TENSOR || forced == PE_PATH_TENSOR_NARROW) && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
+  if (forced >= PE_PATH_TENSOR && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
   if (tc_ok && forced != PE_PATH_SIMT) {
     g_last_path.store(PE_PATH_TENSOR);
     return launch_tc_norms(di, X, dY, B, T, d_in, d_out, out_norms, st);
@@ -495,7 +521,7 @@ pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_
   const int forced = g_path.load();
   const long long rows = (long long)B * T;
   const bool shape_ok = tc_shape_ok(B, T, d_in, d_out) && rows < (1ll << 31);
-  if ((forced == PE_PATH_TENSOR || forced == PE_PATH_TENSOR_NARROW) && !shape_ok) return PE_ERR_UNSUPPORTED_SHAPE;
+  if (forced >= PE_PATH_TENSOR && !shape_ok) return PE_ERR_UNSUPPORTED_SHAPE;
   if (shape_ok && rows >= TOKEN_TC_MIN_ROWS && forced != PE_PATH_SIMT) {
     g_last_path.store(PE_PATH_TENSOR);
     return launch_tok(di, X, dY, rows, d_in, d_out, out_stat, st);
@@ -549,7 +575,7 @@ pe_status_t pe_token_sqstats_staged(const void* X, const void* dY, int B, int T,
   if (B == 0 || T == 0) return zero_outputs(out_stat, nullptr, (size_t)d_in * d_out * sizeof(float), st);
   const int forced = g_path.load();
   const bool tc_ok = token_tc_ok(B, T, d_in, d_out);
-  if ((forced == PE_PATH_TENSOR || forced == PE_PATH_TENSOR_NARROW) && !tc_shape_ok(B, T, d_in, d_out)) return PE_ERR_UNSUPPORTED_SHAPE;
+  if (forced >= PE_PATH_TENSOR && !tc_shape_ok(B, T, d_in, d_out)) return PE_ERR_UNSUPPORTED_SHAPE;
   if (tc_ok && forced != PE_PATH_SIMT) {
     const long long rows = (long long)B * T;
     const StagedLayout l = staged_layout(B, T, d_in, d_out);
@@ -737,7 +763,7 @@ pe_status_t pe_get_async_status(pe_stream_t stream, int* detail) {
 }
 
 int pe_set_path(int path) {
-  if (path < PE_PATH_AUTO || path > PE_PATH_TENSOR_NARROW) return -1;
+  if (path < PE_PATH_AUTO || path > PE_PATH_TENSOR_WIDE) return -1;
   return g_path.exchange(path);
 }
 int pe_last_path(void) { return g_last_path.load(); }

@@ -11,6 +11,8 @@
 // 128 x 128 tile would need 128 B/clk at full tensor rate, a 256 x 128 pair 96, a 256 x 256 pair 64.
 //
 //   MEAN_REGS, NT = 128: two running sums per thread (64 + 64 registers)         -- both outputs, short sequences
+//   MEAN_REGS, NT = 192: two running sums per thread (96 + 96 registers; the control
+//                        warps shrink to 48 registers so that the epilogue warps can take 232) -- both outputs
 //   MEAN_REGS_SIGN, NT = 128: the same plus sum_b sign(G_b), counted in 16-bit halves
 //                        of 32 more registers                                      -- mean, square and sign in one pass
 //   MEAN_TMEM, NT = 256: sum_b phi(G_b) in 128 registers per thread, sum_b G_b in
@@ -53,7 +55,8 @@ constexpr int TC_THREADS = 384;
 constexpr int TC_REGS_CONTROL = 64;     // setmaxnreg of warps 0..3
 constexpr int TC_REGS_EPILOGUE = 216;   // setmaxnreg of warps 4..11  (4*32*64 + 8*32*216 = 63488 <= 65536)
 constexpr int TC_BAR_BYTES = 512;
-constexpr int TC_SMEM_BUDGET = 200 * 1024;   // operand ring; leaves room for barriers and alignment slack
+// operand ring; leaves room for barriers and alignment slack.  The 256 x 192 tile's four 56 KiB stages take 224 KiB.
+__host__ __device__ constexpr int tc_smem_budget(int nt) { return (nt == 192 ? 224 : 200) * 1024; }
 
 // Operand element type of the MMA.  bf16 (kind::f16, 16 tokens per instruction) for the per-example
 // statistics; tf32 (kind::tf32, fp32 storage, 8 tokens per instruction) for the per-token statistic,
@@ -61,7 +64,7 @@ constexpr int TC_SMEM_BUDGET = 200 * 1024;   // operand ring; leaves room for ba
 // Default tokens per pipeline stage: 128 for the 256 x 128 tile, 64 for the 256 x 256 tile, 32 for
 // tf32.  With both outputs and short sequences (T <= 32) the 256 x 128 tile takes 32-token stages
 // instead: a 128-token box would be mostly zero fill, and 16 small slots keep more examples in flight.
-__host__ __device__ constexpr int tc_default_bk(bool tf32, int nt) { return tf32 ? 32 : (nt == 128 ? 128 : 64); }
+__host__ __device__ constexpr int tc_default_bk(bool tf32, int nt) { return tf32 ? 32 : (nt == 256 ? 64 : 128); }
 constexpr int TC_SHORT_BK = 32;
 constexpr int TC_SHORT_T = 32;
 template <bool TF32, int NT, int BK_ = tc_default_bk(TF32, NT)>
@@ -76,19 +79,35 @@ struct TcOperand {
   static constexpr int BOX_BYTES = 128 * BK;                    // one box: BK tokens x 128 bytes
   static constexpr int A_BOXES = TC_TILE_M / BOX_FEATS;         // this block's 128 rows of dY^T
   static constexpr int B_FEATS = NT / 2;                        // this block's half of the tile's d_in columns
-  static constexpr int B_BOXES = B_FEATS / BOX_FEATS;
-  static constexpr int A_BYTES = A_BOXES * BOX_BYTES;           // 32 KiB (NT = 128) | 16 KiB
-  static constexpr int B_BYTES = B_BOXES * BOX_BYTES;           // 16 KiB
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;         // per block: 48 KiB | 32 KiB
-  static constexpr int STAGES = (TC_SMEM_BUDGET / STAGE_BYTES) & ~1;   // 4 | 6 | 16 with 32-token stages
+  // NT = 192: 96 columns of X per block are one and a half 128-byte rows.  X is then loaded in
+  // 64-byte rows (32 features per box, TMA SWIZZLE_64B) and described to the MMA with the 64-byte
+  // swizzle (descriptor layout 4: 8-token x 32-feature atoms of 512 bytes); dY keeps 128-byte rows.
+  static constexpr bool B_NARROW = (B_FEATS % BOX_FEATS) != 0;
+  static_assert(!B_NARROW || !TF32, "64-byte rows are only set up for 16-bit operands");
+  static constexpr int B_ROW_BYTES = B_NARROW ? 64 : 128;
+  static constexpr int B_BOX_FEATS = B_ROW_BYTES / ELEM_BYTES;  // 64 | 32
+  static constexpr int B_BOX_BYTES = B_ROW_BYTES * BK;
+  static constexpr int B_BOXES = B_FEATS / B_BOX_FEATS;         // 1 | 2 | 3
+  static constexpr int A_BYTES = A_BOXES * BOX_BYTES;           // 32 KiB (BK = 128) | 16 KiB
+  static constexpr int B_BYTES = B_BOXES * B_BOX_BYTES;         // 16 KiB | 24 KiB (NT = 192)
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;         // per block: 48 KiB | 56 KiB | 32 KiB
+  static constexpr int STAGES = (tc_smem_budget(NT) / STAGE_BYTES) & ~1;   // 4 | 4 | 6 | 16 with 32-token stages
   static_assert(STAGES % 2 == 0, "slots must alternate between the two issuers");
   static constexpr int K_STEP_BYTES = MMA_K * 128;              // smem advance per MMA: 2048 | 1024
-  static constexpr int ACC_BUFS = TC_TMEM_COLS / NT;            // 4 | 2 accumulators in tensor memory
+  static constexpr int B_K_STEP_BYTES = MMA_K * B_ROW_BYTES;
+  static constexpr int ACC_BUFS = TC_TMEM_COLS / NT;            // 4 | 2 | 2 accumulators in tensor memory
   // MN-major swizzle atoms: bf16 = 8 tokens x 128 B with 16-byte chunks (descriptor layout 2, TMA
   // SWIZZLE_128B); tf32 = 4 tokens x 128 B with 32-byte chunks (layout 1, TMA SWIZZLE_128B_ATOM_32B).
   static constexpr uint32_t DESC_LAYOUT = TF32 ? 1u : 2u;
   static constexpr uint32_t SBO_BYTES = TF32 ? 512u : 1024u;   // next swizzle atom along the tokens
+  static constexpr uint32_t B_DESC_LAYOUT = B_NARROW ? 4u : DESC_LAYOUT;
+  static constexpr uint32_t B_SBO_BYTES = B_NARROW ? 512u : SBO_BYTES;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + TC_BAR_BYTES + 1024;   // + alignment slack
+  // Register split between the four control warps and the eight epilogue warps (setmaxnreg; 128 * control
+  // + 256 * epilogue <= 65536).  Two running sums of 96 floats each need the larger epilogue share.
+  static constexpr int REGS_CONTROL = (NT == 192) ? 48 : TC_REGS_CONTROL;
+  static constexpr int REGS_EPILOGUE = (NT == 192) ? 232 : TC_REGS_EPILOGUE;
+  static_assert(128 * REGS_CONTROL + 256 * REGS_EPILOGUE <= 65536, "register file");
 };
 
 // error codes latched in the device status word (which wait gave up)
@@ -180,7 +199,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   using namespace sm100;
   using Op = TcOperand<TF32, NT, BKT>;
   constexpr bool TRIPLE = (MEAN == MEAN_REGS_SIGN);
-  static_assert((MEAN != MEAN_REGS && !TRIPLE) || NT == 128, "two running sums only fit the registers at NT = 128");
+  static_assert((MEAN != MEAN_REGS && !TRIPLE) || NT == 128 || (NT == 192 && !TRIPLE), "two running sums only fit the registers up to NT = 192");
+  static_assert(NT != 192 || MEAN == MEAN_REGS, "the 256 x 192 tile exists for the two register-resident sums");
   static_assert(!TRIPLE || PHI == 1, "the three-statistic mode is mean + square + sign");
   constexpr bool NORMS = (MEAN == MEAN_NORMS);
   static_assert(!NORMS || (PHI == 1 && NT == 256), "per-example norms: squares on the 256 x 256 tile");
@@ -228,7 +248,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   // read per thread; the producer / MMA warpgroup needs little.  Each setmaxnreg sits inside the
   // branch of the role it applies to.
   if (warp < 4) {
-    setmaxnreg_dec<TC_REGS_CONTROL>();
+    setmaxnreg_dec<Op::REGS_CONTROL>();
     if (warp == 0 || warp == 2) {
       // ---------------------------------------------------------- TMA producers (both blocks)
       // Warp 0 loads this block's rows of dY^T (and, in the leader, posts the stage's byte count);
@@ -243,6 +263,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         const CUtensorMap* tmap = is_a ? &tmap_dy : &tmap_x;
         const int c0 = is_a ? tile_m * TC_TILE_M : tile_n * NT + (int)rank * Op::B_FEATS;   // first feature of this warp's boxes
         const int n_boxes = is_a ? Op::A_BOXES : Op::B_BOXES;
+        const int box_feats = is_a ? Op::BOX_FEATS : Op::B_BOX_FEATS;
+        const int box_bytes = is_a ? BOX_BYTES : Op::B_BOX_BYTES;
         prefetch_tensormap(tmap);
         int s = 0; uint32_t ph = 0;
         for (StageWalk<ISSUERS> cur(nb, nk); cur.valid(); cur.next()) {
@@ -252,7 +274,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             const uint32_t leader_full = map_to_cta(full_bar(s), 0);
             const uint32_t dst = smem_base + s * STAGE_BYTES + (is_a ? 0 : A_BYTES);
             for (int g = 0; g < n_boxes; ++g)
-              tma_load_3d_pair(dst + g * BOX_BYTES, tmap, leader_full, c0 + g * Op::BOX_FEATS, cur.kc * BK, b_begin + cur.e());
+              tma_load_3d_pair(dst + g * box_bytes, tmap, leader_full, c0 + g * box_feats, cur.kc * BK, b_begin + cur.e());
           }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
@@ -299,7 +321,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
               // rows past T are zero-filled by TMA; whole MMA steps past T are skipped
               if (k * Op::MMA_K < t_left) {
                 const uint64_t ad = make_smem_desc(a_src + k * Op::K_STEP_BYTES, BOX_BYTES, Op::SBO_BYTES, Op::DESC_LAYOUT);
-                const uint64_t bd = make_smem_desc(b_src + k * Op::K_STEP_BYTES, BOX_BYTES, Op::SBO_BYTES, Op::DESC_LAYOUT);
+                const uint64_t bd = make_smem_desc(b_src + k * Op::B_K_STEP_BYTES, Op::B_BOX_BYTES, Op::B_SBO_BYTES, Op::B_DESC_LAYOUT);
                 umma_ss_pair<TF32>(d_tmem, ad, bd, idesc, accumulate);
                 accumulate = 1;
               }
@@ -314,7 +336,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     }
   } else {
     // ------------------------------------------------------------ epilogue (both blocks)
-    setmaxnreg_inc<TC_REGS_EPILOGUE>();
+    setmaxnreg_inc<Op::REGS_EPILOGUE>();
     const int q = warp & 3;                 // TMEM lane quadrant this warp may access
     const int h = (warp - 4) >> 2;          // column half of the tile
     constexpr bool KEEP_MEAN = MEAN == MEAN_REGS || TRIPLE || PHI == 0;     // running sum of G_b in registers
@@ -341,7 +363,9 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       const int x = a % ISSUERS, grp = p.per_example ? (a / ISSUERS) : 0;
       const int buf = BUFS_PER_ISSUER * x + (grp % BUFS_PER_ISSUER);
       const uint32_t acc_ph = (uint32_t)(grp / BUFS_PER_ISSUER) & 1u;
-      if (!mbar_wait_bounded(acc_full_bar(buf), acc_ph, abort_flag, p.dev_status, TC_WAIT_ACC_FULL)) { ok = false; break; }
+      // every lane polls, but the warp acts on one answer: the tensor-memory loads below are warp-wide
+      // instructions, so no lane may leave the loop alone when its own wait is the one that gives up
+      if (!__all_sync(0xffffffffu, mbar_wait_bounded(acc_full_bar(buf), acc_ph, abort_flag, p.dev_status, TC_WAIT_ACC_FULL))) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = lane_base + (uint32_t)(buf * NT + h * COLS);
       if constexpr (MEAN == MEAN_TMEM) {
@@ -395,41 +419,44 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
         if (lane == 0) atomicAdd(p.out_norms + b_begin + a, s);
       } else {
+        // CH columns per tensor-memory read: 32, or 16 where the two running sums leave few registers (NT = 192)
+        constexpr int CH = (NT == 192) ? 16 : 32;
 #pragma unroll
-        for (int c = 0; c < COLS / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld_32x32b_x32_wait(taddr + c * 32, r);
-          if (c == COLS / 32 - 1) {
+        for (int c = 0; c < COLS / CH; ++c) {
+          uint32_t r[CH];
+          if constexpr (CH == 32) tmem_ld_32x32b_x32_wait(taddr + c * CH, r);
+          else tmem_ld_32x32b_x16_wait(taddr + c * CH, r);
+          if (c == COLS / CH - 1) {
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));   // buffer free for the issuer's next example
           }
           if constexpr (PHI == 2) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
+            for (int j = 0; j < CH; ++j) {
               const float g = __uint_as_float(r[j]);
-              if (KEEP_MEAN) acc_mean[c * 32 + j] += g;
-              acc_stat[c * 32 + j] += phi_apply<PHI>(g);
+              if (KEEP_MEAN) acc_mean[c * CH + j] += g;
+              acc_stat[c * CH + j] += phi_apply<PHI>(g);
             }
           } else {
             // two columns per instruction: packed fp32 add for sum_b G_b, packed fma for sum_b G_b^2
 #pragma unroll
-            for (int j = 0; j < 32; j += 2) {
+            for (int j = 0; j < CH; j += 2) {
               const uint64_t g2 = f32x2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
               if (KEEP_MEAN) {
-                const uint64_t m2 = f32x2_add(f32x2_pack(acc_mean[c * 32 + j], acc_mean[c * 32 + j + 1]), g2);
-                f32x2_unpack(m2, acc_mean[c * 32 + j], acc_mean[c * 32 + j + 1]);
+                const uint64_t m2 = f32x2_add(f32x2_pack(acc_mean[c * CH + j], acc_mean[c * CH + j + 1]), g2);
+                f32x2_unpack(m2, acc_mean[c * CH + j], acc_mean[c * CH + j + 1]);
               }
               if (PHI == 1) {
-                const uint64_t s2 = f32x2_fma(g2, g2, f32x2_pack(acc_stat[c * 32 + j], acc_stat[c * 32 + j + 1]));
-                f32x2_unpack(s2, acc_stat[c * 32 + j], acc_stat[c * 32 + j + 1]);
+                const uint64_t s2 = f32x2_fma(g2, g2, f32x2_pack(acc_stat[c * CH + j], acc_stat[c * CH + j + 1]));
+                f32x2_unpack(s2, acc_stat[c * CH + j], acc_stat[c * CH + j + 1]);
               }
               if (TRIPLE) {
                 // sign(g) as a float, plus 2^23 * 1.5 + 1: the low 16 bits of the sum's bit pattern are
                 // sign(g) + 1 in {0, 1, 2}; one byte permute packs the two columns' low halves
                 const float t0 = phi_apply<2>(__uint_as_float(r[j])) + 12582913.f;
                 const float t1 = phi_apply<2>(__uint_as_float(r[j + 1])) + 12582913.f;
-                acc_cnt[(c * 32 + j) >> 1] += __byte_perm(__float_as_uint(t0), __float_as_uint(t1), 0x5410);
+                acc_cnt[(c * CH + j) >> 1] += __byte_perm(__float_as_uint(t0), __float_as_uint(t1), 0x5410);
               }
             }
           }
@@ -447,7 +474,10 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       constexpr int PANELS = COLS / 32;
       int tile_m, tile_n;
       tc_tile_of_block(p, rank, tile_m, tile_n);
-      const uint32_t stage_base = smem_base + (uint32_t)(warp - 4) * (4u * 4096u);     // 16 KiB per epilogue warp
+      // each epilogue warp stages in its own eighth of the operand ring: 6 panels of 4 KiB (7 at NT = 192)
+      constexpr int WARP_PANELS = (STAGES * STAGE_BYTES / 8) / 4096;
+      static_assert(WARP_PANELS >= PANELS, "an epilogue warp stages one output at a time");
+      const uint32_t stage_base = smem_base + (uint32_t)(warp - 4) * (uint32_t)(WARP_PANELS * 4096);
       const int row0 = tile_m * TC_TILE_M + q * 32;
       const int col0 = tile_n * NT + h * COLS;
       auto put_panel = [&](uint32_t panel_addr, const float* v) {      // v: this lane's 32 consecutive columns
@@ -480,7 +510,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       if (p.out_mean && (KEEP_MEAN || MEAN == MEAN_TMEM)) {
         uint32_t first = stage_base + PANELS * 4096;          // MEAN_REGS / PHI == 0: second half of the warp's 16 KiB
         if constexpr (MEAN == MEAN_TMEM) {
-          // all 16 KiB are needed again: wait until TMA has read the first output out of them
+          // the panels are needed again: wait until TMA has read the first output out of them
           if (lane == 0) bulk_wait_read_all();
           __syncwarp();
           first = stage_base;
@@ -492,7 +522,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             put_panel(first + c * 4096, reinterpret_cast<const float*>(m));
           }
         } else if constexpr (KEEP_MEAN) {
-          if constexpr (PANELS * 2 * 4096 > 4 * 4096) {       // PHI == 0 at NT = 256: one output only ever
+          if constexpr (PANELS * 2 > WARP_PANELS) {           // PHI == 0 at NT = 256: one output only ever
             if (lane == 0) bulk_wait_read_all();
             __syncwarp();
             first = stage_base;
@@ -503,7 +533,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         send(&tmap_mean, first);
       }
       if constexpr (TRIPLE) {
-        // sum_b sign(G_b): the warp's 16 KiB are in use, so wait until TMA has read them
+        // sum_b sign(G_b): the warp's staging area is in use, so wait until TMA has read it
         if (p.out_sign) {
           if (lane == 0) bulk_wait_read_all();
           __syncwarp();

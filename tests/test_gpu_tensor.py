@@ -103,6 +103,32 @@ def test_register_mean_kernel_at_any_sequence_length(B, T, d_in, d_out):
     assert pe.pe_last_path() == pe.PATH_TENSOR
 
 
+def test_wide_tile_structured_inputs_catch_layout_mistakes():
+    """The 256 x 192 tile loads X in 64-byte rows with the 64-byte swizzle.  Distinct small integers per
+    (token, feature), exactly representable in bf16: a wrong swizzle, stride or column offset of that
+    layout changes results by whole numbers.  d_in = 400 spans three 192-column tiles, the last ragged."""
+    pe.pe_set_path(pe.PATH_TENSOR_WIDE)
+    B, T, d_in, d_out = 3, 144, 400, 264
+    t = torch.arange(T, dtype=torch.float32).view(1, T, 1)
+    X = ((t % 5) - 2 + (torch.arange(d_in).view(1, 1, d_in) % 13 - 6) + torch.arange(B).view(B, 1, 1)).to(torch.bfloat16)
+    dY = ((t % 3) - 1 + (torch.arange(d_out).view(1, 1, d_out) % 11 - 5) * 0.5 - torch.arange(B).view(B, 1, 1)).to(torch.bfloat16)
+    li = inputs.LayerInputs("structured", X.to(DEV).contiguous(), dY.to(DEV).contiguous())
+    rep = check_all(li, phis=("square", "sign"), token=False, tol=1e-6)
+    assert pe.pe_last_path() == pe.PATH_TENSOR
+    assert rep["sign_disagreements"] == 0
+
+
+@pytest.mark.parametrize("B,T,d_in,d_out", [(5, 200, 136, 264), (40, 96, 384, 256), (3, 2000, 264, 520), (7, 128, 192, 512),
+                                            (9, 16, 320, 192), (2, 1, 64, 72), (70, 48, 8, 8), (33, 300, 776, 264)])
+def test_wide_tile_kernel_at_any_shape(B, T, d_in, d_out):
+    """The 256 x 192 kernel (both running sums in registers, 96 columns per thread), forced on shapes
+    with ragged 192-column tiles, short and long sequences and split batches."""
+    pe.pe_set_path(pe.PATH_TENSOR_WIDE)
+    li = inputs.gaussian_layer(B, T, d_in, d_out, seed=1500 + T, device=DEV)
+    check_all(li, phis=("square", "sign"), token=False)
+    assert pe.pe_last_path() == pe.PATH_TENSOR
+
+
 @pytest.mark.parametrize("B,T,d_in,d_out", [(5, 200, 136, 264), (64, 64, 512, 256), (3, 1000, 520, 776), (1, 257, 8, 8), (16, 512, 1024, 1024)])
 def test_token_stat_fused_staged_and_oracle_agree(B, T, d_in, d_out):
     """The one-kernel per-token statistic, the two-pass one and the oracle give the same matrix; the two
