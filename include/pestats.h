@@ -49,11 +49,12 @@ typedef enum { PE_PHI_IDENTITY = 0, PE_PHI_SQUARE = 1, PE_PHI_SIGN = 2 } pe_phi_
 
 /* Which kernel family a call may use.  AUTO picks the tensor-core kernel whenever the shape allows
  * it (bf16 inputs, d_in % 8 == 0, d_out % 8 == 0) and the SIMT kernel otherwise.  When both outputs
- * are wanted AUTO and TENSOR keep both running sums in registers on a 256 x 128 tile for T < 256, on a
- * 256 x 192 tile for 256 <= T < 4096 (unless d_in pads badly to multiples of 192), and from T = 4096 on
- * keep sum_b G_b in tensor memory beside a 256 x 256 tile.  TENSOR_NARROW is TENSOR with the 256 x 128
- * tile and TENSOR_WIDE is TENSOR with the 256 x 192 tile, both at any T; they exist so that tests can
- * reach those kernels on every shape. */
+ * are wanted AUTO and TENSOR keep both running sums in registers: on a 256 x 192 tile for T >= 64 when
+ * d_in rounded up to a multiple of 192 is at most 13 % above d_in rounded up to a multiple of 128, else
+ * on a 256 x 128 tile, except that from T = 4096 on those remaining shapes keep sum_b G_b in tensor
+ * memory beside a 256 x 256 tile.  TENSOR_NARROW is TENSOR with the 256 x 128 tile and TENSOR_WIDE is
+ * TENSOR with the 256 x 192 tile, both at any T; they exist so that tests can reach those kernels on
+ * every shape. */
 typedef enum { PE_PATH_AUTO = 0, PE_PATH_SIMT = 1, PE_PATH_TENSOR = 2, PE_PATH_TENSOR_NARROW = 3, PE_PATH_TENSOR_WIDE = 4 } pe_path_t;
 
 typedef struct CUstream_st* pe_stream_t; /* a cudaStream_t */

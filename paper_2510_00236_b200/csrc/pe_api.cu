@@ -28,9 +28,12 @@ static std::atomic<long long> g_launches{0};
 // Both outputs: from this sequence length on the running sum of G_b lives in tensor memory beside a
 // 256-column accumulator (measured: wins or ties at T = 4096, loses 16 % at T = 2048, 17 % at T = 1024).
 constexpr int TC_MEAN_TMEM_MIN_T = 4096;
-// Both outputs, phi = square or sign: from this sequence length on (and below TC_MEAN_TMEM_MIN_T) the pair
-// tile is 256 x 192 instead of 256 x 128, unless d_in is so narrow that the wider tile's padding eats the gain.
-constexpr int TC_WIDE_MIN_T = 256;
+// Both outputs, phi = square or sign: from this sequence length on the pair tile is 256 x 192 instead of
+// 256 x 128 (measured: ties at T = 64 and 128, 3-21 % faster from T = 256 on, 17-25 % faster than the
+// tensor-memory mean at T = 4096; 18-22 % slower at T = 32), unless d_in is so narrow that the wider
+// tile's padding (columns up to the next multiple of 192) eats the gain.
+constexpr int TC_WIDE_MIN_T = 64;
+constexpr int TC_WIDE_MAX_PAD_PERCENT = 13;
 constexpr int TC_BAND = 8;          // pair rows per band of the tile order (8 x 256 rows of d_out)
 
 constexpr int MAX_DEVICES = 64;
@@ -227,11 +230,11 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   // Both outputs: sum_b G_b in tensor memory beside a 256-wide accumulator, unless the sequences are
   // so short that the per-example drain of that single accumulator would dominate.
   const int forced = g_path.load();
-  const bool mean_regs = both && (triple || T < TC_MEAN_TMEM_MIN_T || forced == PE_PATH_TENSOR_NARROW || forced == PE_PATH_TENSOR_WIDE);
-  // 256 x 192 tile: a third less operand traffic per flop than 256 x 128; its column padding must stay below ~7 %
+  // 256 x 192 tile: 22 % less operand traffic per flop than 256 x 128
   const long long pad192 = (long long)((d_in + 191) / 192) * 192, pad128 = (long long)((d_in + 127) / 128) * 128;
-  const bool wide = mean_regs && !triple && forced != PE_PATH_TENSOR_NARROW &&
-                    (forced == PE_PATH_TENSOR_WIDE || (T >= TC_WIDE_MIN_T && pad192 * 100 <= pad128 * 107));
+  const bool wide = both && !triple && forced != PE_PATH_TENSOR_NARROW &&
+                    (forced == PE_PATH_TENSOR_WIDE || (T >= TC_WIDE_MIN_T && pad192 * 100 <= pad128 * (100 + TC_WIDE_MAX_PAD_PERCENT)));
+  const bool mean_regs = both && (triple || wide || T < TC_MEAN_TMEM_MIN_T || forced == PE_PATH_TENSOR_NARROW);
   const int nt = mean_regs ? (wide ? 192 : 128) : 256;
   const int box_feats = TcOperand<false, 256>::BOX_FEATS;
   const bool short_seq = mean_regs && !wide && !triple && T <= TC_SHORT_T;      // many short examples, both outputs: small stages

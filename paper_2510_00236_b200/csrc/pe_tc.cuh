@@ -53,7 +53,8 @@ constexpr int TC_PAIR_M = 2 * TC_TILE_M;
 constexpr int TC_TMEM_COLS = 512;
 constexpr int TC_THREADS = 384;
 constexpr int TC_REGS_CONTROL = 64;     // setmaxnreg of warps 0..3
-constexpr int TC_REGS_EPILOGUE = 216;   // setmaxnreg of warps 4..11  (4*32*64 + 8*32*216 = 63488 <= 65536)
+constexpr int TC_REGS_EPILOGUE = 216;   // setmaxnreg of warps 4..11  (4*32*64 + 8*32*216 = 63488 <= 384*168)
+constexpr int TC_REGS_AT_LAUNCH = 168;  // registers per thread of a 384-thread block at one block per SM (65536 / 384, in eights)
 constexpr int TC_BAR_BYTES = 512;
 // operand ring; leaves room for barriers and alignment slack.  The 256 x 192 tile's four 56 KiB stages take 224 KiB.
 __host__ __device__ constexpr int tc_smem_budget(int nt) { return (nt == 192 ? 224 : 200) * 1024; }
@@ -103,11 +104,13 @@ struct TcOperand {
   static constexpr uint32_t B_DESC_LAYOUT = B_NARROW ? 4u : DESC_LAYOUT;
   static constexpr uint32_t B_SBO_BYTES = B_NARROW ? 512u : SBO_BYTES;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + TC_BAR_BYTES + 1024;   // + alignment slack
-  // Register split between the four control warps and the eight epilogue warps (setmaxnreg; 128 * control
-  // + 256 * epilogue <= 65536).  Two running sums of 96 floats each need the larger epilogue share.
-  static constexpr int REGS_CONTROL = (NT == 192) ? 48 : TC_REGS_CONTROL;
+  // Register split between the four control warps and the eight epilogue warps (setmaxnreg).  The pool
+  // is what the block was launched with, 384 threads x 168 registers, NOT the SM's whole register file: an
+  // increase that the decreases of the control warps do not cover never returns.  Two running sums of
+  // 96 floats each need the larger epilogue share.
+  static constexpr int REGS_CONTROL = (NT == 192) ? 40 : TC_REGS_CONTROL;
   static constexpr int REGS_EPILOGUE = (NT == 192) ? 232 : TC_REGS_EPILOGUE;
-  static_assert(128 * REGS_CONTROL + 256 * REGS_EPILOGUE <= 65536, "register file");
+  static_assert(128 * REGS_CONTROL + 256 * REGS_EPILOGUE <= TC_THREADS * TC_REGS_AT_LAUNCH, "setmaxnreg: the epilogue's increase must fit what the control warps give up");
 };
 
 // error codes latched in the device status word (which wait gave up)

@@ -46,7 +46,8 @@ def test_structured_single_tile_catches_layout_mistakes():
     (21, 64, 136, 520),     # half-filled stages
     (11, 33, 128, 256),     # just above the short-stage limit
     (13, 32, 264, 136),     # exactly one short stage per example
-    (2, 4100, 136, 264),    # very long sequences: sum_b G_b kept in tensor memory when both outputs are wanted
+    (2, 4100, 136, 264),    # very long sequences on the 256 x 192 tile
+    (2, 4100, 200, 264),    # d_in pads badly to 192: sum_b G_b kept in tensor memory beside a 256 x 256 tile
 ])
 def test_tensor_small_shapes_full_comparison(B, T, d_in, d_out):
     li = inputs.gaussian_layer(B, T, d_in, d_out, seed=300 + 7 * B + T, device=DEV)
