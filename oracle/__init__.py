@@ -73,6 +73,16 @@ def _load():
             c_double_p, c_double_p, c_double_p, ctypes.c_longlong, ctypes.c_int, ctypes.c_double,
             ctypes.c_double, ctypes.c_double,
         ]
+        lib.oracle_linear_stats_ragged.restype = ctypes.c_int
+        lib.oracle_linear_stats_ragged.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_longlong), ctypes.c_int,
+            ctypes.c_int, ctypes.c_double, c_double_p, c_double_p, c_double_p, c_double_p, c_int32_p, c_double_p,
+        ]
+        lib.oracle_clipped_sum.restype = ctypes.c_int
+        lib.oracle_clipped_sum.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+            ctypes.c_double, c_double_p, c_double_p, c_double_p,
+        ]
         lib.oracle_num_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -144,6 +154,59 @@ def example_sqnorms(X: np.ndarray, dY: np.ndarray) -> np.ndarray:
     if rc != 0:
         raise RuntimeError("oracle_example_sqnorms failed")
     return out
+
+
+@dataclass
+class RaggedStats(LinearStats):
+    """Outputs of :func:`linear_stats_ragged`: those of :class:`LinearStats` plus ``sq_norms`` [B]."""
+    sq_norms: np.ndarray = None
+
+
+def linear_stats_ragged(X: np.ndarray, dY: np.ndarray, offsets, small_rel: float = 1e-3) -> RaggedStats:
+    """Per-example statistics of a packed batch (Section 2.3; Eq. (2)): X [rows, d_in], dY [rows, d_out],
+    example b owns rows offsets[b] .. offsets[b+1]-1 and its gradient is contracted over those rows only."""
+    if X.dtype != dY.dtype or X.dtype not in (np.float32, np.uint16):
+        raise TypeError("X and dY must both be float32, or both uint16 (bf16 bit patterns)")
+    if X.ndim != 2 or dY.ndim != 2 or X.shape[0] != dY.shape[0]:
+        raise ValueError("X must be [rows, d_in] and dY [rows, d_out] with the same row count")
+    offs = np.ascontiguousarray(np.asarray(offsets, np.int64))
+    if offs.ndim != 1 or offs.size < 1 or (offs.size > 1 and offs[-1] > X.shape[0]):
+        raise ValueError("offsets must be [B+1] and end within the rows")
+    B = offs.size - 1
+    X = np.ascontiguousarray(X)
+    dY = np.ascontiguousarray(dY)
+    d_in, d_out = X.shape[1], dY.shape[1]
+    sg = np.empty((d_out, d_in), np.float64)
+    sg2 = np.empty((d_out, d_in), np.float64)
+    ss = np.empty((d_out, d_in), np.float64)
+    mx = np.zeros((max(B, 1),), np.float64)
+    nr = np.zeros((max(B, 1),), np.float64)
+    ns = np.empty((d_out, d_in), np.int32)
+    rc = _load().oracle_linear_stats_ragged(
+        X.ctypes.data, dY.ctypes.data, int(X.dtype == np.uint16), B, offs.ctypes.data_as(ctypes.POINTER(ctypes.c_longlong)),
+        d_in, d_out, float(small_rel), _dp(sg), _dp(sg2), _dp(ss), _dp(mx), ns.ctypes.data_as(c_int32_p), _dp(nr))
+    if rc != 0:
+        raise RuntimeError("oracle_linear_stats_ragged failed")
+    return RaggedStats(sg, sg2, ss, mx[:B], ns, nr[:B])
+
+
+def clipped_sum(X: np.ndarray, dY: np.ndarray, clip_norm: float, sq_norms=None):
+    """Sum over examples of the norm-clipped per-example gradients, c_b = min(1, C / sqrt(N_b)) (Section 2.1's
+    clipping statistic with Section 2.3's squared norms N_b).  sq_norms: optional [B] squared norms to clip
+    by (default: this layer's own).  Returns (sum [d_out, d_in], coefficients [B])."""
+    X, dY, is_bf16, B, T, d_in, d_out = _check_inputs(X, dY)
+    out = np.empty((d_out, d_in), np.float64)
+    coef = np.zeros((max(B, 1),), np.float64)
+    nin = None
+    if sq_norms is not None:
+        nin = np.ascontiguousarray(np.asarray(sq_norms, np.float64))
+        if nin.shape != (B,):
+            raise ValueError("sq_norms must be [B]")
+    rc = _load().oracle_clipped_sum(X.ctypes.data, dY.ctypes.data, is_bf16, B, T, d_in, d_out, float(clip_norm),
+                                    _dp(nin), _dp(out), _dp(coef))
+    if rc != 0:
+        raise RuntimeError("oracle_clipped_sum failed")
+    return out, coef[:B]
 
 
 def microadam_step(theta, m, v, sum_g, sum_g2, B, *, grad_scale=1.0, lr, beta1, beta2, eps,

@@ -264,6 +264,116 @@ int oracle_microsignsgd_step(double* theta, double* m, const double* sum_sgn, lo
   return 0;
 }
 
+/*
+ * Sequence-level per-example statistics of a PACKED (ragged) batch: the same definition as
+ * oracle_linear_stats (Section 2.3; Eq. (2)), but example b owns the token rows
+ * offsets[b] .. offsets[b+1]-1 of X [rows, d_in] and dY [rows, d_out], so every gradient is contracted
+ * over its own sequence's tokens, however many those are:
+ *     G_b[o,i] = sum_{r = offsets[b]}^{offsets[b+1]-1} dY[r,o] * X[r,i].
+ * An empty sequence has G_b = 0 (and sign(0) = 0).  offsets must be non-decreasing with offsets[0] >= 0.
+ * Outputs as in oracle_linear_stats; sq_norms [B] (may be NULL) receives ||G_b||_F^2.
+ */
+int oracle_linear_stats_ragged(const void* X, const void* dY, int is_bf16, int B, const long long* offsets,
+                               int d_in, int d_out, double small_rel, double* sum_g, double* sum_g2,
+                               double* sum_sgn, double* max_abs, int32_t* n_small, double* sq_norms) {
+  if (!X || !dY || !offsets || B < 0 || d_in <= 0 || d_out <= 0) return 1;
+  if (B > 0 && offsets[0] < 0) return 1;
+  for (int b = 0; b < B; ++b) if (offsets[b + 1] < offsets[b]) return 1;
+  long long n = (long long)d_out * d_in;
+  double* G = (double*)malloc(sizeof(double) * (size_t)n);
+  if (!G) return 1;
+  for (long long k = 0; k < n; ++k) {
+    if (sum_g) sum_g[k] = 0.0;
+    if (sum_g2) sum_g2[k] = 0.0;
+    if (sum_sgn) sum_sgn[k] = 0.0;
+    if (n_small) n_small[k] = 0;
+  }
+  for (int b = 0; b < B; ++b) {
+    long long r0 = offsets[b], len = offsets[b + 1] - offsets[b];
+    double* xb = (double*)malloc(sizeof(double) * (size_t)((len > 0 ? len : 1) * d_in));
+    double* yb = (double*)malloc(sizeof(double) * (size_t)((len > 0 ? len : 1) * d_out));
+    if (!xb || !yb) { free(xb); free(yb); free(G); return 1; }
+    widen_rows(X, is_bf16, r0, len, d_in, xb);
+    widen_rows(dY, is_bf16, r0, len, d_out, yb);
+#pragma omp parallel for schedule(static)
+    for (int o = 0; o < d_out; ++o) {
+      double* g = G + (long long)o * d_in;
+      for (int i = 0; i < d_in; ++i) g[i] = 0.0;
+      for (long long t = 0; t < len; ++t) {
+        double lam = yb[t * d_out + o];
+        const double* h = xb + t * d_in;
+        for (int i = 0; i < d_in; ++i) g[i] += lam * h[i];
+      }
+    }
+    free(xb); free(yb);
+    double mx = 0.0, nrm = 0.0;
+    for (long long k = 0; k < n; ++k) {
+      double a = fabs(G[k]);
+      if (a > mx) mx = a;
+      nrm += G[k] * G[k];
+    }
+    if (max_abs) max_abs[b] = mx;
+    if (sq_norms) sq_norms[b] = nrm;
+    for (long long k = 0; k < n; ++k) {
+      double g = G[k];
+      if (sum_g) sum_g[k] += g;
+      if (sum_g2) sum_g2[k] += g * g;
+      if (sum_sgn) sum_sgn[k] += sign3(g);
+      if (n_small && fabs(g) <= small_rel * mx) n_small[k] += 1;
+    }
+  }
+  free(G);
+  return 0;
+}
+
+/*
+ * Sum of norm-clipped per-example gradients (Section 2.1 lists clipping among the statistics
+ * E[phi(grad f)] of Eq. (2); Section 2.3's "ghost clipping" remark names the per-example squared norms
+ * N_b it needs).  The paper does not spell the clipping function out; the standard per-example L2
+ * clipping is taken:
+ *     c_b = min(1, C / sqrt(N_b)),      out[o,i] = sum_b c_b * G_b[o,i],      G_b = dY_b^T X_b,
+ * with N_b = ||G_b||_F^2 of THIS layer when sq_norms_in is NULL, or the caller's numbers otherwise (a
+ * model-wide clip passes the squared norms summed over all layers).  N_b = 0 gives c_b = 1.  The 1/B
+ * of the mean is left to the caller, as everywhere else.  coef [B] (may be NULL) receives c_b.
+ */
+int oracle_clipped_sum(const void* X, const void* dY, int is_bf16, int B, int T, int d_in, int d_out,
+                       double clip_norm, const double* sq_norms_in, double* out, double* coef) {
+  if (!X || !dY || !out || B < 0 || T < 0 || d_in <= 0 || d_out <= 0 || !(clip_norm >= 0.0)) return 1;
+  long long n = (long long)d_out * d_in;
+  double* G = (double*)malloc(sizeof(double) * (size_t)n);
+  double* xb = (double*)malloc(sizeof(double) * (size_t)((long long)(T > 0 ? T : 1) * d_in));
+  double* yb = (double*)malloc(sizeof(double) * (size_t)((long long)(T > 0 ? T : 1) * d_out));
+  if (!G || !xb || !yb) { free(G); free(xb); free(yb); return 1; }
+  for (long long k = 0; k < n; ++k) out[k] = 0.0;
+  for (int b = 0; b < B; ++b) {
+    widen_rows(X, is_bf16, (long long)b * T, T, d_in, xb);
+    widen_rows(dY, is_bf16, (long long)b * T, T, d_out, yb);
+#pragma omp parallel for schedule(static)
+    for (int o = 0; o < d_out; ++o) {
+      double* g = G + (long long)o * d_in;
+      for (int i = 0; i < d_in; ++i) g[i] = 0.0;
+      for (int t = 0; t < T; ++t) {
+        double lam = yb[(long long)t * d_out + o];
+        const double* h = xb + (long long)t * d_in;
+        for (int i = 0; i < d_in; ++i) g[i] += lam * h[i];
+      }
+    }
+    double nb;
+    if (sq_norms_in) {
+      nb = sq_norms_in[b];
+    } else {
+      nb = 0.0;
+      for (long long k = 0; k < n; ++k) nb += G[k] * G[k];
+    }
+    double norm = sqrt(nb);
+    double c = (norm > clip_norm) ? clip_norm / norm : 1.0;
+    if (coef) coef[b] = c;
+    for (long long k = 0; k < n; ++k) out[k] += c * G[k];
+  }
+  free(G); free(xb); free(yb);
+  return 0;
+}
+
 /* Number of OpenMP threads the loops above will use (1 when built without OpenMP). */
 #ifdef _OPENMP
 #include <omp.h>
