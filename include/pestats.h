@@ -88,11 +88,53 @@ pe_status_t pe_linear_stats_f32(const float* X, const float* dY, int B, int T, i
  * bf16 inputs as for pe_linear_stats; out_norms: fp32 [B], 4-byte aligned, overwritten (may be NULL
  * only if B = 0).  Each G_b tile is formed on chip, squared and reduced there; every tile adds its
  * share to out_norms[b] with an fp32 atomic, so the result is reproducible only to rounding.  A
- * clipped batch gradient is then sum_b c_b G_b with c_b = min(1, C / sqrt(N_b)): scale the rows of dY
- * by c_b and run the ordinary weight-gradient contraction (pe_linear_stats with phi = identity).
+ * clipped batch gradient is then sum_b c_b G_b with c_b = min(1, C / sqrt(N_b)): pe_linear_clipped_sum.
  */
 pe_status_t pe_example_sqnorms(const void* X, const void* dY, int B, int T, int d_in, int d_out,
                                float* out_norms, pe_stream_t stream);
+
+/*
+ * pe_linear_stats for a PACKED batch of sequences of different lengths (Section 2.3: the per-example
+ * gradient of a sequence-level dense layer is the contraction over THAT sequence's tokens; Eq. (2)).
+ * X is [total_rows, d_in] and dY [total_rows, d_out] (bf16, 16-byte aligned); example b owns the token
+ * rows seq_offsets[b] .. seq_offsets[b+1]-1, so
+ *     G_b[o,i] = sum_{r in example b} dY[r,o] * X[r,i],   out_mean = sum_b G_b,   out_stat = sum_b phi(G_b).
+ * seq_offsets: DEVICE array of B+1 int32, 4-byte aligned, non-decreasing, 0 <= seq_offsets[0],
+ * seq_offsets[B] <= total_rows < 2^31 (it is read by the kernels only, so a producer on the same stream
+ * may still be writing it when this call returns).  An empty sequence contributes nothing.  Offsets
+ * that break these rules give unspecified statistics but never an access outside the tensors.
+ * workspace: device memory, 256-byte aligned, at least pe_linear_stats_ragged_workspace_bytes(B, d_in,
+ * d_out) bytes (32 * B * (d_in + d_out) bytes plus padding), contents undefined afterwards: the tensor-core
+ * kernel contracts 16 tokens per instruction, and a pre-pass copies every sequence's last len % 16
+ * tokens there, zero-padded to 16.  The SIMT path (widths not multiples of 8, or forced) ignores it.
+ * Outputs and phi as for pe_linear_stats; B == 0 or total_rows == 0 writes zeros.
+ */
+pe_status_t pe_linear_stats_ragged(const void* X, const void* dY, const int* seq_offsets, int B,
+                                   long long total_rows, int d_in, int d_out, pe_phi_t phi, float* out_mean,
+                                   float* out_stat, void* workspace, size_t workspace_bytes, pe_stream_t stream);
+/* Bytes of workspace the packed-batch calls need under the current path setting (0 on the SIMT path). */
+size_t pe_linear_stats_ragged_workspace_bytes(int B, int d_in, int d_out);
+/* pe_example_sqnorms for a packed batch (same layout, offsets and workspace as pe_linear_stats_ragged):
+ * out_norms[b] = ||G_b||_F^2 (Section 2.3). */
+pe_status_t pe_example_sqnorms_ragged(const void* X, const void* dY, const int* seq_offsets, int B,
+                                      long long total_rows, int d_in, int d_out, float* out_norms,
+                                      void* workspace, size_t workspace_bytes, pe_stream_t stream);
+
+/*
+ * Sum of norm-clipped per-example gradients (Section 2.1 lists clipping among the statistics
+ * E[phi(grad f)] of Eq. (2); Section 2.3 names the per-example squared norms N_b it needs).  The paper
+ * does not spell the function out; per-example L2 clipping is taken:
+ *     c_b = min(1, clip_norm / sqrt(N_b)),     out_sum[o,i] = sum_b c_b * G_b[o,i],     G_b = dY_b^T X_b
+ * (not divided by B).  sq_norms: fp32 [B], 4-byte aligned.  norms_given == 0: the call first computes
+ * this layer's N_b = ||G_b||_F^2 into sq_norms (pe_example_sqnorms) and clips by them; norms_given != 0:
+ * sq_norms is an input, e.g. the squared norms summed over all layers of a model for a model-wide clip.
+ * N_b = 0 gives c_b = 1.  Two passes over the inputs (norms, then the contraction with every G_b scaled
+ * on chip as it is added); G_b never reaches global memory.  X, dY, shapes as for pe_linear_stats;
+ * out_sum fp32 [d_out, d_in], 16-byte aligned, overwritten; clip_norm >= 0.
+ */
+pe_status_t pe_linear_clipped_sum(const void* X, const void* dY, int B, int T, int d_in, int d_out,
+                                  float clip_norm, float* sq_norms, int norms_given, float* out_sum,
+                                  pe_stream_t stream);
 
 /*
  * pe_linear_stats for gradient accumulation over micro-batches: the statistics of this call's B

@@ -18,6 +18,7 @@ __all__ = [
     "microadam_step", "microsignsgd_step", "pe_status_string", "pe_get_async_status", "pe_set_path", "pe_last_path",
     "pe_launch_count", "pe_reset_launch_count", "pe_token_sqstats_static", "STATIC_SCRATCH_BYTES",
     "microadam_family_step", "ADAM_VARIANTS", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms",
+    "pe_linear_stats_ragged", "pe_linear_stats_ragged_workspace_bytes", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
 ]
 
 PHI_IDENTITY, PHI_SQUARE, PHI_SIGN = 0, 1, 2
@@ -30,6 +31,7 @@ EXPORTED_SYMBOLS = [
     "pe_token_sqstats_staged_workspace_bytes", "microadam_step", "microsignsgd_step", "pe_status_string",
     "pe_get_async_status", "pe_set_path", "pe_last_path", "pe_launch_count", "pe_reset_launch_count",
     "pe_token_sqstats_static", "microadam_family_step", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms",
+    "pe_linear_stats_ragged", "pe_linear_stats_ragged_workspace_bytes", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
 ]
 ADAM_VARIANTS = {"adam": 0, "microadam": 1, "microadam_var": 2, "microadam_msq": 3}      # pe_adam_variant_t
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024      # PE_STATIC_SCRATCH_BYTES of pestats.h
@@ -66,6 +68,11 @@ def load_library() -> ctypes.CDLL:
     lib.pe_linear_stats_accumulate.argtypes = [vp, vp, i, i, i, i, i, vp, vp, vp]
     lib.pe_example_sqnorms.argtypes = [vp, vp, i, i, i, i, vp, vp]
     lib.pe_token_sqstats.argtypes = [vp, vp, i, i, i, i, vp, vp]
+    lib.pe_linear_stats_ragged.argtypes = [vp, vp, vp, i, ll, i, i, i, vp, vp, vp, sz, vp]
+    lib.pe_linear_stats_ragged_workspace_bytes.argtypes = [i, i, i]
+    lib.pe_linear_stats_ragged_workspace_bytes.restype = sz
+    lib.pe_example_sqnorms_ragged.argtypes = [vp, vp, vp, i, ll, i, i, vp, vp, sz, vp]
+    lib.pe_linear_clipped_sum.argtypes = [vp, vp, i, i, i, i, f, vp, i, vp, vp]
     lib.pe_token_sqstats_staged.argtypes = [vp, vp, i, i, i, i, vp, vp, sz, vp]
     lib.pe_token_sqstats_f32.argtypes = [vp, vp, i, i, i, i, vp, vp]
     lib.pe_token_sqstats_static.argtypes = [vp, vp, i, i, i, i, vp, vp]
@@ -85,6 +92,7 @@ def load_library() -> ctypes.CDLL:
     lib.pe_reset_launch_count.restype = None
     for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_static",
                  "pe_token_sqstats_staged",
+                 "pe_linear_stats_ragged", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
                  "microadam_step", "microadam_family_step", "microsignsgd_step", "pe_get_async_status", "pe_set_path", "pe_last_path"):
         getattr(lib, name).restype = i
     _lib = lib
@@ -160,6 +168,81 @@ def pe_example_sqnorms(X, dY, out_norms=None):
         _check("pe_example_sqnorms", load_library().pe_example_sqnorms(
             X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, out_norms.data_ptr() if B > 0 else None, _stream(X)))
     return out_norms
+
+
+def _ragged_check(X, dY, seq_offsets):
+    if X.dtype != torch.bfloat16 or dY.dtype != torch.bfloat16:
+        raise TypeError("X and dY must be torch.bfloat16")
+    if X.dim() != 2 or dY.dim() != 2 or X.shape[0] != dY.shape[0]:
+        raise ValueError("X must be [rows, d_in] and dY [rows, d_out] with equal row counts")
+    if not (X.is_contiguous() and dY.is_contiguous()):
+        raise ValueError("X and dY must be contiguous")
+    if seq_offsets.dtype != torch.int32 or seq_offsets.dim() != 1 or seq_offsets.numel() < 1 or not seq_offsets.is_contiguous() \
+            or seq_offsets.device != X.device:
+        raise ValueError("seq_offsets must be a contiguous int32 [B+1] tensor on the inputs' device")
+    return seq_offsets.numel() - 1, X.shape[0], X.shape[1], dY.shape[1]
+
+
+def pe_linear_stats_ragged_workspace_bytes(B, d_in, d_out) -> int:
+    return int(load_library().pe_linear_stats_ragged_workspace_bytes(int(B), int(d_in), int(d_out)))
+
+
+def _ragged_workspace(workspace, B, d_in, d_out, device):
+    need = pe_linear_stats_ragged_workspace_bytes(B, d_in, d_out)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=device)
+    return workspace, (workspace.numel() * workspace.element_size() if workspace is not None else 0)
+
+
+def pe_linear_stats_ragged(X, dY, seq_offsets, phi, out_mean=None, out_stat=None, workspace=None):
+    """pe_linear_stats for a packed batch: X [rows, d_in], dY [rows, d_out], example b owns rows
+    seq_offsets[b] .. seq_offsets[b+1]-1 (int32 device tensor).  Returns (out_mean, out_stat)."""
+    B, rows, d_in, d_out = _ragged_check(X, dY, seq_offsets)
+    if out_mean is None and out_stat is None:
+        out_mean = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)
+        out_stat = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)
+    _out_check("out_mean", out_mean, d_out, d_in)
+    _out_check("out_stat", out_stat, d_out, d_in)
+    workspace, wbytes = _ragged_workspace(workspace, B, d_in, d_out, X.device)
+    with _dev_ctx(X):
+        _check("pe_linear_stats_ragged", load_library().pe_linear_stats_ragged(
+            X.data_ptr(), dY.data_ptr(), seq_offsets.data_ptr(), B, rows, d_in, d_out, _phi(phi), _ptr(out_mean), _ptr(out_stat),
+            _ptr(workspace), wbytes, _stream(X)))
+    return out_mean, out_stat
+
+
+def pe_example_sqnorms_ragged(X, dY, seq_offsets, out_norms=None, workspace=None):
+    """Per-example squared gradient norms of a packed batch, float32 [B]."""
+    B, rows, d_in, d_out = _ragged_check(X, dY, seq_offsets)
+    if out_norms is None:
+        out_norms = torch.empty((B,), dtype=torch.float32, device=X.device)
+    if out_norms.dtype != torch.float32 or tuple(out_norms.shape) != (B,) or not out_norms.is_contiguous():
+        raise ValueError("out_norms must be a contiguous float32 [B] tensor")
+    workspace, wbytes = _ragged_workspace(workspace, B, d_in, d_out, X.device)
+    with _dev_ctx(X):
+        _check("pe_example_sqnorms_ragged", load_library().pe_example_sqnorms_ragged(
+            X.data_ptr(), dY.data_ptr(), seq_offsets.data_ptr(), B, rows, d_in, d_out, out_norms.data_ptr() if B > 0 else None,
+            _ptr(workspace), wbytes, _stream(X)))
+    return out_norms
+
+
+def pe_linear_clipped_sum(X, dY, clip_norm, sq_norms=None, out_sum=None):
+    """sum_b min(1, clip_norm / sqrt(N_b)) * G_b.  sq_norms None: this layer's own squared norms are computed
+    (and returned); otherwise the given float32 [B] tensor is used.  Returns (out_sum, sq_norms)."""
+    B, T, d_in, d_out = _io_check(X, dY, torch.bfloat16)
+    given = sq_norms is not None
+    if sq_norms is None:
+        sq_norms = torch.empty((B,), dtype=torch.float32, device=X.device)
+    if sq_norms.dtype != torch.float32 or tuple(sq_norms.shape) != (B,) or not sq_norms.is_contiguous():
+        raise ValueError("sq_norms must be a contiguous float32 [B] tensor")
+    if out_sum is None:
+        out_sum = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)
+    _out_check("out_sum", out_sum, d_out, d_in)
+    with _dev_ctx(X):
+        _check("pe_linear_clipped_sum", load_library().pe_linear_clipped_sum(
+            X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, float(clip_norm), sq_norms.data_ptr() if B > 0 else None, int(given),
+            out_sum.data_ptr(), _stream(X)))
+    return out_sum, sq_norms
 
 
 def pe_linear_stats_accumulate(X, dY, phi, out_mean, out_stat):

@@ -34,6 +34,7 @@ constexpr int TC_MEAN_TMEM_MIN_T = 4096;
 // tile's padding (columns up to the next multiple of 192) eats the gain.
 constexpr int TC_WIDE_MIN_T = 64;
 constexpr int TC_WIDE_MAX_PAD_PERCENT = 13;
+constexpr int PHI_CLIP_SCALE = 3;   // internal phi of the clipped sum: c_b * G_b (not part of pe_phi_t)
 constexpr int TC_BAND = 8;          // pair rows per band of the tile order (8 x 256 rows of d_out)
 
 constexpr int MAX_DEVICES = 64;
@@ -41,7 +42,7 @@ struct DeviceInfo {
   std::atomic<int> state{0};     // 0 unknown, 1 ready, -1 failed
   int cc_major = 0, sm_count = 0;
   unsigned int* status_ptr = nullptr;
-  bool tc_attr_set[16] = {};
+  bool tc_attr_set[24] = {};
   bool tok_attr_set = false;
 };
 static DeviceInfo g_dev[MAX_DEVICES];
@@ -201,22 +202,25 @@ static pe_status_t launch_pair_kernel(Kernel kernel, dim3 grid, int smem, cudaSt
   return check_launch();
 }
 
-template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT)>
+// mxt, myt: the maps of the zero-padded tail groups of a packed batch (RAGGED); any valid map otherwise.
+template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT), bool RAGGED = false>
 static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& mm,
-                                  const CUtensorMap& ms, const CUtensorMap& msgn, const TcParams& p, dim3 grid, cudaStream_t st) {
+                                  const CUtensorMap& ms, const CUtensorMap& msgn, const TcParams& p, dim3 grid, cudaStream_t st,
+                                  const CUtensorMap* mxt = nullptr, const CUtensorMap* myt = nullptr) {
   const bool after_zeroing = p.nsplit > 1 && !p.accumulate;
   constexpr int smem = TcOperand<TF32, NT, BKT>::SMEM_BYTES;
   {
     std::lock_guard<std::mutex> lock(g_dev_mutex);
     if (!di->tc_attr_set[slot]) {
-      if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+      if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT, RAGGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
         cudaGetLastError();
         return PE_ERR_CUDA;
       }
       di->tc_attr_set[slot] = true;
     }
   }
-  return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT>, grid, smem, st, after_zeroing, mx, my, mm, ms, msgn, p);
+  return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT, RAGGED>, grid, smem, st, after_zeroing, mx, my, mm, ms, msgn,
+                            mxt ? *mxt : mx, myt ? *myt : my, p);
 }
 
 // Tensor-core launch.  per_example = 0 runs the plain contraction over all B*T rows (its result goes
@@ -224,7 +228,7 @@ static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& m
 // pair tile is 256 x 128 (two running sums per thread); with only out_stat it is 256 x 256.
 static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int B, int T, int d_in, int d_out, int phi,
                              int per_example, float* out_mean, float* out_stat, cudaStream_t st, bool half_ops = false,
-                             float* out_sign = nullptr, bool accumulate = false) {
+                             float* out_sign = nullptr, bool accumulate = false, const float* sq_norms = nullptr, float clip_norm = 0.f) {
   const bool triple = out_sign != nullptr;       // mean + square + sign in one pass (phi = square, all three outputs given)
   const bool both = per_example && out_mean && out_stat;
   // Both outputs: sum_b G_b in tensor memory beside a 256-wide accumulator, unless the sequences are
@@ -265,7 +269,9 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   p.accumulate = accumulate ? 1 : 0;
   p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
   p.out_mean = out_mean; p.out_stat = out_stat; p.out_sign = out_sign; p.out_norms = nullptr; p.dev_status = di->status_ptr;
+  p.seq_offsets = nullptr; p.sq_norms = sq_norms; p.clip_norm = clip_norm;
   dim3 grid(2 * pairs_m * tiles_n, 1, ns);
+  if (phi == PHI_CLIP_SCALE) return launch_tc_inst<3, false, 256, MEAN_NONE>(di, 14, mx, my, mm, ms, msgn, p, grid, st);
   if (triple) return launch_tc_inst<1, false, 128, MEAN_REGS_SIGN>(di, 10, mx, my, mm, ms, msgn, p, grid, st);
   if (!per_example) return launch_tc_inst<0, false, 256, MEAN_NONE>(di, 4, mx, my, mm, ms, msgn, p, grid, st);
   if (short_seq) {
@@ -306,13 +312,14 @@ static pe_status_t launch_tc_norms(DeviceInfo* di, const void* X, const void* dY
   p.accumulate = 1;       // nothing is zeroed by a preceding kernel and no matrix is written
   p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
   p.out_mean = nullptr; p.out_stat = nullptr; p.out_sign = nullptr; p.out_norms = norms; p.dev_status = di->status_ptr;
+  p.seq_offsets = nullptr; p.sq_norms = nullptr; p.clip_norm = 0.f;
   // the three output maps are never used by this variant: any valid map will do
   return launch_tc_inst<1, false, 256, MEAN_NORMS>(di, 11, mx, my, mx, mx, mx, p, dim3(2 * pairs_m * tiles_n, 1, ns), st);
 }
 
 template <typename TIn, int MODE>
 static pe_status_t launch_simt(DeviceInfo* di, const TIn* X, const TIn* dY, int B, int T, int d_in, int d_out, int phi,
-                               float* out_mean, float* out_stat, cudaStream_t st, bool accumulate = false) {
+                               float* out_mean, float* out_stat, cudaStream_t st, bool accumulate = false, SimtExtra ex = SimtExtra{}) {
   const int tx = (d_in + SIMT_TILE - 1) / SIMT_TILE, ty = (d_out + SIMT_TILE - 1) / SIMT_TILE;
   if (ty > 65535) return PE_ERR_DIM;
   const int ns = choose_nsplit((long long)tx * ty, B, T, di->sm_count * 3, 64);
@@ -320,8 +327,91 @@ static pe_status_t launch_simt(DeviceInfo* di, const TIn* X, const TIn* dY, int 
     pe_status_t rc = zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
     if (rc != PE_OK) return rc;
   }
-  simt_stats_kernel<TIn, MODE><<<dim3(tx, ty, ns), SIMT_THREADS, 0, st>>>(X, dY, B, T, d_in, d_out, phi, out_mean, out_stat, accumulate ? 1 : 0);
+  simt_stats_kernel<TIn, MODE><<<dim3(tx, ty, ns), SIMT_THREADS, 0, st>>>(X, dY, B, T, d_in, d_out, phi, out_mean, out_stat, accumulate ? 1 : 0, ex);
   return check_launch();
+}
+
+// Side buffer of a packed batch: the zero-padded last partial 16-token group of every sequence, X's [B, 16, d_in]
+// then dY's [B, 16, d_out] (bf16), each part 256-byte aligned.
+struct RaggedLayout {
+  size_t x_bytes, y_bytes;
+  size_t total() const { return x_bytes + y_bytes; }
+};
+static RaggedLayout ragged_layout(int B, int d_in, int d_out) {
+  RaggedLayout l;
+  l.x_bytes = ((size_t)B * 16 * (size_t)d_in * 2 + 255) / 256 * 256;
+  l.y_bytes = ((size_t)B * 16 * (size_t)d_out * 2 + 255) / 256 * 256;
+  return l;
+}
+
+// Tensor-core launch for a packed batch.  norms != NULL: per-example squared norms (zeroed by the caller);
+// otherwise the statistics of pe_linear_stats.  phi = identity (or only out_mean wanted) runs the per-example
+// kernel with the identity, whose running sum is sum_b G_b.
+static pe_status_t launch_tc_ragged(DeviceInfo* di, const void* X, const void* dY, const int* offsets, int B, long long rows, int d_in,
+                                    int d_out, int phi, float* out_mean, float* out_stat, float* norms, void* ws, cudaStream_t st) {
+  const RaggedLayout l = ragged_layout(B, d_in, d_out);
+  uint16_t* xt = static_cast<uint16_t*>(ws);
+  uint16_t* yt = reinterpret_cast<uint16_t*>(static_cast<char*>(ws) + l.x_bytes);
+  const TailTensor tx = {static_cast<const uint16_t*>(X), xt, d_in}, ty = {static_cast<const uint16_t*>(dY), yt, d_out};
+  pack_tails_kernel<<<dim3((unsigned)B, 2, 1), STAGE_THREADS, 0, st>>>(tx, ty, offsets, rows);
+  pe_status_t rc = check_launch();
+  if (rc != PE_OK) return rc;
+  const bool both = !norms && out_mean && out_stat && phi != PE_PHI_IDENTITY;
+  const bool plain = !norms && (phi == PE_PHI_IDENTITY || !out_stat);      // only sum_b G_b
+  const int nt = both ? 192 : 256;
+  const int box_tokens = tc_default_bk(false, nt);
+  const int rows_i = (int)(rows > 0 ? rows : 1);
+  CUtensorMap mx, my, mxt, myt;
+  const int bf = TcOperand<false, 256>::BOX_FEATS;
+  if (both) {
+    rc = make_operand_map(&mx, X, 1, rows_i, d_in, false, TcOperand<false, 192>::B_BOX_FEATS, box_tokens, true);
+    if (rc == PE_OK) rc = make_operand_map(&mxt, xt, B, 16, d_in, false, TcOperand<false, 192>::B_BOX_FEATS, box_tokens, true);
+  } else {
+    rc = make_operand_map(&mx, X, 1, rows_i, d_in, false, bf, box_tokens);
+    if (rc == PE_OK) rc = make_operand_map(&mxt, xt, B, 16, d_in, false, bf, box_tokens);
+  }
+  if (rc == PE_OK) rc = make_operand_map(&my, dY, 1, rows_i, d_out, false, bf, box_tokens);
+  if (rc == PE_OK) rc = make_operand_map(&myt, yt, B, 16, d_out, false, bf, box_tokens);
+  if (rc != PE_OK) return rc;
+  float* first = plain ? (out_mean ? out_mean : out_stat) : out_stat;
+  CUtensorMap mm = mx, ms = mx;       // never used by the norms variant
+  if (!norms) {
+    rc = make_output_map(&ms, first, d_in, d_out);
+    if (rc == PE_OK) rc = make_output_map(&mm, both ? out_mean : first, d_in, d_out);
+    if (rc != PE_OK) return rc;
+  }
+  const int tiles_n = (d_in + nt - 1) / nt, pairs_m = (d_out + TC_PAIR_M - 1) / TC_PAIR_M;
+  if ((long long)tiles_n * pairs_m > (1ll << 29)) return PE_ERR_DIM;
+  const long long t_avg = rows / B > 0 ? rows / B : 1;
+  const int ns = choose_nsplit((long long)tiles_n * pairs_m, B, (int)(t_avg > (1 << 20) ? (1 << 20) : t_avg),
+                               di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 16);
+  if (ns > 1 && !norms) {
+    rc = zero_for_split(di, both ? out_mean : nullptr, first, (size_t)d_in * d_out, st);
+    if (rc != PE_OK) return rc;
+  }
+  TcParams p;
+  p.B = B; p.T = 0; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = 1; p.half_operands = 0;
+  p.accumulate = norms ? 1 : 0;
+  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
+  p.out_mean = both ? out_mean : nullptr; p.out_stat = norms ? nullptr : first; p.out_sign = nullptr; p.out_norms = norms;
+  p.seq_offsets = offsets; p.sq_norms = nullptr; p.clip_norm = 0.f; p.dev_status = di->status_ptr;
+  const dim3 grid(2 * pairs_m * tiles_n, 1, ns);
+  if (norms) return launch_tc_inst<1, false, 256, MEAN_NORMS, 64, true>(di, 15, mx, my, mm, ms, ms, p, grid, st, &mxt, &myt);
+  if (plain) {
+    rc = launch_tc_inst<0, false, 256, MEAN_NONE, 64, true>(di, 20, mx, my, mm, ms, ms, p, grid, st, &mxt, &myt);
+    if (rc == PE_OK && out_mean && out_stat &&
+        cudaMemcpyAsync(out_stat, out_mean, (size_t)d_in * d_out * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
+      cudaGetLastError();
+      return PE_ERR_CUDA;
+    }
+    return rc;
+  }
+  if (both) {
+    if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 192, MEAN_REGS, 128, true>(di, 16, mx, my, mm, ms, ms, p, grid, st, &mxt, &myt);
+    return launch_tc_inst<2, false, 192, MEAN_REGS, 128, true>(di, 17, mx, my, mm, ms, ms, p, grid, st, &mxt, &myt);
+  }
+  if (phi == PE_PHI_SQUARE) return launch_tc_inst<1, false, 256, MEAN_NONE, 64, true>(di, 18, mx, my, mm, ms, ms, p, grid, st, &mxt, &myt);
+  return launch_tc_inst<2, false, 256, MEAN_NONE, 64, true>(di, 19, mx, my, mm, ms, ms, p, grid, st, &mxt, &myt);
 }
 
 static pe_status_t validate_stats(const void* X, const void* dY, int B, int T, int d_in, int d_out, const float* o1,
@@ -504,6 +594,94 @@ pe_status_t pe_linear_stats_all(const void* X, const void* dY, int B, int T, int
   rc = linear_stats_impl<__nv_bfloat16>(Xb, Yb, B, T, d_in, d_out, PE_PHI_SQUARE, out_mean, out_square, st, true);
   if (rc != PE_OK) return rc;
   return linear_stats_impl<__nv_bfloat16>(Xb, Yb, B, T, d_in, d_out, PE_PHI_SIGN, nullptr, out_sign, st, true);
+}
+
+size_t pe_linear_stats_ragged_workspace_bytes(int B, int d_in, int d_out) {
+  if (B < 1 || d_in < 1 || d_out < 1 || (d_in % 8) || (d_out % 8) || g_path.load() == PE_PATH_SIMT) return 0;
+  return ragged_layout(B, d_in, d_out).total();
+}
+
+// Shared by pe_linear_stats_ragged and pe_example_sqnorms_ragged (norms != NULL).
+static pe_status_t ragged_impl(const void* X, const void* dY, const int* seq_offsets, int B, long long total_rows, int d_in, int d_out,
+                               int phi, float* out_mean, float* out_stat, float* norms, void* workspace, size_t workspace_bytes,
+                               cudaStream_t st) {
+  if (B < 0 || total_rows < 0 || total_rows >= (1ll << 31) || d_in < 1 || d_out < 1) return PE_ERR_DIM;
+  if (B > 0 && !seq_offsets) return PE_ERR_NULL;
+  if ((!X || !dY) && B > 0 && total_rows > 0) return PE_ERR_NULL;
+  if (!norms && !out_mean && !out_stat) return PE_ERR_NULL;
+  if (total_rows * (long long)(d_in > d_out ? d_in : d_out) >= (1ll << 40) || (long long)d_in * d_out >= (1ll << 40)) return PE_ERR_DIM;
+  if (!aligned(X, 16) || !aligned(dY, 16) || !aligned(seq_offsets, 4)) return PE_ERR_ALIGN;
+  if ((out_mean && !aligned(out_mean, 16)) || (out_stat && !aligned(out_stat, 16)) || (norms && !aligned(norms, 4))) return PE_ERR_ALIGN;
+  if (!norms && phi != PE_PHI_IDENTITY && phi != PE_PHI_SQUARE && phi != PE_PHI_SIGN) return PE_ERR_PHI;
+  DeviceInfo* di = nullptr;
+  pe_status_t rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  if (norms) {
+    if (B == 0) return PE_OK;
+    if (cudaMemsetAsync(norms, 0, (size_t)B * sizeof(float), st) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
+  }
+  if (B == 0 || total_rows == 0) return norms ? PE_OK : zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
+  const int forced = g_path.load();
+  const bool tc_ok = (d_in % 8) == 0 && (d_out % 8) == 0;
+  if (forced >= PE_PATH_TENSOR && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
+  if (tc_ok && forced != PE_PATH_SIMT) {
+    if (!workspace || workspace_bytes < ragged_layout(B, d_in, d_out).total()) return PE_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return PE_ERR_ALIGN;
+    g_last_path.store(PE_PATH_TENSOR);
+    return launch_tc_ragged(di, X, dY, seq_offsets, B, total_rows, d_in, d_out, phi, out_mean, out_stat, norms, workspace, st);
+  }
+  g_last_path.store(PE_PATH_SIMT);
+  SimtExtra ex{};
+  ex.seq_offsets = seq_offsets; ex.total_rows = total_rows;
+  const long long t_avg = total_rows / B > 0 ? total_rows / B : 1;
+  const __nv_bfloat16* Xb = static_cast<const __nv_bfloat16*>(X);
+  const __nv_bfloat16* Yb = static_cast<const __nv_bfloat16*>(dY);
+  if (norms) return launch_simt<__nv_bfloat16, MODE_NORMS>(di, Xb, Yb, B, (int)t_avg, d_in, d_out, 1, nullptr, norms, st, true, ex);
+  return launch_simt<__nv_bfloat16, MODE_STATS>(di, Xb, Yb, B, (int)t_avg, d_in, d_out, phi, out_mean, out_stat, st, false, ex);
+}
+
+pe_status_t pe_linear_stats_ragged(const void* X, const void* dY, const int* seq_offsets, int B, long long total_rows, int d_in,
+                                   int d_out, pe_phi_t phi, float* out_mean, float* out_stat, void* workspace,
+                                   size_t workspace_bytes, pe_stream_t stream) {
+  return ragged_impl(X, dY, seq_offsets, B, total_rows, d_in, d_out, (int)phi, out_mean, out_stat, nullptr, workspace, workspace_bytes,
+                     reinterpret_cast<cudaStream_t>(stream));
+}
+
+pe_status_t pe_example_sqnorms_ragged(const void* X, const void* dY, const int* seq_offsets, int B, long long total_rows, int d_in,
+                                      int d_out, float* out_norms, void* workspace, size_t workspace_bytes, pe_stream_t stream) {
+  if (!out_norms && B > 0) return PE_ERR_NULL;
+  return ragged_impl(X, dY, seq_offsets, B, total_rows, d_in, d_out, PE_PHI_SQUARE, nullptr, nullptr, out_norms, workspace,
+                     workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+pe_status_t pe_linear_clipped_sum(const void* X, const void* dY, int B, int T, int d_in, int d_out, float clip_norm, float* sq_norms,
+                                  int norms_given, float* out_sum, pe_stream_t stream) {
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (!out_sum || (!sq_norms && B > 0)) return PE_ERR_NULL;
+  if (!(clip_norm >= 0.f)) return PE_ERR_DIM;
+  pe_status_t rc = validate_stats(X, dY, B, T, d_in, d_out, out_sum, nullptr, false, 16);
+  if (rc != PE_OK) return rc;
+  if (sq_norms && !aligned(sq_norms, 4)) return PE_ERR_ALIGN;
+  DeviceInfo* di = nullptr;
+  rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  if (B == 0 || T == 0) return zero_outputs(out_sum, nullptr, (size_t)d_in * d_out * sizeof(float), st);
+  if (!norms_given) {
+    rc = pe_example_sqnorms(X, dY, B, T, d_in, d_out, sq_norms, stream);
+    if (rc != PE_OK) return rc;
+  }
+  const int forced = g_path.load();
+  const bool tc_ok = tc_shape_ok(B, T, d_in, d_out);
+  if (forced >= PE_PATH_TENSOR && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
+  if (tc_ok && forced != PE_PATH_SIMT) {
+    g_last_path.store(PE_PATH_TENSOR);
+    return launch_tc(di, X, dY, B, T, d_in, d_out, PHI_CLIP_SCALE, 1, nullptr, out_sum, st, false, nullptr, false, sq_norms, clip_norm);
+  }
+  g_last_path.store(PE_PATH_SIMT);
+  SimtExtra ex{};
+  ex.sq_norms = sq_norms; ex.clip_norm = clip_norm;
+  return launch_simt<__nv_bfloat16, MODE_STATS>(di, static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T,
+                                                d_in, d_out, PHI_CLIP_SCALE, nullptr, out_sum, st, false, ex);
 }
 
 pe_status_t pe_linear_stats_f32(const float* X, const float* dY, int B, int T, int d_in, int d_out, pe_phi_t phi,

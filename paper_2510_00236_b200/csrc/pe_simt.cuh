@@ -17,11 +17,21 @@ enum : int { MODE_STATS = 0, MODE_TOKEN = 1, MODE_NORMS = 2 };
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
 
-__device__ __forceinline__ float apply_phi(float g, int phi) {
+// phi: 0 identity, 1 square, 2 sign, 3 the clipping scale coef * g
+__device__ __forceinline__ float apply_phi(float g, int phi, float coef) {
   if (phi == 1) return g * g;
   if (phi == 2) return (g > 0.f ? 1.f : 0.f) - (g < 0.f ? 1.f : 0.f);
+  if (phi == 3) return coef * g;
   return g;
 }
+
+// What a packed batch or a clipped sum adds to the plain call; all NULL / 0 otherwise.
+struct SimtExtra {
+  const int* seq_offsets;     // [B + 1]: example b owns token rows offsets[b] .. offsets[b+1]-1 of X [rows, d_in], dY [rows, d_out]
+  long long total_rows;       // rows of the packed tensors (reads are kept inside)
+  const float* sq_norms;      // phi == 3: [B] squared norms N_b;  coef_b = min(1, clip_norm / sqrt(N_b))
+  float clip_norm;
+};
 
 // MODE_STATS: out_mean = sum_b G_b, out_stat = sum_b phi(G_b)         (Section 2.3, Eq. (2))
 // MODE_TOKEN: out_stat = sum_{b,t} dY^2 X^2; operands are squared as they are staged and the
@@ -34,7 +44,7 @@ __device__ __forceinline__ float apply_phi(float g, int phi) {
 template <typename TIn, int MODE>
 __global__ void __launch_bounds__(SIMT_THREADS)
 simt_stats_kernel(const TIn* __restrict__ X, const TIn* __restrict__ dY, int B, int T, int d_in, int d_out,
-                  int phi, float* __restrict__ out_mean, float* __restrict__ out_stat, int accumulate) {
+                  int phi, float* __restrict__ out_mean, float* __restrict__ out_stat, int accumulate, SimtExtra ex) {
   __shared__ float sY[SIMT_TK][SIMT_TILE];
   __shared__ float sX[SIMT_TK][SIMT_TILE];
 
@@ -57,9 +67,22 @@ simt_stats_kernel(const TIn* __restrict__ X, const TIn* __restrict__ dY, int B, 
 #pragma unroll
         for (int c = 0; c < 4; ++c) g[r][c] = 0.f;
     }
-    const TIn* Xb = X + (size_t)b * T * d_in;
-    const TIn* Yb = dY + (size_t)b * T * d_out;
-    for (int t0 = 0; t0 < T; t0 += SIMT_TK) {
+    long long row0 = (long long)b * T;
+    int Tb = T;
+    if (ex.seq_offsets) {            // packed batch: this example's own token range, clamped to the tensor
+      const long long r0 = ex.seq_offsets[b], r1 = ex.seq_offsets[b + 1];
+      row0 = r0 < 0 ? 0 : r0;
+      const long long end = r1 > ex.total_rows ? ex.total_rows : r1;
+      Tb = end > row0 ? (int)(end - row0) : 0;
+    }
+    float coef = 1.f;
+    if (phi == 3) {
+      const float nrm = sqrtf(ex.sq_norms[b]);
+      coef = nrm > ex.clip_norm ? ex.clip_norm / nrm : 1.f;
+    }
+    const TIn* Xb = X + (size_t)row0 * d_in;
+    const TIn* Yb = dY + (size_t)row0 * d_out;
+    for (int t0 = 0; t0 < Tb; t0 += SIMT_TK) {
       // stage SIMT_TK tokens of both operands, zero-filling past T and past the matrix edge
 #pragma unroll
       for (int k = 0; k < (SIMT_TK * SIMT_TILE) / SIMT_THREADS; ++k) {
@@ -67,7 +90,7 @@ simt_stats_kernel(const TIn* __restrict__ X, const TIn* __restrict__ dY, int B, 
         int tt = idx / SIMT_TILE, cc = idx % SIMT_TILE;
         int t = t0 + tt;
         float xv = 0.f, yv = 0.f;
-        if (t < T) {
+        if (t < Tb) {
           if (i0 + cc < d_in) xv = to_f32(Xb[(size_t)t * d_in + i0 + cc]);
           if (o0 + cc < d_out) yv = to_f32(Yb[(size_t)t * d_out + o0 + cc]);
         }
@@ -106,7 +129,7 @@ simt_stats_kernel(const TIn* __restrict__ X, const TIn* __restrict__ dY, int B, 
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           acc_mean[r][c] += g[r][c];
-          acc_stat[r][c] += apply_phi(g[r][c], phi);
+          acc_stat[r][c] += apply_phi(g[r][c], phi, coef);
         }
     }
   }

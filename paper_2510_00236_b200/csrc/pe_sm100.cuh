@@ -63,10 +63,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The same test without the bounded suspension try_wait may add: for a thread that polls several barriers in turn.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 
-// Cycle budget of any single wait (about 2 s at 2 GHz).  A wait that exhausts it latches an error
-// code and raises the block-wide abort flag so that every other role leaves its loops as well.
-constexpr long long WAIT_CYCLE_LIMIT = 1ll << 32;
+// Cycle budget of any single wait (by default about 2 s at 2 GHz; the host may lower it).  A wait that
+// exhausts it latches an error code and raises the block-wide abort flag so that every other role
+// leaves its loops as well.
+constexpr long long WAIT_CYCLE_LIMIT_DEFAULT = 1ll << 32;
+__device__ long long g_wait_cycle_limit = WAIT_CYCLE_LIMIT_DEFAULT;
+__device__ __forceinline__ long long wait_cycle_limit() { return *(volatile long long*)&g_wait_cycle_limit; }
 
 // Returns false if the wait was abandoned (its own timeout, or another role's).  SLEEP_NS > 0 backs
 // off between polls: every poll is a shared-memory access, and shared-memory bandwidth is what the
@@ -82,7 +97,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 0xff) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > WAIT_CYCLE_LIMIT) {
+      if (clock64() - t0 > wait_cycle_limit()) {
         *abort_flag = 1;
         atomicCAS(dev_status, 0u, (unsigned int)code);
         return false;

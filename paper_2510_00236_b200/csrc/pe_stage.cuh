@@ -129,4 +129,32 @@ unscale_kernel(float* __restrict__ out, int d_out, int d_in, const uint32_t* __r
   }
 }
 
+// Packed (ragged) batches, Section 2.3: example b owns token rows offsets[b] .. offsets[b+1]-1.  The tensor-core
+// kernel contracts 16 tokens per instruction, so a sequence's last len % 16 tokens are copied here, followed
+// by zero rows up to 16, into tails [B, 16, d] (an empty sequence gets 16 zero rows): that group is then
+// contracted like any other and the zero rows add nothing.  gridDim = (B, 2): y picks X or dY.
+// src: [rows, d] bf16 bit patterns, d a multiple of 8, 16-byte aligned.
+struct TailTensor {
+  const uint16_t* src;
+  uint16_t* tails;
+  int d;
+};
+__global__ void __launch_bounds__(STAGE_THREADS)
+pack_tails_kernel(TailTensor tx_, TailTensor ty_, const int* __restrict__ offsets, long long total_rows) {
+  const TailTensor& tn = blockIdx.y == 0 ? tx_ : ty_;
+  const int b = blockIdx.x, d8 = tn.d / 8;
+  const int r0 = offsets[b], r1 = offsets[b + 1];
+  const int len = r1 > r0 ? r1 - r0 : 0;
+  const int rem = len & 15;
+  const long long first = (long long)r0 + (len - rem);         // first row of the partial group
+  uint4* __restrict__ dst = reinterpret_cast<uint4*>(tn.tails) + (size_t)b * 16 * d8;
+  for (int k = threadIdx.x; k < 16 * d8; k += STAGE_THREADS) {
+    const int r = k / d8, c = k - r * d8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    const long long row = first + r;
+    if (r < rem && row >= 0 && row < total_rows) v = __ldg(reinterpret_cast<const uint4*>(tn.src) + row * d8 + c);
+    dst[k] = v;
+  }
+}
+
 }  // namespace pe

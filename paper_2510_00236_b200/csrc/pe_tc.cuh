@@ -128,8 +128,39 @@ struct TcParams {
   float* out_stat;     // may be NULL; written through tmap_stat
   float* out_sign;     // MEAN_REGS_SIGN only: sum_b sign(G_b), written through tmap_sign
   float* out_norms;    // MEAN_NORMS only: [B], zero on entry; every tile adds its share of ||G_b||_F^2
+  const int* seq_offsets;   // RAGGED only: [B + 1] token-row offsets; example b owns rows offsets[b] .. offsets[b+1]-1
+  const float* sq_norms;    // PHI == 3 only: [B] per-example squared norms the clipping coefficient is taken from
+  float clip_norm;          // PHI == 3 only: C of c_b = min(1, C / sqrt(N_b))
   unsigned int* dev_status;
 };
+
+// Where an example's tokens are and how many pipeline stages they take.  Fixed-length batches: the
+// operand maps are 3-D (d, T, B), an example is the coordinate `seq` of the last dimension and its
+// stages start at token 0.  Packed (ragged) batches: the maps are (d, rows, 1), the example starts at
+// row `row0`; its whole 16-token groups (`main` tokens) come from there in `nk_main` stages, and its
+// last `len % 16` tokens come, zero-padded to 16, from a side buffer that a pre-pass fills (a map
+// (d, 16, B)): one more stage with one MMA step.  An empty sequence is such a tail stage of zeros, so
+// that every example owns at least one stage and one accumulator.
+struct SeqGeom {
+  int row0, main, nk_main, nk;
+};
+template <bool RAGGED>
+__device__ __forceinline__ SeqGeom seq_geom(const TcParams& p, int b, int bk) {
+  SeqGeom g;
+  if constexpr (RAGGED) {
+    const int r0 = __ldg(p.seq_offsets + b), r1 = __ldg(p.seq_offsets + b + 1);
+    const int len = r1 > r0 ? r1 - r0 : 0;
+    g.row0 = r0;
+    g.main = len & ~15;
+    g.nk_main = (g.main + bk - 1) / bk;
+    g.nk = g.nk_main + (((len & 15) != 0 || len == 0) ? 1 : 0);
+  } else {
+    g.row0 = 0;
+    g.main = p.T;
+    g.nk_main = g.nk = (p.T + bk - 1) / bk;
+  }
+  return g;
+}
 
 // Tile order.  Pairs that run at the same time should share operand panels in L2, so consecutive
 // pair indices sweep the d_in tiles inside a band of p.band pair rows before moving to the next band:
@@ -155,21 +186,17 @@ __device__ __forceinline__ float phi_apply(float g) {
   return g;
 }
 
-// Walks the slots of the operand ring in the order the producers fill them.  With two issuers the
-// examples are taken two at a time and their stages interleaved: slot 2*kc of a pair of examples
-// belongs to its first example (issuer 0, even slots), slot 2*kc+1 to its second (issuer 1, odd
-// slots).  An unpaired last example leaves its partner's slots unused (used() is false there), so
-// that each slot is only ever consumed by the issuer of its own parity.
-template <int ISSUERS>
-struct StageWalk {
-  int nb, nk, e0, kc, x;
-  __device__ StageWalk(int nb_, int nk_) : nb(nb_), nk(nk_), e0(0), kc(0), x(0) {}
-  __device__ bool valid() const { return e0 < nb; }
-  __device__ bool used() const { return e0 + x < nb; }
-  __device__ int e() const { return e0 + x; }
-  __device__ void next() {
-    if (++x == ISSUERS) { x = 0; if (++kc == nk) { kc = 0; e0 += ISSUERS; } }
-  }
+// The operand ring and the two issuers.  Issuer x owns the ring slots of parity x (a sub-ring of
+// STAGES / 2 slots with its own phase) and the examples x, x + 2, ... of the slice, so the two issuers
+// run independently of each other.  The producers fill the two sub-rings in alternation, one stage of
+// each in turn while both still have stages to fill: with equal sequence lengths that is stage kc of an
+// even example, stage kc of the next odd one, stage kc + 1 of the even one, ...; with unequal lengths
+// (packed batches) the issuer of a short example simply moves on to its next example earlier.  A parity
+// wait is only meaningful while the waiter is at most one phase away from the barrier; since a slot
+// only ever sees the stages of ONE sub-ring, in order, that always holds.
+struct RingCursor {
+  int e, kc, n;       // example (slice-local), stage within it, stages of this sub-ring filled so far
+  SeqGeom g;
 };
 
 // Zeroes the outputs of a split-batch launch.  The statistics kernel that follows is launched as a
@@ -194,11 +221,15 @@ enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2, MEAN_REGS_SIGN = 3, ME
 constexpr int TC_SIGN_COUNT_MAX = 32767;   // examples per block in MEAN_REGS_SIGN mode: 2 * count must fit 16 bits
 
 // gridDim = (2 * pairs_m * tiles_n, 1, nsplit); blockIdx.x = 2 * (pair index in the tile order) + rank in pair.
-template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT)>
+// RAGGED: packed batch with per-example token ranges (tmap_x / tmap_dy are then (d, rows, 1), tmap_x_tail /
+// tmap_dy_tail (d, 16, B) over the zero-padded last partial token groups); otherwise the tail maps are unused.
+// PHI: 0 identity, 1 square, 2 sign, 3 the clipping scale c_b * g with c_b = min(1, C / sqrt(N_b)).
+template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT), bool RAGGED = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
                 const __grid_constant__ CUtensorMap tmap_mean, const __grid_constant__ CUtensorMap tmap_stat,
-                const __grid_constant__ CUtensorMap tmap_sign, TcParams p) {
+                const __grid_constant__ CUtensorMap tmap_sign, const __grid_constant__ CUtensorMap tmap_x_tail,
+                const __grid_constant__ CUtensorMap tmap_dy_tail, TcParams p) {
   using namespace sm100;
   using Op = TcOperand<TF32, NT, BKT>;
   constexpr bool TRIPLE = (MEAN == MEAN_REGS_SIGN);
@@ -208,6 +239,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   constexpr bool NORMS = (MEAN == MEAN_NORMS);
   static_assert(!NORMS || (PHI == 1 && NT == 256), "per-example norms: squares on the 256 x 256 tile");
   static_assert(MEAN != MEAN_TMEM || (NT == 256 && PHI != 0), "the tensor-memory mean sits beside one 256-column accumulator");
+  static_assert(!RAGGED || (!TF32 && MEAN != MEAN_TMEM), "packed batches: 16-bit operands, two issuers");
+  static_assert(PHI != 3 || MEAN == MEAN_NONE, "the clipped sum is a statistic-only pass");
   constexpr int STAGES = Op::STAGES, BK = Op::BK;
   constexpr int BOX_BYTES = Op::BOX_BYTES, A_BYTES = Op::A_BYTES, STAGE_BYTES = Op::STAGE_BYTES;
   constexpr int ISSUERS = (MEAN == MEAN_TMEM) ? 1 : 2;
@@ -233,7 +266,6 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   const int b_begin = (int)(((long long)p.B * blockIdx.z) / p.nsplit);
   const int b_end = (int)(((long long)p.B * (blockIdx.z + 1)) / p.nsplit);
   const int nb = b_end - b_begin;
-  const int nk = (p.T + BK - 1) / BK;               // stages per example
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -255,31 +287,71 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     if (warp == 0 || warp == 2) {
       // ---------------------------------------------------------- TMA producers (both blocks)
       // Warp 0 loads this block's rows of dY^T (and, in the leader, posts the stage's byte count);
-      // warp 2 loads this block's half of the X^T rows.  Both wait for the same "stage empty" phase.
-      // With two issuers, stages are filled for two examples at a time, alternating between them:
-      // stage 2*kc of a pair of examples belongs to its first example (issuer 0, even slots), stage
-      // 2*kc+1 to its second (issuer 1, odd slots); the ring has an even number of slots.
+      // warp 2 loads this block's half of the X^T rows.  Both wait for the same "stage empty" phase and
+      // fill the two issuers' sub-rings in alternation (see RingCursor).
       if (lane == 0) {
         const bool is_a = (warp == 0);
         int tile_m, tile_n;
         tc_tile_of_block(p, rank, tile_m, tile_n);
         const CUtensorMap* tmap = is_a ? &tmap_dy : &tmap_x;
+        const CUtensorMap* tmap_tail = is_a ? &tmap_dy_tail : &tmap_x_tail;
         const int c0 = is_a ? tile_m * TC_TILE_M : tile_n * NT + (int)rank * Op::B_FEATS;   // first feature of this warp's boxes
         const int n_boxes = is_a ? Op::A_BOXES : Op::B_BOXES;
         const int box_feats = is_a ? Op::BOX_FEATS : Op::B_BOX_FEATS;
         const int box_bytes = is_a ? BOX_BYTES : Op::B_BOX_BYTES;
         prefetch_tensormap(tmap);
-        int s = 0; uint32_t ph = 0;
-        for (StageWalk<ISSUERS> cur(nb, nk); cur.valid(); cur.next()) {
-          if (cur.used()) {
-            if (!mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_EMPTY)) break;
-            if (is_a && rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);     // both blocks' bytes
-            const uint32_t leader_full = map_to_cta(full_bar(s), 0);
-            const uint32_t dst = smem_base + s * STAGE_BYTES + (is_a ? 0 : A_BYTES);
+        if constexpr (RAGGED) prefetch_tensormap(tmap_tail);
+        constexpr int SUB = STAGES / ISSUERS;            // slots per sub-ring
+        auto start = [&](RingCursor& c, int x) {
+          c.e = x; c.kc = 0; c.n = 0;
+          if (c.e < nb) c.g = seq_geom<RAGGED>(p, b_begin + c.e, BK);
+        };
+        // Fills the next stage of sub-ring x if it has one and its slot is free; never blocks, because a
+        // sub-ring may stay full for as long as the OTHER one has to be filled (its issuer waits for an
+        // accumulator that the epilogue frees only after the other issuer's example).
+        auto try_fill = [&](RingCursor& c, int x) -> bool {
+          if (c.e >= nb) return false;
+          const int s = ISSUERS * (c.n % SUB) + x;
+          const uint32_t ph = (uint32_t)(c.n / SUB) & 1u;
+          if (!mbar_test_wait(empty_bar(s), ph ^ 1u)) return false;
+          if (is_a && rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);     // both blocks' bytes
+          const uint32_t leader_full = map_to_cta(full_bar(s), 0);
+          const uint32_t dst = smem_base + s * STAGE_BYTES + (is_a ? 0 : A_BYTES);
+          if constexpr (RAGGED) {
+            const bool tail = c.kc >= c.g.nk_main;       // the zero-padded last partial group, from the side buffer
             for (int g = 0; g < n_boxes; ++g)
-              tma_load_3d_pair(dst + g * box_bytes, tmap, leader_full, c0 + g * box_feats, cur.kc * BK, b_begin + cur.e());
+              tma_load_3d_pair(dst + g * box_bytes, tail ? tmap_tail : tmap, leader_full, c0 + g * box_feats,
+                               tail ? 0 : c.g.row0 + c.kc * BK, tail ? b_begin + c.e : 0);
+          } else {
+            for (int g = 0; g < n_boxes; ++g)
+              tma_load_3d_pair(dst + g * box_bytes, tmap, leader_full, c0 + g * box_feats, c.kc * BK, b_begin + c.e);
           }
-          if (++s == STAGES) { s = 0; ph ^= 1u; }
+          ++c.n;
+          if (++c.kc == c.g.nk) {
+            c.kc = 0;
+            c.e += ISSUERS;
+            if (c.e < nb) c.g = seq_geom<RAGGED>(p, b_begin + c.e, BK);
+          }
+          return true;
+        };
+        RingCursor ca, cb;
+        start(ca, 0);
+        start(cb, ISSUERS == 2 ? 1 : nb);
+        long long t0 = -1;
+        unsigned int spins = 0;
+        while (ca.e < nb || cb.e < nb) {
+          bool progressed = try_fill(ca, 0);
+          if (ISSUERS == 2 && try_fill(cb, 1)) progressed = true;
+          if (progressed) { t0 = -1; spins = 0; continue; }
+          if ((++spins & 0xffu) == 0) {                  // bounded like every other wait
+            if (*abort_flag) break;
+            if (t0 < 0) t0 = clock64();
+            else if (clock64() - t0 > wait_cycle_limit()) {
+              *abort_flag = 1;
+              atomicCAS(p.dev_status, 0u, (unsigned int)TC_WAIT_EMPTY);
+              break;
+            }
+          }
         }
       }
       __syncwarp();
@@ -294,8 +366,11 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         const uint32_t idesc = (!TF32 && p.half_operands) ? make_idesc_half_mn_major(TC_PAIR_M, NT) : make_idesc_mn_major(TC_PAIR_M, NT, TF32);
         bool ok = true;
         uint32_t accumulate = 0;
+        constexpr int SUB = STAGES / ISSUERS;              // slots of this issuer's sub-ring
         int i_local = 0;                                   // examples this issuer has started
+        int n_local = 0;                                   // stages this issuer has consumed
         for (int e = x; e < nb && ok; e += ISSUERS, ++i_local) {
+          const SeqGeom sg = seq_geom<RAGGED>(p, b_begin + e, BK);
           const int grp = p.per_example ? i_local : 0;
           const int buf = BUFS_PER_ISSUER * x + (grp % BUFS_PER_ISSUER);
           if (p.per_example || i_local == 0) {
@@ -305,20 +380,15 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             accumulate = 0;
           }
           const uint32_t d_tmem = tmem_base + (uint32_t)(buf * NT);
-          // position of this example's stages in the producer's sequence
-          const long long n0 = (long long)(e / ISSUERS) * ISSUERS * nk;
-          for (int kc = 0; kc < nk; ++kc) {
-            const long long n = n0 + ISSUERS * kc + x;
-            const int s = (int)(n % STAGES);
-            const uint32_t ph = (uint32_t)(n / STAGES) & 1u;
-            // A parity wait is only meaningful while the waiter is at most one phase away from the
-            // barrier.  Every slot this issuer waits on has its own parity (x), so it sees each of
-            // the slot's phases in turn and that always holds.
+          for (int kc = 0; kc < sg.nk; ++kc, ++n_local) {
+            const int s = ISSUERS * (n_local % SUB) + x;
+            const uint32_t ph = (uint32_t)(n_local / SUB) & 1u;
             if (!mbar_wait_bounded(full_bar(s), ph, abort_flag, p.dev_status, TC_WAIT_FULL)) { ok = false; break; }
             tc_fence_after();
             const uint32_t a_src = smem_base + s * STAGE_BYTES;
             const uint32_t b_src = a_src + A_BYTES;
-            const int t_left = p.T - kc * BK;              // tokens of this example still to contract
+            // tokens of this example in this stage: the rest of its whole 16-token groups, or the padded tail group
+            const int t_left = (RAGGED && kc >= sg.nk_main) ? 16 : sg.main - kc * BK;
 #pragma unroll
             for (int k = 0; k < BK / Op::MMA_K; ++k) {
               // rows past T are zero-filled by TMA; whole MMA steps past T are skipped
@@ -366,6 +436,15 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       const int x = a % ISSUERS, grp = p.per_example ? (a / ISSUERS) : 0;
       const int buf = BUFS_PER_ISSUER * x + (grp % BUFS_PER_ISSUER);
       const uint32_t acc_ph = (uint32_t)(grp / BUFS_PER_ISSUER) & 1u;
+      // PHI == 3: this example's clipping coefficient c_b = min(1, C / sqrt(N_b)); the load is issued before
+      // the wait for the accumulator, which hides its latency.  N_b = 0 (a zero gradient) gives 1.
+      uint64_t coef2 = 0;
+      if constexpr (PHI == 3) {
+        const float nb2 = __ldg(p.sq_norms + b_begin + a);
+        const float nrm = sqrtf(nb2);
+        const float c = nrm > p.clip_norm ? p.clip_norm / nrm : 1.f;
+        coef2 = f32x2_pack(c, c);
+      }
       // every lane polls, but the warp acts on one answer: the tensor-memory loads below are warp-wide
       // instructions, so no lane may leave the loop alone when its own wait is the one that gives up
       if (!__all_sync(0xffffffffu, mbar_wait_bounded(acc_full_bar(buf), acc_ph, abort_flag, p.dev_status, TC_WAIT_ACC_FULL))) { ok = false; break; }
@@ -450,8 +529,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 const uint64_t m2 = f32x2_add(f32x2_pack(acc_mean[c * CH + j], acc_mean[c * CH + j + 1]), g2);
                 f32x2_unpack(m2, acc_mean[c * CH + j], acc_mean[c * CH + j + 1]);
               }
-              if (PHI == 1) {
-                const uint64_t s2 = f32x2_fma(g2, g2, f32x2_pack(acc_stat[c * CH + j], acc_stat[c * CH + j + 1]));
+              if (PHI == 1 || PHI == 3) {
+                const uint64_t s2 = f32x2_fma(g2, PHI == 1 ? g2 : coef2, f32x2_pack(acc_stat[c * CH + j], acc_stat[c * CH + j + 1]));
                 f32x2_unpack(s2, acc_stat[c * CH + j], acc_stat[c * CH + j + 1]);
               }
               if (TRIPLE) {
