@@ -271,6 +271,46 @@ pe_status_t microsignsgd_step(float* theta, void* theta_lp, float* m, const floa
                               long long n, int B, float lr, float beta, float weight_decay,
                               pe_stream_t stream);
 
+/*
+ * Statistics and parameter update in ONE launch (Algorithm 1 applied to the statistics of Eq. (2) where
+ * they are formed: the thread block that holds, or completes, a tile's sums over the whole batch applies
+ * the update to that tile of the parameters, so the sums need not be written out and read back and the
+ * update needs no launch of its own).  The result is that of pe_linear_stats(phi = square) followed by
+ * microadam_family_step on its two outputs:
+ *     theta, m, v [d_out, d_in] fp32 updated in place, theta_lp the optional bf16 copy of the new theta.
+ * out_mean / out_stat (sum_b G_b, sum_b G_b^2): written when not NULL.  workspace: device memory, 256-byte
+ * aligned, pe_linear_fused_workspace_bytes(d_in, d_out) bytes (tile counters; contents undefined
+ * afterwards); needed, together with both outputs, when the schedule splits the batch across thread
+ * blocks: every block then adds its partial sums to the outputs and the one that adds the last part
+ * of a tile applies the update.  If the workspace or an output is missing the batch is not split (one
+ * block per tile walks all examples: correct, slower on layers with few tiles).  B >= 1, T >= 1; other
+ * arguments as for pe_linear_stats and microadam_family_step.  The _f32 form takes fp32 inputs (SIMT
+ * kernel, never splits the batch).  After PE_ERR_TIMEOUT the parameters of unfinished tiles are left as
+ * they were.
+ */
+pe_status_t pe_linear_microadam_step(const void* X, const void* dY, int B, int T, int d_in, int d_out,
+                                     float* theta, void* theta_lp, float* m, float* v, float* out_mean,
+                                     float* out_stat, pe_adam_variant_t variant, float grad_scale, float lr,
+                                     float beta1, float beta2, float eps, int eps_inside_sqrt,
+                                     float weight_decay, int step, void* workspace, size_t workspace_bytes,
+                                     pe_stream_t stream);
+pe_status_t pe_linear_microadam_step_f32(const float* X, const float* dY, int B, int T, int d_in, int d_out,
+                                         float* theta, void* theta_lp, float* m, float* v, float* out_mean,
+                                         float* out_stat, pe_adam_variant_t variant, float grad_scale,
+                                         float lr, float beta1, float beta2, float eps, int eps_inside_sqrt,
+                                         float weight_decay, int step, pe_stream_t stream);
+/*
+ * The same for MicroSignSGD (Section 3.1: EMA o avg o sign): pe_linear_stats(phi = sign, statistic only)
+ * followed by microsignsgd_step, in one launch.  out_sign (sum_b sign(G_b)) is written when not NULL and,
+ * like the workspace, is needed for a split batch.
+ */
+pe_status_t pe_linear_microsignsgd_step(const void* X, const void* dY, int B, int T, int d_in, int d_out,
+                                        float* theta, void* theta_lp, float* m, float* out_sign, float lr,
+                                        float beta, float weight_decay, void* workspace,
+                                        size_t workspace_bytes, pe_stream_t stream);
+/* Bytes of workspace the two calls above can use (one 32-bit counter per thread block of the widest grid). */
+size_t pe_linear_fused_workspace_bytes(int d_in, int d_out);
+
 /* Human-readable name of a status code (static storage). */
 const char* pe_status_string(pe_status_t status);
 

@@ -19,6 +19,7 @@ __all__ = [
     "pe_launch_count", "pe_reset_launch_count", "pe_token_sqstats_static", "STATIC_SCRATCH_BYTES",
     "microadam_family_step", "ADAM_VARIANTS", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms",
     "pe_linear_stats_ragged", "pe_linear_stats_ragged_workspace_bytes", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
+    "pe_linear_microadam_step", "pe_linear_microadam_step_f32", "pe_linear_microsignsgd_step", "pe_linear_fused_workspace_bytes",
 ]
 
 PHI_IDENTITY, PHI_SQUARE, PHI_SIGN = 0, 1, 2
@@ -32,6 +33,7 @@ EXPORTED_SYMBOLS = [
     "pe_get_async_status", "pe_set_path", "pe_last_path", "pe_launch_count", "pe_reset_launch_count",
     "pe_token_sqstats_static", "microadam_family_step", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms",
     "pe_linear_stats_ragged", "pe_linear_stats_ragged_workspace_bytes", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
+    "pe_linear_microadam_step", "pe_linear_microadam_step_f32", "pe_linear_microsignsgd_step", "pe_linear_fused_workspace_bytes",
 ]
 ADAM_VARIANTS = {"adam": 0, "microadam": 1, "microadam_var": 2, "microadam_msq": 3}      # pe_adam_variant_t
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024      # PE_STATIC_SCRATCH_BYTES of pestats.h
@@ -73,6 +75,11 @@ def load_library() -> ctypes.CDLL:
     lib.pe_linear_stats_ragged_workspace_bytes.restype = sz
     lib.pe_example_sqnorms_ragged.argtypes = [vp, vp, vp, i, ll, i, i, vp, vp, sz, vp]
     lib.pe_linear_clipped_sum.argtypes = [vp, vp, i, i, i, i, f, vp, i, vp, vp]
+    lib.pe_linear_microadam_step.argtypes = [vp, vp, i, i, i, i, vp, vp, vp, vp, vp, vp, i, f, f, f, f, f, i, f, i, vp, sz, vp]
+    lib.pe_linear_microadam_step_f32.argtypes = [vp, vp, i, i, i, i, vp, vp, vp, vp, vp, vp, i, f, f, f, f, f, i, f, i, vp]
+    lib.pe_linear_microsignsgd_step.argtypes = [vp, vp, i, i, i, i, vp, vp, vp, vp, f, f, f, vp, sz, vp]
+    lib.pe_linear_fused_workspace_bytes.argtypes = [i, i]
+    lib.pe_linear_fused_workspace_bytes.restype = sz
     lib.pe_token_sqstats_staged.argtypes = [vp, vp, i, i, i, i, vp, vp, sz, vp]
     lib.pe_token_sqstats_f32.argtypes = [vp, vp, i, i, i, i, vp, vp]
     lib.pe_token_sqstats_static.argtypes = [vp, vp, i, i, i, i, vp, vp]
@@ -93,6 +100,7 @@ def load_library() -> ctypes.CDLL:
     for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_static",
                  "pe_token_sqstats_staged",
                  "pe_linear_stats_ragged", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
+                 "pe_linear_microadam_step", "pe_linear_microadam_step_f32", "pe_linear_microsignsgd_step",
                  "microadam_step", "microadam_family_step", "microsignsgd_step", "pe_get_async_status", "pe_set_path", "pe_last_path"):
         getattr(lib, name).restype = i
     _lib = lib
@@ -243,6 +251,62 @@ def pe_linear_clipped_sum(X, dY, clip_norm, sq_norms=None, out_sum=None):
             X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, float(clip_norm), sq_norms.data_ptr() if B > 0 else None, int(given),
             out_sum.data_ptr(), _stream(X)))
     return out_sum, sq_norms
+
+
+def pe_linear_fused_workspace_bytes(d_in, d_out) -> int:
+    return int(load_library().pe_linear_fused_workspace_bytes(int(d_in), int(d_out)))
+
+
+def _param_check(name, t, d_out, d_in, dtype=torch.float32):
+    if t.dtype != dtype or tuple(t.shape) != (d_out, d_in) or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous {dtype} [d_out, d_in] tensor")
+
+
+def pe_linear_microadam_step(X, dY, theta, m, v, *, lr, beta1, beta2, eps, step, variant="microadam", grad_scale=1.0,
+                             eps_inside_sqrt=False, weight_decay=0.0, theta_lp=None, out_mean=None, out_stat=None, workspace=None):
+    """Per-example statistics (phi = square) and the Adam-family update of theta, m, v in one launch.
+    X, dY bf16 (tensor-core / SIMT kernel) or float32 (SIMT kernel).  `workspace`: uint8 tensor of
+    pe_linear_fused_workspace_bytes(d_in, d_out) bytes; with it and both outputs the batch may be split."""
+    B, T, d_in, d_out = _io_check(X, dY, X.dtype)
+    for name, t in (("theta", theta), ("m", m), ("v", v)):
+        _param_check(name, t, d_out, d_in)
+    if theta_lp is not None:
+        _param_check("theta_lp", theta_lp, d_out, d_in, torch.bfloat16)
+    _out_check("out_mean", out_mean, d_out, d_in)
+    _out_check("out_stat", out_stat, d_out, d_in)
+    common = (B, T, d_in, d_out, theta.data_ptr(), _ptr(theta_lp), m.data_ptr(), v.data_ptr(), _ptr(out_mean), _ptr(out_stat),
+              ADAM_VARIANTS[variant] if isinstance(variant, str) else int(variant), float(grad_scale), float(lr), float(beta1),
+              float(beta2), float(eps), int(bool(eps_inside_sqrt)), float(weight_decay), int(step))
+    with _dev_ctx(X):
+        if X.dtype == torch.float32:
+            _check("pe_linear_microadam_step_f32", load_library().pe_linear_microadam_step_f32(X.data_ptr(), dY.data_ptr(), *common, _stream(X)))
+        else:
+            wb = workspace.numel() * workspace.element_size() if workspace is not None else 0
+            _check("pe_linear_microadam_step", load_library().pe_linear_microadam_step(X.data_ptr(), dY.data_ptr(), *common, _ptr(workspace), wb, _stream(X)))
+    return theta, m, v
+
+
+def pe_linear_microadam_step_f32(X, dY, theta, m, v, **kw):
+    """pe_linear_microadam_step for float32 inputs (the C entry point of the same name)."""
+    if X.dtype != torch.float32:
+        raise TypeError("X and dY must be torch.float32")
+    return pe_linear_microadam_step(X, dY, theta, m, v, **kw)
+
+
+def pe_linear_microsignsgd_step(X, dY, theta, m, *, lr, beta, weight_decay=0.0, theta_lp=None, out_sign=None, workspace=None):
+    """Per-example sign statistic and the MicroSignSGD update of theta, m in one launch (bf16 inputs)."""
+    B, T, d_in, d_out = _io_check(X, dY, torch.bfloat16)
+    _param_check("theta", theta, d_out, d_in)
+    _param_check("m", m, d_out, d_in)
+    if theta_lp is not None:
+        _param_check("theta_lp", theta_lp, d_out, d_in, torch.bfloat16)
+    _out_check("out_sign", out_sign, d_out, d_in)
+    wb = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    with _dev_ctx(X):
+        _check("pe_linear_microsignsgd_step", load_library().pe_linear_microsignsgd_step(
+            X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, theta.data_ptr(), _ptr(theta_lp), m.data_ptr(), _ptr(out_sign), float(lr),
+            float(beta), float(weight_decay), _ptr(workspace), wb, _stream(X)))
+    return theta, m
 
 
 def pe_linear_stats_accumulate(X, dY, phi, out_mean, out_stat):

@@ -42,7 +42,7 @@ struct DeviceInfo {
   std::atomic<int> state{0};     // 0 unknown, 1 ready, -1 failed
   int cc_major = 0, sm_count = 0;
   unsigned int* status_ptr = nullptr;
-  bool tc_attr_set[24] = {};
+  bool tc_attr_set[32] = {};
   bool tok_attr_set = false;
 };
 static DeviceInfo g_dev[MAX_DEVICES];
@@ -177,7 +177,8 @@ static pe_status_t zero_outputs(float* a, float* b, size_t bytes, cudaStream_t s
 }
 
 // Zeroes up to three [d_out, d_in] outputs with a kernel that lets its successor start at once.
-static pe_status_t zero_for_split(DeviceInfo* di, float* a, float* b, size_t n, cudaStream_t st, float* c = nullptr) {
+static pe_status_t zero_for_split(DeviceInfo* di, float* a, float* b, size_t n, cudaStream_t st, float* c = nullptr,
+                                  unsigned int* counters = nullptr, int n_counters = 0) {
   float* first = a ? a : b;
   float* second = a ? b : nullptr;
   if (!first) return PE_OK;
@@ -185,7 +186,7 @@ static pe_status_t zero_for_split(DeviceInfo* di, float* a, float* b, size_t n, 
   long long blocks = (n4 + 255) / 256;
   if (blocks > di->sm_count) blocks = di->sm_count;   // few blocks: the dependent kernel needs the SMs
   zero_outputs_kernel<<<(int)(blocks < 1 ? 1 : blocks), 256, 0, st>>>(reinterpret_cast<float4*>(first), reinterpret_cast<float4*>(second),
-                                                                            reinterpret_cast<float4*>(c), n4);
+                                                                            reinterpret_cast<float4*>(c), n4, counters, n_counters);
   return check_launch();
 }
 
@@ -203,24 +204,24 @@ static pe_status_t launch_pair_kernel(Kernel kernel, dim3 grid, int smem, cudaSt
 }
 
 // mxt, myt: the maps of the zero-padded tail groups of a packed batch (RAGGED); any valid map otherwise.
-template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT), bool RAGGED = false>
+template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT), bool RAGGED = false, int OPT = OPT_NONE>
 static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& mm,
                                   const CUtensorMap& ms, const CUtensorMap& msgn, const TcParams& p, dim3 grid, cudaStream_t st,
-                                  const CUtensorMap* mxt = nullptr, const CUtensorMap* myt = nullptr) {
+                                  const CUtensorMap* mxt = nullptr, const CUtensorMap* myt = nullptr, const FusedOpt* opt = nullptr) {
   const bool after_zeroing = p.nsplit > 1 && !p.accumulate;
   constexpr int smem = TcOperand<TF32, NT, BKT>::SMEM_BYTES;
   {
     std::lock_guard<std::mutex> lock(g_dev_mutex);
     if (!di->tc_attr_set[slot]) {
-      if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT, RAGGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+      if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT, RAGGED, OPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
         cudaGetLastError();
         return PE_ERR_CUDA;
       }
       di->tc_attr_set[slot] = true;
     }
   }
-  return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT, RAGGED>, grid, smem, st, after_zeroing, mx, my, mm, ms, msgn,
-                            mxt ? *mxt : mx, myt ? *myt : my, p);
+  return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT, RAGGED, OPT>, grid, smem, st, after_zeroing, mx, my, mm, ms, msgn,
+                            mxt ? *mxt : mx, myt ? *myt : my, p, opt ? *opt : FusedOpt{});
 }
 
 // Tensor-core launch.  per_example = 0 runs the plain contraction over all B*T rows (its result goes
@@ -319,15 +320,18 @@ static pe_status_t launch_tc_norms(DeviceInfo* di, const void* X, const void* dY
 
 template <typename TIn, int MODE>
 static pe_status_t launch_simt(DeviceInfo* di, const TIn* X, const TIn* dY, int B, int T, int d_in, int d_out, int phi,
-                               float* out_mean, float* out_stat, cudaStream_t st, bool accumulate = false, SimtExtra ex = SimtExtra{}) {
+                               float* out_mean, float* out_stat, cudaStream_t st, bool accumulate = false, SimtExtra ex = SimtExtra{},
+                               const FusedOpt* opt = nullptr) {
   const int tx = (d_in + SIMT_TILE - 1) / SIMT_TILE, ty = (d_out + SIMT_TILE - 1) / SIMT_TILE;
   if (ty > 65535) return PE_ERR_DIM;
-  const int ns = choose_nsplit((long long)tx * ty, B, T, di->sm_count * 3, 64);
+  // a fused update needs the whole batch in one block (this kernel has no cross-block completion protocol)
+  const int ns = opt ? 1 : choose_nsplit((long long)tx * ty, B, T, di->sm_count * 3, 64);
   if (ns > 1 && !accumulate) {
     pe_status_t rc = zero_outputs(out_mean, out_stat, (size_t)d_in * d_out * sizeof(float), st);
     if (rc != PE_OK) return rc;
   }
-  simt_stats_kernel<TIn, MODE><<<dim3(tx, ty, ns), SIMT_THREADS, 0, st>>>(X, dY, B, T, d_in, d_out, phi, out_mean, out_stat, accumulate ? 1 : 0, ex);
+  simt_stats_kernel<TIn, MODE><<<dim3(tx, ty, ns), SIMT_THREADS, 0, st>>>(X, dY, B, T, d_in, d_out, phi, out_mean, out_stat, accumulate ? 1 : 0, ex,
+                                                                            opt ? *opt : FusedOpt{});
   return check_launch();
 }
 
@@ -478,6 +482,72 @@ static pe_status_t linear_stats_impl(const TIn* X, const TIn* dY, int B, int T, 
 }
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Constants of one Adam-family step (Algorithm 1): the scales that turn the sums into averages, the
+// bias corrections of step t, and the factor 1 / (1 - 1/B) of Eq. (6).
+static AdamParams make_adam_params(int B, float grad_scale, float lr, float beta1, float beta2, float eps, int eps_inside_sqrt,
+                                   float weight_decay, int step) {
+  AdamParams p;
+  p.mu_scale = (float)((double)grad_scale / (double)B);
+  p.nu_scale = (float)((double)grad_scale * (double)grad_scale / (double)B);
+  p.beta1 = beta1; p.beta2 = beta2;
+  p.inv_c1 = (float)(1.0 / (1.0 - std::pow((double)beta1, (double)step)));
+  p.inv_c2 = (float)(1.0 / (1.0 - std::pow((double)beta2, (double)step)));
+  p.eps = eps; p.lr = lr; p.wd = weight_decay; p.eps_inside = eps_inside_sqrt ? 1 : 0;
+  p.inv_B = (float)(1.0 / (double)B);
+  p.bessel = B > 1 ? (float)(1.0 / (1.0 - 1.0 / (double)B)) : 1.f;
+  return p;
+}
+
+// Words of tile counters a fused statistics + update launch may need: one per thread block of the widest grid
+// (256 x 128 tiles), i.e. two per pair tile.
+static size_t fused_counter_words(int d_in, int d_out) {
+  return 2 * (size_t)((d_out + TC_PAIR_M - 1) / TC_PAIR_M) * (size_t)((d_in + 127) / 128);
+}
+
+// Statistics and parameter update in one tensor-core launch.  kind = OPT_ADAM: sum_b G_b and sum_b G_b^2 (256 x 192 or
+// 256 x 128 tile, both sums in registers) feed Algorithm 1; kind = OPT_SIGN: sum_b sign(G_b) (256 x 256 tile) feeds
+// MicroSignSGD.  out_a = out_mean (Adam only), out_b = the statistic; they may be NULL when the schedule does not
+// split the batch, which is forced when they (or the counters) are missing.
+static pe_status_t launch_tc_fused(DeviceInfo* di, const void* X, const void* dY, int B, int T, int d_in, int d_out, int kind,
+                                   float* out_a, float* out_b, FusedOpt opt, unsigned int* counters, size_t counter_words,
+                                   cudaStream_t st) {
+  const bool adam = kind == OPT_ADAM;
+  const long long pad192 = (long long)((d_in + 191) / 192) * 192, pad128 = (long long)((d_in + 127) / 128) * 128;
+  const int forced = g_path.load();
+  const bool wide = adam && forced != PE_PATH_TENSOR_NARROW &&
+                    (forced == PE_PATH_TENSOR_WIDE || (T >= TC_WIDE_MIN_T && pad192 * 100 <= pad128 * (100 + TC_WIDE_MAX_PAD_PERCENT)));
+  const int nt = adam ? (wide ? 192 : 128) : 256;
+  const int box_feats = TcOperand<false, 256>::BOX_FEATS, box_tokens = tc_default_bk(false, nt);
+  CUtensorMap mx, my, mm, ms;
+  pe_status_t rc = wide ? make_operand_map(&mx, X, B, T, d_in, false, TcOperand<false, 192>::B_BOX_FEATS, box_tokens, true)
+                        : make_operand_map(&mx, X, B, T, d_in, false, box_feats, box_tokens);
+  if (rc == PE_OK) rc = make_operand_map(&my, dY, B, T, d_out, false, box_feats, box_tokens);
+  // an output that is not wanted gets a map over the parameters and is never written through it
+  if (rc == PE_OK) rc = make_output_map(&mm, out_a ? out_a : opt.theta, d_in, d_out);
+  if (rc == PE_OK) rc = make_output_map(&ms, out_b ? out_b : opt.theta, d_in, d_out);
+  if (rc != PE_OK) return rc;
+  const int tiles_n = (d_in + nt - 1) / nt, pairs_m = (d_out + TC_PAIR_M - 1) / TC_PAIR_M;
+  if ((long long)tiles_n * pairs_m > (1ll << 29)) return PE_ERR_DIM;
+  int ns = choose_nsplit((long long)tiles_n * pairs_m, B, T, di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 16);
+  const size_t blocks = 2 * (size_t)tiles_n * pairs_m;
+  if (ns > 1 && (!out_b || (adam && !out_a) || !counters || counter_words < blocks)) ns = 1;
+  if (ns > 1) {
+    rc = zero_for_split(di, adam ? out_a : nullptr, out_b, (size_t)d_in * d_out, st, nullptr, counters, (int)blocks);
+    if (rc != PE_OK) return rc;
+  }
+  TcParams p;
+  p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = 1; p.half_operands = 0; p.accumulate = 0;
+  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
+  p.out_mean = adam ? out_a : nullptr; p.out_stat = out_b; p.out_sign = nullptr; p.out_norms = nullptr; p.dev_status = di->status_ptr;
+  p.seq_offsets = nullptr; p.sq_norms = nullptr; p.clip_norm = 0.f;
+  opt.kind = kind;
+  opt.tile_counters = counters;
+  const dim3 grid((unsigned)blocks, 1, ns);
+  if (!adam) return launch_tc_inst<2, false, 256, MEAN_NONE, 64, false, OPT_SIGN>(di, 23, mx, my, mm, ms, ms, p, grid, st, nullptr, nullptr, &opt);
+  if (wide) return launch_tc_inst<1, false, 192, MEAN_REGS, 128, false, OPT_ADAM>(di, 21, mx, my, mm, ms, ms, p, grid, st, nullptr, nullptr, &opt);
+  return launch_tc_inst<1, false, 128, MEAN_REGS, 128, false, OPT_ADAM>(di, 22, mx, my, mm, ms, ms, p, grid, st, nullptr, nullptr, &opt);
+}
 
 static int grid_for(long long work_items, int sm_count) {
   long long blocks = (work_items + OPT_THREADS - 1) / OPT_THREADS;
@@ -684,6 +754,87 @@ pe_status_t pe_linear_clipped_sum(const void* X, const void* dY, int B, int T, i
                                                 d_in, d_out, PHI_CLIP_SCALE, nullptr, out_sum, st, false, ex);
 }
 
+size_t pe_linear_fused_workspace_bytes(int d_in, int d_out) {
+  if (d_in < 1 || d_out < 1) return 0;
+  return align_up(fused_counter_words(d_in, d_out) * sizeof(unsigned int), 256);
+}
+
+// Shared by the three fused entry points.  kind: OPT_ADAM / OPT_SIGN; out_a: sum_b G_b (Adam), out_b: the statistic.
+extern "C++" template <typename TIn>
+pe_status_t fused_impl(const TIn* X, const TIn* dY, int B, int T, int d_in, int d_out, int kind, float* theta, void* theta_lp,
+                              float* m, float* v, float* out_a, float* out_b, FusedOpt opt, void* workspace, size_t workspace_bytes,
+                              cudaStream_t st, bool allow_tc) {
+  if (!theta || !m || (kind == OPT_ADAM && !v)) return PE_ERR_NULL;
+  if (B < 1 || T < 1) return PE_ERR_DIM;
+  pe_status_t rc = validate_stats(X, dY, B, T, d_in, d_out, out_a, out_b, false, allow_tc ? 16 : 4);
+  if (rc != PE_OK) return rc;
+  if (!aligned(theta, 16) || !aligned(m, 16) || (v && !aligned(v, 16)) || (theta_lp && !aligned(theta_lp, 16))) return PE_ERR_ALIGN;
+  if (workspace && !aligned(workspace, 256)) return PE_ERR_ALIGN;
+  DeviceInfo* di = nullptr;
+  rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  opt.kind = kind;
+  opt.theta = theta; opt.theta_lp = static_cast<__nv_bfloat16*>(theta_lp); opt.m = m; opt.v = v; opt.tile_counters = nullptr;
+  const int forced = g_path.load();
+  const bool tc_ok = allow_tc && tc_shape_ok(B, T, d_in, d_out);
+  if (forced >= PE_PATH_TENSOR && !tc_ok) return PE_ERR_UNSUPPORTED_SHAPE;
+  if (tc_ok && forced != PE_PATH_SIMT) {
+    if constexpr (sizeof(TIn) == 2) {
+      g_last_path.store(PE_PATH_TENSOR);
+      return launch_tc_fused(di, X, dY, B, T, d_in, d_out, kind, out_a, out_b, opt, static_cast<unsigned int*>(workspace),
+                             workspace_bytes / sizeof(unsigned int), st);
+    }
+  }
+  g_last_path.store(PE_PATH_SIMT);
+  return launch_simt<TIn, MODE_STATS>(di, X, dY, B, T, d_in, d_out, kind == OPT_ADAM ? (int)PE_PHI_SQUARE : (int)PE_PHI_SIGN, out_a, out_b, st,
+                                      false, SimtExtra{}, &opt);
+}
+
+static pe_status_t check_adam_args(int B, pe_adam_variant_t variant, int step) {
+  if (B < 1 || step < 1) return PE_ERR_DIM;
+  if ((int)variant < 0 || (int)variant > 3) return PE_ERR_PHI;
+  if (((int)variant == ADAM_MICRO_VAR || (int)variant == ADAM_MICRO_MSQ) && B < 2) return PE_ERR_DIM;
+  return PE_OK;
+}
+
+pe_status_t pe_linear_microadam_step(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* theta, void* theta_lp,
+                                     float* m, float* v, float* out_mean, float* out_stat, pe_adam_variant_t variant, float grad_scale,
+                                     float lr, float beta1, float beta2, float eps, int eps_inside_sqrt, float weight_decay, int step,
+                                     void* workspace, size_t workspace_bytes, pe_stream_t stream) {
+  pe_status_t rc = check_adam_args(B, variant, step);
+  if (rc != PE_OK) return rc;
+  FusedOpt opt{};
+  opt.variant = (int)variant;
+  opt.adam = make_adam_params(B, grad_scale, lr, beta1, beta2, eps, eps_inside_sqrt, weight_decay, step);
+  return fused_impl<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T, d_in, d_out, OPT_ADAM,
+                                   theta, theta_lp, m, v, out_mean, out_stat, opt, workspace, workspace_bytes,
+                                   reinterpret_cast<cudaStream_t>(stream), true);
+}
+
+pe_status_t pe_linear_microadam_step_f32(const float* X, const float* dY, int B, int T, int d_in, int d_out, float* theta, void* theta_lp,
+                                         float* m, float* v, float* out_mean, float* out_stat, pe_adam_variant_t variant,
+                                         float grad_scale, float lr, float beta1, float beta2, float eps, int eps_inside_sqrt,
+                                         float weight_decay, int step, pe_stream_t stream) {
+  pe_status_t rc = check_adam_args(B, variant, step);
+  if (rc != PE_OK) return rc;
+  FusedOpt opt{};
+  opt.variant = (int)variant;
+  opt.adam = make_adam_params(B, grad_scale, lr, beta1, beta2, eps, eps_inside_sqrt, weight_decay, step);
+  return fused_impl<float>(X, dY, B, T, d_in, d_out, OPT_ADAM, theta, theta_lp, m, v, out_mean, out_stat, opt, nullptr, 0,
+                           reinterpret_cast<cudaStream_t>(stream), false);
+}
+
+pe_status_t pe_linear_microsignsgd_step(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* theta, void* theta_lp,
+                                        float* m, float* out_sign, float lr, float beta, float weight_decay, void* workspace,
+                                        size_t workspace_bytes, pe_stream_t stream) {
+  if (B < 1) return PE_ERR_DIM;
+  FusedOpt opt{};
+  opt.sign.inv_B = (float)(1.0 / (double)B); opt.sign.beta = beta; opt.sign.lr = lr; opt.sign.wd = weight_decay;
+  return fused_impl<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T, d_in, d_out, OPT_SIGN,
+                                   theta, theta_lp, m, nullptr, nullptr, out_sign, opt, workspace, workspace_bytes,
+                                   reinterpret_cast<cudaStream_t>(stream), true);
+}
+
 pe_status_t pe_linear_stats_f32(const float* X, const float* dY, int B, int T, int d_in, int d_out, pe_phi_t phi,
                                 float* out_mean, float* out_stat, pe_stream_t stream) {
   return linear_stats_impl<float>(X, dY, B, T, d_in, d_out, phi, out_mean, out_stat, reinterpret_cast<cudaStream_t>(stream), false);
@@ -868,15 +1019,7 @@ pe_status_t microadam_family_step(float* theta, void* theta_lp, float* m, float*
   pe_status_t rc = device_info(&di);
   if (rc != PE_OK) return rc;
   if (n == 0) return PE_OK;
-  AdamParams p;
-  p.mu_scale = (float)((double)grad_scale / (double)B);
-  p.nu_scale = (float)((double)grad_scale * (double)grad_scale / (double)B);
-  p.beta1 = beta1; p.beta2 = beta2;
-  p.inv_c1 = (float)(1.0 / (1.0 - std::pow((double)beta1, (double)step)));
-  p.inv_c2 = (float)(1.0 / (1.0 - std::pow((double)beta2, (double)step)));
-  p.eps = eps; p.lr = lr; p.wd = weight_decay; p.eps_inside = eps_inside_sqrt ? 1 : 0;
-  p.inv_B = (float)(1.0 / (double)B);
-  p.bessel = B > 1 ? (float)(1.0 / (1.0 - 1.0 / (double)B)) : 1.f;
+  const AdamParams p = make_adam_params(B, grad_scale, lr, beta1, beta2, eps, eps_inside_sqrt, weight_decay, step);
   const int grid = grid_for(n / 4 + 4, di->sm_count);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   __nv_bfloat16* lp = static_cast<__nv_bfloat16*>(theta_lp);

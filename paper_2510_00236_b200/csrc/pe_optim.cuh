@@ -43,6 +43,16 @@ __device__ __forceinline__ void adam_one(float& th, float& m, float& v, float sg
   th = th - p.lr * u - p.wd * th;
 }
 
+// The same with the member of the family chosen at run time (the update fused into the statistics kernels).
+__device__ __forceinline__ void adam_one_rt(int variant, float& th, float& m, float& v, float sg, float sg2, const AdamParams& p) {
+  switch (variant) {
+    case ADAM_ORIGINAL: adam_one<ADAM_ORIGINAL>(th, m, v, sg, sg2, p); break;
+    case ADAM_MICRO: adam_one<ADAM_MICRO>(th, m, v, sg, sg2, p); break;
+    case ADAM_MICRO_VAR: adam_one<ADAM_MICRO_VAR>(th, m, v, sg, sg2, p); break;
+    default: adam_one<ADAM_MICRO_MSQ>(th, m, v, sg, sg2, p); break;
+  }
+}
+
 __device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
 
 constexpr int OPT_THREADS = 256;
@@ -128,6 +138,40 @@ microsignsgd_kernel(float* __restrict__ theta, __nv_bfloat16* __restrict__ theta
     theta[k] = th; m[k] = mm;
     if (theta_lp) theta_lp[k] = __float2bfloat16_rn(th);
   }
+}
+
+// The parameter update a statistics kernel applies itself once a tile's sums over the whole batch are
+// known (Algorithm 1 / Section 3.1 applied where the sums already are, instead of in a second kernel).
+// kind: 0 none, 1 a member of the Adam family (needs sum_b G_b and sum_b G_b^2), 2 MicroSignSGD (needs
+// sum_b sign(G_b)).  theta, m, v: [d_out, d_in] fp32, updated in place; theta_lp: optional bf16 copy.
+// tile_counters: one word per thread block of the grid's x dimension, zero on entry, used when the
+// batch is split across blocks: the block that adds the last partial sum of a tile applies the update.
+enum : int { OPT_NONE = 0, OPT_ADAM = 1, OPT_SIGN = 2 };
+struct FusedOpt {
+  int kind, variant;
+  AdamParams adam;
+  SignParams sign;
+  float* theta;
+  __nv_bfloat16* theta_lp;
+  float* m;
+  float* v;
+  unsigned int* tile_counters;
+};
+
+// One parameter of the fused update; s1 = sum_b G_b (Adam) or sum_b sign(G_b) (MicroSignSGD), s2 = sum_b G_b^2.
+template <int OPT>
+__device__ __forceinline__ void fused_update_one(const FusedOpt& o, long long idx, float s1, float s2) {
+  float th = o.theta[idx], mm = o.m[idx];
+  if constexpr (OPT == OPT_ADAM) {
+    float vv = o.v[idx];
+    adam_one_rt(o.variant, th, mm, vv, s1, s2, o.adam);
+    o.v[idx] = vv;
+  } else {
+    sign_one(th, mm, s1, o.sign);
+  }
+  o.theta[idx] = th;
+  o.m[idx] = mm;
+  if (o.theta_lp) o.theta_lp[idx] = __float2bfloat16_rn(th);
 }
 
 }  // namespace pe

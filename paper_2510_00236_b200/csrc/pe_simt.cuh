@@ -6,6 +6,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include "pe_optim.cuh"
+
 namespace pe {
 
 constexpr int SIMT_TILE = 64;   // output tile edge
@@ -40,11 +42,13 @@ struct SimtExtra {
 //             out_stat[b] (Section 2.3, per-example squared norms); no [d_out, d_in] output
 // gridDim = (ceil(d_in/64), ceil(d_out/64), nsplit); block z handles examples [z*B/nsplit, (z+1)*B/nsplit).
 // With nsplit > 1 the outputs must be zero on entry and partial sums are added atomically; with
-// accumulate != 0 the results are added to whatever the outputs hold.
+// accumulate != 0 the results are added to whatever the outputs hold.  opt.kind != 0 (nsplit == 1 only):
+// the block also applies the parameter update to its tile (phi must then be square for the Adam family,
+// sign for MicroSignSGD); out_mean / out_stat may then be NULL.
 template <typename TIn, int MODE>
 __global__ void __launch_bounds__(SIMT_THREADS)
 simt_stats_kernel(const TIn* __restrict__ X, const TIn* __restrict__ dY, int B, int T, int d_in, int d_out,
-                  int phi, float* __restrict__ out_mean, float* __restrict__ out_stat, int accumulate, SimtExtra ex) {
+                  int phi, float* __restrict__ out_mean, float* __restrict__ out_stat, int accumulate, SimtExtra ex, FusedOpt opt) {
   __shared__ float sY[SIMT_TK][SIMT_TILE];
   __shared__ float sX[SIMT_TK][SIMT_TILE];
 
@@ -148,6 +152,9 @@ simt_stats_kernel(const TIn* __restrict__ X, const TIn* __restrict__ dY, int B, 
         if (nsplit == 1 && !accumulate) {
           if (out_stat) out_stat[at] = vs;
           if (MODE == MODE_STATS && out_mean) out_mean[at] = acc_mean[r][c];
+          // the parameter update of Algorithm 1 / Section 3.1, applied where the sums over the whole batch are
+          if (MODE == MODE_STATS && opt.kind == OPT_ADAM) fused_update_one<OPT_ADAM>(opt, (long long)at, acc_mean[r][c], vs);
+          if (MODE == MODE_STATS && opt.kind == OPT_SIGN) fused_update_one<OPT_SIGN>(opt, (long long)at, vs, 0.f);
         } else {
           if (out_stat) atomicAdd(out_stat + at, vs);
           if (MODE == MODE_STATS && out_mean) atomicAdd(out_mean + at, acc_mean[r][c]);

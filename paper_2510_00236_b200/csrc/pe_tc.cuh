@@ -44,6 +44,7 @@
 // 8 tokens 1 KiB further (stride byte offset), the next 64 features one box further (leading byte
 // offset).
 #pragma once
+#include "pe_optim.cuh"
 #include "pe_sm100.cuh"
 
 namespace pe {
@@ -202,12 +203,14 @@ struct RingCursor {
 // Zeroes the outputs of a split-batch launch.  The statistics kernel that follows is launched as a
 // programmatic dependent: it starts right away (it only touches the outputs in its very last step,
 // behind griddepcontrol.wait), so the zeroing costs no time on the stream.  a, b, c: n4 float4 each; b and
-// c may be NULL.
+// c may be NULL.  counters: the tile counters of a fused update (n_counters words; may be NULL).
 __global__ void __launch_bounds__(256) zero_outputs_kernel(float4* __restrict__ a, float4* __restrict__ b, float4* __restrict__ c,
-                                                           long long n4) {
+                                                           long long n4, unsigned int* __restrict__ counters, int n_counters) {
   sm100::griddep_launch_dependents();
   const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
   const long long stride = (long long)gridDim.x * blockDim.x;
+  if (counters)
+    for (long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x; k < n_counters; k += stride) counters[k] = 0u;
   for (long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x; k < n4; k += stride) {
     a[k] = z;
     if (b) b[k] = z;
@@ -221,15 +224,73 @@ enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2, MEAN_REGS_SIGN = 3, ME
 constexpr int TC_SIGN_COUNT_MAX = 32767;   // examples per block in MEAN_REGS_SIGN mode: 2 * count must fit 16 bits
 
 // gridDim = (2 * pairs_m * tiles_n, 1, nsplit); blockIdx.x = 2 * (pair index in the tile order) + rank in pair.
+// The fused parameter update of one epilogue warp's 32-row x (PANELS * 32)-column piece of the tile.  Here a
+// lane is a COLUMN (global accesses of a warp are 128 contiguous bytes of one row), whereas the running
+// sums live one ROW per lane: the sums therefore come either from the warp's staged panels in shared
+// memory (the 128-byte-swizzled 32 x 32 panels the write-out also hands to TMA; chunk k of row r sits at
+// chunk position k ^ (r & 7)) or, when the batch was split and this block added the last partial sum,
+// from the outputs in global memory (read past L1).  16 rows are in flight per lane at a time.
+template <int OPT, int PANELS>
+__device__ __forceinline__ void fused_update_piece(const FusedOpt& o, const TcParams& p, int row0, int col0, int lane,
+                                                   const uint8_t* stat_panels, const uint8_t* mean_panels) {
+  for (int c = 0; c < PANELS; ++c) {
+    if (col0 + c * 32 >= p.d_in) break;
+    const int col = col0 + c * 32 + lane;
+    const bool col_ok = col < p.d_in;
+#pragma unroll
+    for (int rb = 0; rb < 32; rb += 16) {
+      float th[16], mm[16], vv[16], s1[16], s2[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int r = rb + i;
+        const bool in = col_ok && row0 + r < p.d_out;
+        const long long idx = (long long)(row0 + r) * p.d_in + col;
+        th[i] = in ? o.theta[idx] : 0.f;
+        mm[i] = in ? o.m[idx] : 0.f;
+        vv[i] = (OPT == OPT_ADAM && in) ? o.v[idx] : 0.f;
+        float st, mn = 0.f;
+        if (stat_panels) {
+          const int off = c * 4096 + r * 128 + (((lane >> 2) ^ (r & 7)) << 4) + (lane & 3) * 4;
+          st = *reinterpret_cast<const float*>(stat_panels + off);
+          if (OPT == OPT_ADAM) mn = *reinterpret_cast<const float*>(mean_panels + off);
+        } else {
+          st = in ? __ldcg(p.out_stat + idx) : 0.f;
+          if (OPT == OPT_ADAM) mn = in ? __ldcg(p.out_mean + idx) : 0.f;
+        }
+        s1[i] = (OPT == OPT_ADAM) ? mn : st;
+        s2[i] = st;
+      }
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int r = rb + i;
+        if (col_ok && row0 + r < p.d_out) {
+          const long long idx = (long long)(row0 + r) * p.d_in + col;
+          if constexpr (OPT == OPT_ADAM) {
+            adam_one_rt(o.variant, th[i], mm[i], vv[i], s1[i], s2[i], o.adam);
+            o.v[idx] = vv[i];
+          } else {
+            sign_one(th[i], mm[i], s1[i], o.sign);
+          }
+          o.theta[idx] = th[i];
+          o.m[idx] = mm[i];
+          if (o.theta_lp) o.theta_lp[idx] = __float2bfloat16_rn(th[i]);
+        }
+      }
+    }
+  }
+}
+
 // RAGGED: packed batch with per-example token ranges (tmap_x / tmap_dy are then (d, rows, 1), tmap_x_tail /
 // tmap_dy_tail (d, 16, B) over the zero-padded last partial token groups); otherwise the tail maps are unused.
 // PHI: 0 identity, 1 square, 2 sign, 3 the clipping scale c_b * g with c_b = min(1, C / sqrt(N_b)).
-template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT), bool RAGGED = false>
+// OPT: the parameter update applied by the block that completes a tile's sums (OPT_ADAM needs both running
+// sums, OPT_SIGN the sign statistic alone); `o` is ignored when OPT == OPT_NONE.
+template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT), bool RAGGED = false, int OPT = OPT_NONE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
                 const __grid_constant__ CUtensorMap tmap_mean, const __grid_constant__ CUtensorMap tmap_stat,
                 const __grid_constant__ CUtensorMap tmap_sign, const __grid_constant__ CUtensorMap tmap_x_tail,
-                const __grid_constant__ CUtensorMap tmap_dy_tail, TcParams p) {
+                const __grid_constant__ CUtensorMap tmap_dy_tail, TcParams p, FusedOpt o) {
   using namespace sm100;
   using Op = TcOperand<TF32, NT, BKT>;
   constexpr bool TRIPLE = (MEAN == MEAN_REGS_SIGN);
@@ -241,6 +302,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   static_assert(MEAN != MEAN_TMEM || (NT == 256 && PHI != 0), "the tensor-memory mean sits beside one 256-column accumulator");
   static_assert(!RAGGED || (!TF32 && MEAN != MEAN_TMEM), "packed batches: 16-bit operands, two issuers");
   static_assert(PHI != 3 || MEAN == MEAN_NONE, "the clipped sum is a statistic-only pass");
+  static_assert(OPT != OPT_ADAM || (MEAN == MEAN_REGS && PHI == 1), "the Adam family consumes sum_b G_b and sum_b G_b^2");
+  static_assert(OPT != OPT_SIGN || (MEAN == MEAN_NONE && PHI == 2), "MicroSignSGD consumes sum_b sign(G_b)");
   constexpr int STAGES = Op::STAGES, BK = Op::BK;
   constexpr int BOX_BYTES = Op::BOX_BYTES, A_BYTES = Op::A_BYTES, STAGE_BYTES = Op::STAGE_BYTES;
   constexpr int ISSUERS = (MEAN == MEAN_TMEM) ? 1 : 2;
@@ -552,16 +615,19 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     // whatever lies outside the matrix.  The tensor-memory loads are warp-wide instructions: the
     // condition around them is made uniform over the warp.
     ok = __all_sync(0xffffffffu, ok);
+    constexpr int PANELS = COLS / 32;
+    int tile_m, tile_n;
+    tc_tile_of_block(p, rank, tile_m, tile_n);
+    // each epilogue warp stages in its own eighth of the operand ring: 6 panels of 4 KiB (7 at NT = 192)
+    constexpr int WARP_PANELS = (STAGES * STAGE_BYTES / 8) / 4096;
+    static_assert(WARP_PANELS >= PANELS, "an epilogue warp stages one output at a time");
+    static_assert(OPT != OPT_ADAM || WARP_PANELS >= 2 * PANELS, "the fused Adam update reads both staged sums");
+    const uint32_t stage_base = smem_base + (uint32_t)(warp - 4) * (uint32_t)(WARP_PANELS * 4096);
+    const int row0 = tile_m * TC_TILE_M + q * 32;
+    const int col0 = tile_n * NT + h * COLS;
+    // fused update on the unsplit schedule: the sums are staged even when the caller does not want them written
+    const bool stage_for_update = OPT != OPT_NONE && p.nsplit == 1;
     if (ok && n_acc > 0) {
-      constexpr int PANELS = COLS / 32;
-      int tile_m, tile_n;
-      tc_tile_of_block(p, rank, tile_m, tile_n);
-      // each epilogue warp stages in its own eighth of the operand ring: 6 panels of 4 KiB (7 at NT = 192)
-      constexpr int WARP_PANELS = (STAGES * STAGE_BYTES / 8) / 4096;
-      static_assert(WARP_PANELS >= PANELS, "an epilogue warp stages one output at a time");
-      const uint32_t stage_base = smem_base + (uint32_t)(warp - 4) * (uint32_t)(WARP_PANELS * 4096);
-      const int row0 = tile_m * TC_TILE_M + q * 32;
-      const int col0 = tile_n * NT + h * COLS;
       auto put_panel = [&](uint32_t panel_addr, const float* v) {      // v: this lane's 32 consecutive columns
         uint8_t* dst = smem_gen + (panel_addr - smem_base) + lane * 128;
 #pragma unroll
@@ -583,13 +649,13 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         }
       };
       // sum_b phi(G_b), or the plain contraction when PHI == 0
-      if (p.out_stat) {
+      if (p.out_stat || stage_for_update) {
 #pragma unroll
         for (int c = 0; c < PANELS; ++c) put_panel(stage_base + c * 4096, (PHI != 0) ? &acc_stat[c * 32] : &acc_mean[c * 32]);
-        send(&tmap_stat, stage_base);
+        if (p.out_stat) send(&tmap_stat, stage_base);
       }
       // sum_b G_b
-      if (p.out_mean && (KEEP_MEAN || MEAN == MEAN_TMEM)) {
+      if ((p.out_mean || (stage_for_update && OPT == OPT_ADAM)) && (KEEP_MEAN || MEAN == MEAN_TMEM)) {
         uint32_t first = stage_base + PANELS * 4096;          // MEAN_REGS / PHI == 0: second half of the warp's 16 KiB
         if constexpr (MEAN == MEAN_TMEM) {
           // the panels are needed again: wait until TMA has read the first output out of them
@@ -612,7 +678,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 #pragma unroll
           for (int c = 0; c < PANELS; ++c) put_panel(first + c * 4096, &acc_mean[c * 32]);
         }
-        send(&tmap_mean, first);
+        if (p.out_mean) send(&tmap_mean, first);
       }
       if constexpr (TRIPLE) {
         // sum_b sign(G_b): the warp's staging area is in use, so wait until TMA has read it
@@ -633,6 +699,40 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       if (lane == 0) bulk_wait_read_all();       // shared memory must outlive TMA's reads
     }
     __syncwarp();
+    if constexpr (OPT != OPT_NONE) {
+      // The parameter update, by the block that holds (unsplit batch) or has just completed (split batch)
+      // the tile's sums over the whole batch.  Split batch: every block adds its partial tile to the
+      // outputs, waits until those adds have been performed, and takes a ticket from the tile's counter;
+      // the block that draws the last ticket reads the finished sums back and applies the update.  A block
+      // that gave up on a wait marks the counter so that nobody updates the parameters from incomplete sums.
+      bool apply = ok && n_acc > 0;
+      if (p.nsplit > 1) {
+        if (lane == 0) { bulk_wait_all(); __threadfence(); }
+        __syncwarp();
+        named_bar_sync(1, 256);                   // the eight epilogue warps; executed by all of them whatever `ok` says
+        volatile int* last_flag = reinterpret_cast<volatile int*>(tail + 12);
+        if (warp == 4 && lane == 0) {
+          griddep_wait();                         // the counters are zeroed by the kernel that zeroes the outputs
+          const unsigned int inc = 1u + (*abort_flag ? 0x10000u : 0u);
+          const unsigned int now = atomicAdd(o.tile_counters + blockIdx.x, inc) + inc;
+          int last = 0;
+          if ((now & 0xffffu) == (unsigned int)p.nsplit) {
+            last = (now >> 16) ? 0 : 1;
+            atomicExch(o.tile_counters + blockIdx.x, 0u);
+          }
+          *last_flag = last;
+        }
+        named_bar_sync(1, 256);
+        apply = (*last_flag != 0);
+        if (apply) __threadfence();
+      }
+      if (apply) {
+        const bool from_smem = p.nsplit == 1;
+        const uint8_t* stat_panels = from_smem ? smem_gen + (stage_base - smem_base) : nullptr;
+        fused_update_piece<OPT, PANELS>(o, p, row0, col0, lane, stat_panels, stat_panels ? stat_panels + PANELS * 4096 : nullptr);
+      }
+      __syncwarp();
+    }
   }
 
   // ---------------------------------------------------------------- teardown
