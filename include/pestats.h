@@ -197,6 +197,28 @@ pe_status_t pe_token_sqstats_staged(const void* X, const void* dY, int B, int T,
 size_t pe_token_sqstats_staged_workspace_bytes(int B, int T, int d_in, int d_out);
 
 /*
+ * The two-pass per-token statistic (Section 2.3) with fp8 operands: as pe_token_sqstats_staged, but the
+ * scaled squares are staged as e4m3 (one byte each: half the workspace and half the staged traffic) and
+ * contracted by the 8-bit tensor-core path at twice the 16-bit rate.  Two error sources, both measured:
+ * (1) e4m3 keeps 4 significant bits, so a staged square carries up to 2^-4 relative rounding error (0.027
+ * rms, to nearest even, unbiased) and a term of the sum about 0.0375 rms, independent from row to row:
+ * with w_r = dY[r,o]^2 X[r,i]^2 >= 0 an entry's random relative error is about
+ * 0.0375 * sqrt(sum_r w_r^2) / sum_r w_r, i.e. 0.11 / sqrt(B*T) for Gaussian inputs (9e-4 at B*T = 16384),
+ * more when a few rows carry the sum; (2) the 8-bit tensor-core path aligns the products of one instruction
+ * to their largest exponent and drops what falls below its internal width, which for these all-positive
+ * sums is a systematic deficit of about 2.4e-3, whatever the number of rows.  Together: 2.6e-3 to 3.1e-3
+ * relative Frobenius error on 16384-row layers, ABOVE the 2e-3 the other routes are held to (they reach
+ * 1e-5).  An approximation to opt into where that is acceptable; pe_token_sqstats and pe_token_sqstats_staged keep
+ * 11 significant bits.  Needs d_in % 16 == 0 and d_out % 16 == 0; other tensor-core shapes are served by
+ * the half route (same workspace call, which then reports the larger size), tiny or odd ones by the SIMT
+ * kernel.  workspace: 256-byte aligned, pe_token_sqstats_fp8_workspace_bytes() bytes.
+ */
+pe_status_t pe_token_sqstats_fp8(const void* X, const void* dY, int B, int T, int d_in, int d_out,
+                                 float* out_stat, void* workspace, size_t workspace_bytes,
+                                 pe_stream_t stream);
+size_t pe_token_sqstats_fp8_workspace_bytes(int B, int T, int d_in, int d_out);
+
+/*
  * pe_token_sqstats_staged for callers that have no device memory to give as workspace and no way to
  * get some.  (The paper has no counterpart; this is a convenience of this library.)  Typical cases: a
  * plug-in that is handed input and output pointers but no allocator; a process whose framework

@@ -20,6 +20,7 @@ __all__ = [
     "microadam_family_step", "ADAM_VARIANTS", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms",
     "pe_linear_stats_ragged", "pe_linear_stats_ragged_workspace_bytes", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
     "pe_linear_microadam_step", "pe_linear_microadam_step_f32", "pe_linear_microsignsgd_step", "pe_linear_fused_workspace_bytes",
+    "pe_token_sqstats_fp8", "pe_token_sqstats_fp8_workspace_bytes",
 ]
 
 PHI_IDENTITY, PHI_SQUARE, PHI_SIGN = 0, 1, 2
@@ -34,6 +35,7 @@ EXPORTED_SYMBOLS = [
     "pe_token_sqstats_static", "microadam_family_step", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms",
     "pe_linear_stats_ragged", "pe_linear_stats_ragged_workspace_bytes", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
     "pe_linear_microadam_step", "pe_linear_microadam_step_f32", "pe_linear_microsignsgd_step", "pe_linear_fused_workspace_bytes",
+    "pe_token_sqstats_fp8", "pe_token_sqstats_fp8_workspace_bytes",
 ]
 ADAM_VARIANTS = {"adam": 0, "microadam": 1, "microadam_var": 2, "microadam_msq": 3}      # pe_adam_variant_t
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024      # PE_STATIC_SCRATCH_BYTES of pestats.h
@@ -81,6 +83,9 @@ def load_library() -> ctypes.CDLL:
     lib.pe_linear_fused_workspace_bytes.argtypes = [i, i]
     lib.pe_linear_fused_workspace_bytes.restype = sz
     lib.pe_token_sqstats_staged.argtypes = [vp, vp, i, i, i, i, vp, vp, sz, vp]
+    lib.pe_token_sqstats_fp8.argtypes = [vp, vp, i, i, i, i, vp, vp, sz, vp]
+    lib.pe_token_sqstats_fp8_workspace_bytes.argtypes = [i, i, i, i]
+    lib.pe_token_sqstats_fp8_workspace_bytes.restype = sz
     lib.pe_token_sqstats_f32.argtypes = [vp, vp, i, i, i, i, vp, vp]
     lib.pe_token_sqstats_static.argtypes = [vp, vp, i, i, i, i, vp, vp]
     lib.pe_token_sqstats_staged_workspace_bytes.argtypes = [i, i, i, i]
@@ -98,7 +103,7 @@ def load_library() -> ctypes.CDLL:
     lib.pe_reset_launch_count.argtypes = []
     lib.pe_reset_launch_count.restype = None
     for name in ("pe_linear_stats", "pe_linear_stats_f32", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms", "pe_token_sqstats", "pe_token_sqstats_f32", "pe_token_sqstats_static",
-                 "pe_token_sqstats_staged",
+                 "pe_token_sqstats_staged", "pe_token_sqstats_fp8",
                  "pe_linear_stats_ragged", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
                  "pe_linear_microadam_step", "pe_linear_microadam_step_f32", "pe_linear_microsignsgd_step",
                  "microadam_step", "microadam_family_step", "microsignsgd_step", "pe_get_async_status", "pe_set_path", "pe_last_path"):
@@ -380,6 +385,27 @@ def pe_token_sqstats_staged(X, dY, out_stat=None, workspace=None):
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     with _dev_ctx(X):
         _check("pe_token_sqstats_staged", load_library().pe_token_sqstats_staged(
+            X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, out_stat.data_ptr(), _ptr(workspace), ws_bytes, _stream(X)))
+    return out_stat
+
+
+def pe_token_sqstats_fp8_workspace_bytes(B, T, d_in, d_out) -> int:
+    return int(load_library().pe_token_sqstats_fp8_workspace_bytes(int(B), int(T), int(d_in), int(d_out)))
+
+
+def pe_token_sqstats_fp8(X, dY, out_stat=None, workspace=None):
+    """The two-pass per-token statistic with the squares staged as e4m3 and contracted at the 8-bit tensor-core
+    rate: an approximation with about 0.0375 * sqrt(sum w^2) / sum w relative error per entry (see pestats.h)."""
+    B, T, d_in, d_out = _io_check(X, dY, torch.bfloat16)
+    if out_stat is None:
+        out_stat = torch.empty((d_out, d_in), dtype=torch.float32, device=X.device)
+    _out_check("out_stat", out_stat, d_out, d_in)
+    need = pe_token_sqstats_fp8_workspace_bytes(B, T, d_in, d_out)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=X.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    with _dev_ctx(X):
+        _check("pe_token_sqstats_fp8", load_library().pe_token_sqstats_fp8(
             X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, out_stat.data_ptr(), _ptr(workspace), ws_bytes, _stream(X)))
     return out_stat
 

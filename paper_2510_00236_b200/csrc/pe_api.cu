@@ -204,23 +204,23 @@ static pe_status_t launch_pair_kernel(Kernel kernel, dim3 grid, int smem, cudaSt
 }
 
 // mxt, myt: the maps of the zero-padded tail groups of a packed batch (RAGGED); any valid map otherwise.
-template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT), bool RAGGED = false, int OPT = OPT_NONE>
+template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT), bool RAGGED = false, int OPT = OPT_NONE, bool F8 = false>
 static pe_status_t launch_tc_inst(DeviceInfo* di, int slot, const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& mm,
                                   const CUtensorMap& ms, const CUtensorMap& msgn, const TcParams& p, dim3 grid, cudaStream_t st,
                                   const CUtensorMap* mxt = nullptr, const CUtensorMap* myt = nullptr, const FusedOpt* opt = nullptr) {
   const bool after_zeroing = p.nsplit > 1 && !p.accumulate;
-  constexpr int smem = TcOperand<TF32, NT, BKT>::SMEM_BYTES;
+  constexpr int smem = TcOperand<TF32, NT, BKT, F8>::SMEM_BYTES;
   {
     std::lock_guard<std::mutex> lock(g_dev_mutex);
     if (!di->tc_attr_set[slot]) {
-      if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT, RAGGED, OPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+      if (cudaFuncSetAttribute(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT, RAGGED, OPT, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
         cudaGetLastError();
         return PE_ERR_CUDA;
       }
       di->tc_attr_set[slot] = true;
     }
   }
-  return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT, RAGGED, OPT>, grid, smem, st, after_zeroing, mx, my, mm, ms, msgn,
+  return launch_pair_kernel(tc_stats_kernel<PHI, TF32, NT, MEAN, BKT, RAGGED, OPT, F8>, grid, smem, st, after_zeroing, mx, my, mm, ms, msgn,
                             mxt ? *mxt : mx, myt ? *myt : my, p, opt ? *opt : FusedOpt{});
 }
 
@@ -864,23 +864,29 @@ pe_status_t pe_token_sqstats(const void* X, const void* dY, int B, int T, int d_
 }
 
 // Workspace of the staged per-token statistic: the column maxima of X and dY (one 32-bit word per
-// column), then the scaled squares of X and of dY as IEEE half, each part 256-byte aligned.
+// column), then the scaled squares of X and of dY (IEEE half, or e4m3 in the fp8 form), each part 256-byte aligned.
 struct StagedLayout {
   size_t max_bytes, x_bytes, y_bytes;
   size_t total() const { return max_bytes + x_bytes + y_bytes; }
 };
-static StagedLayout staged_layout(int B, int T, int d_in, int d_out) {
-  const size_t rows = (size_t)B * (size_t)T;
+static StagedLayout staged_layout(int B, int T, int d_in, int d_out, bool fp8 = false) {
+  const size_t rows = (size_t)B * (size_t)T, es = fp8 ? 1 : 2;
   StagedLayout l;
   l.max_bytes = align_up(((size_t)d_in + (size_t)d_out) * 4, 256);
-  l.x_bytes = align_up(rows * d_in * 2, 256);
-  l.y_bytes = align_up(rows * d_out * 2, 256);
+  l.x_bytes = align_up(rows * d_in * es, 256);
+  l.y_bytes = align_up(rows * d_out * es, 256);
   return l;
 }
+// the fp8 form stages one byte per element: TMA wants 16-byte row pitches
+static bool token_fp8_ok(int B, int T, int d_in, int d_out) { return token_tc_ok(B, T, d_in, d_out) && (d_in % 16) == 0 && (d_out % 16) == 0; }
 
 size_t pe_token_sqstats_staged_workspace_bytes(int B, int T, int d_in, int d_out) {
   if (g_path.load() == PE_PATH_SIMT || !token_tc_ok(B, T, d_in, d_out)) return 0;
   return staged_layout(B, T, d_in, d_out).total();
+}
+size_t pe_token_sqstats_fp8_workspace_bytes(int B, int T, int d_in, int d_out) {
+  if (g_path.load() == PE_PATH_SIMT || !token_tc_ok(B, T, d_in, d_out)) return 0;
+  return staged_layout(B, T, d_in, d_out, token_fp8_ok(B, T, d_in, d_out)).total();
 }
 
 // Grid of the column-wise staging kernels: x covers the columns in groups of 256, y slices the rows
@@ -895,9 +901,42 @@ static dim3 stage_grid(long long rows, int d, int sm_count) {
   return dim3((unsigned)gx, (unsigned)gy, 1);
 }
 
-pe_status_t pe_token_sqstats_staged(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_stat,
-                                    void* workspace, size_t workspace_bytes, pe_stream_t stream) {
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+// The plain contraction of e4m3 operands x8 [B, T, d_in], y8 [B, T, d_out] (one byte per element) into out.
+static pe_status_t launch_tc_fp8(DeviceInfo* di, const void* x8, const void* y8, int B, int T, int d_in, int d_out, float* out,
+                                 cudaStream_t st) {
+  using Op = TcOperand<false, 256, 128, true>;
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return PE_ERR_CUDA;
+  auto operand_map = [&](CUtensorMap* m, const void* base, int d) {
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)T, (cuuint64_t)B};
+    cuuint64_t strides[2] = {(cuuint64_t)d, (cuuint64_t)T * (cuuint64_t)d};
+    cuuint32_t box[3] = {(cuuint32_t)Op::BOX_FEATS, (cuuint32_t)Op::BK, 1u};
+    cuuint32_t estr[3] = {1u, 1u, 1u};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  };
+  CUtensorMap mx, my, mo;
+  if (!operand_map(&mx, x8, d_in) || !operand_map(&my, y8, d_out)) return PE_ERR_CUDA;
+  pe_status_t rc = make_output_map(&mo, out, d_in, d_out);
+  if (rc != PE_OK) return rc;
+  const int tiles_n = (d_in + 255) / 256, pairs_m = (d_out + TC_PAIR_M - 1) / TC_PAIR_M;
+  if ((long long)tiles_n * pairs_m > (1ll << 29)) return PE_ERR_DIM;
+  const int ns = choose_nsplit((long long)tiles_n * pairs_m, B, T, di->sm_count / 2 > 0 ? di->sm_count / 2 : 1, 16);
+  if (ns > 1) {
+    rc = zero_for_split(di, out, nullptr, (size_t)d_in * d_out, st);
+    if (rc != PE_OK) return rc;
+  }
+  TcParams p;
+  p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = 0; p.half_operands = 0; p.accumulate = 0;
+  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
+  p.out_mean = nullptr; p.out_stat = out; p.out_sign = nullptr; p.out_norms = nullptr; p.dev_status = di->status_ptr;
+  p.seq_offsets = nullptr; p.sq_norms = nullptr; p.clip_norm = 0.f;
+  return launch_tc_inst<0, false, 256, MEAN_NONE, 128, false, OPT_NONE, true>(di, 25, mx, my, mo, mo, mo, p, dim3(2 * pairs_m * tiles_n, 1, ns), st);
+}
+
+// The two-pass per-token statistic on half (fp8 = false) or e4m3 (fp8 = true) squares.
+static pe_status_t token_staged_impl(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_stat, void* workspace,
+                                     size_t workspace_bytes, cudaStream_t st, bool want_fp8) {
   if (!out_stat) return PE_ERR_NULL;
   pe_status_t rc = validate_stats(X, dY, B, T, d_in, d_out, out_stat, nullptr, false, 16);
   if (rc != PE_OK) return rc;
@@ -909,14 +948,15 @@ pe_status_t pe_token_sqstats_staged(const void* X, const void* dY, int B, int T,
   const bool tc_ok = token_tc_ok(B, T, d_in, d_out);
   if (forced >= PE_PATH_TENSOR && !tc_shape_ok(B, T, d_in, d_out)) return PE_ERR_UNSUPPORTED_SHAPE;
   if (tc_ok && forced != PE_PATH_SIMT) {
+    const bool fp8 = want_fp8 && token_fp8_ok(B, T, d_in, d_out);
     const long long rows = (long long)B * T;
-    const StagedLayout l = staged_layout(B, T, d_in, d_out);
+    const StagedLayout l = staged_layout(B, T, d_in, d_out, fp8);
     if (!workspace || workspace_bytes < l.total()) return PE_ERR_WORKSPACE;
     if (!aligned(workspace, 256)) return PE_ERR_ALIGN;
     uint32_t* max_x = static_cast<uint32_t*>(workspace);
     uint32_t* max_y = max_x + d_in;
-    __half* x2 = reinterpret_cast<__half*>(static_cast<char*>(workspace) + l.max_bytes);
-    __half* y2 = reinterpret_cast<__half*>(static_cast<char*>(workspace) + l.max_bytes + l.x_bytes);
+    void* x2 = static_cast<char*>(workspace) + l.max_bytes;
+    void* y2 = static_cast<char*>(workspace) + l.max_bytes + l.x_bytes;
     const uint16_t* Xb = static_cast<const uint16_t*>(X);
     const uint16_t* Yb = static_cast<const uint16_t*>(dY);
     if (cudaMemsetAsync(max_x, 0, ((size_t)d_in + (size_t)d_out) * 4, st) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
@@ -927,22 +967,36 @@ pe_status_t pe_token_sqstats_staged(const void* X, const void* dY, int B, int T,
     const StageTensor sx = {Xb, x2, max_x, d_in}, sy = {Yb, y2, max_y, d_out};
     column_max_kernel<<<grid, STAGE_THREADS, 0, st>>>(sx, sy, rows);
     if ((rc = check_launch()) != PE_OK) return rc;
-    square_to_half_kernel<<<grid, STAGE_THREADS, 0, st>>>(sx, sy, rows);
+    if (fp8) square_to_lp_kernel<true><<<grid, STAGE_THREADS, 0, st>>>(sx, sy, rows);
+    else square_to_lp_kernel<false><<<grid, STAGE_THREADS, 0, st>>>(sx, sy, rows);
     if ((rc = check_launch()) != PE_OK) return rc;
     // B and T only enter through B*T: regroup the rows into two-stage "examples" when possible so
     // the batch split has many units to balance.
-    constexpr int REGROUP = 2 * TcOperand<false, 256>::BK;
+    const int regroup = fp8 ? 2 * TcOperand<false, 256, 128, true>::BK : 2 * TcOperand<false, 256>::BK;
     int Bp = B, Tp = T;
-    if (T % REGROUP == 0 && rows / REGROUP < (1ll << 30)) { Bp = (int)(rows / REGROUP); Tp = REGROUP; }
+    if (T % regroup == 0 && rows / regroup < (1ll << 30)) { Bp = (int)(rows / regroup); Tp = regroup; }
     g_last_path.store(PE_PATH_TENSOR);
-    rc = launch_tc(di, x2, y2, Bp, Tp, d_in, d_out, PE_PHI_IDENTITY, 0, nullptr, out_stat, st, true);
+    rc = fp8 ? launch_tc_fp8(di, x2, y2, Bp, Tp, d_in, d_out, out_stat, st)
+             : launch_tc(di, x2, y2, Bp, Tp, d_in, d_out, PE_PHI_IDENTITY, 0, nullptr, out_stat, st, true);
     if (rc != PE_OK) return rc;
-    unscale_kernel<<<grid_for((long long)d_in * d_out / 4 + 4, di->sm_count), STAGE_THREADS, 0, st>>>(out_stat, d_out, d_in, max_x, max_y);
+    const int ugrid = grid_for((long long)d_in * d_out / 4 + 4, di->sm_count);
+    if (fp8) unscale_kernel<true><<<ugrid, STAGE_THREADS, 0, st>>>(out_stat, d_out, d_in, max_x, max_y);
+    else unscale_kernel<false><<<ugrid, STAGE_THREADS, 0, st>>>(out_stat, d_out, d_in, max_x, max_y);
     return check_launch();
   }
   g_last_path.store(PE_PATH_SIMT);
   return launch_simt<__nv_bfloat16, MODE_TOKEN>(di, static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(dY), B, T,
                                                 d_in, d_out, 0, nullptr, out_stat, st);
+}
+
+pe_status_t pe_token_sqstats_staged(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_stat,
+                                    void* workspace, size_t workspace_bytes, pe_stream_t stream) {
+  return token_staged_impl(X, dY, B, T, d_in, d_out, out_stat, workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream), false);
+}
+
+pe_status_t pe_token_sqstats_fp8(const void* X, const void* dY, int B, int T, int d_in, int d_out, float* out_stat,
+                                 void* workspace, size_t workspace_bytes, pe_stream_t stream) {
+  return token_staged_impl(X, dY, B, T, d_in, d_out, out_stat, workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream), true);
 }
 
 // ---------------------------------------------------------------------------------------------

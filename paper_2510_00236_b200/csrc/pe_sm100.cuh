@@ -198,13 +198,21 @@ __host__ __device__ constexpr uint32_t make_idesc_half_mn_major(int M, int N) {
 // CTA-pair MMA, issued by one thread of the pair's leader block: M rows are split between the two
 // blocks (each supplies its own A rows and receives its own accumulator rows), the N rows of B are
 // split too (each block's shared memory holds half of them at the same offset).
-template <bool TF32>
+// KIND: 0 = kind::f16 (bf16 or IEEE half operands), 1 = kind::tf32, 2 = kind::f8f6f4 (here: e4m3 operands).
+template <int KIND>
 __device__ __forceinline__ void umma_ss_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  if constexpr (TF32) {
+  if constexpr (KIND == 1) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else if constexpr (KIND == 2) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
   } else {

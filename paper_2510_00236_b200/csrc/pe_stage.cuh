@@ -13,8 +13,16 @@
 // Multiplying by a power of two is exact, so the only rounding is the one to half: at most 2^-11
 // relative per operand, to nearest even, hence unbiased.
 // All three kernels are streaming kernels bound by HBM bandwidth.
+//
+// The same route with fp8 (e4m3) operands, which the tensor cores contract at twice the 16-bit rate from
+// half the staged bytes: the squares are written as e4m3(x^2 * 2^(6 - 2e)) (below 2^8, e4m3's largest
+// finite value being 448).  e4m3 keeps 4 significant bits, so each staged square carries up to 2^-4
+// relative rounding error (to nearest even, unbiased) and each term of the sum up to about 2^-3; the
+// errors of different rows are independent and the terms non-negative, so the error of an entry falls
+// with the square root of the number of rows that carry its sum (see the error model in the host code).
 #pragma once
 #include <cuda_fp16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -28,9 +36,18 @@ __device__ __forceinline__ int stage_exponent(uint32_t max_abs_bits) {
   const int E = (int)(max_abs_bits & 0x7FFFu) >> 7;
   return E < STAGE_EXP_MIN ? STAGE_EXP_MIN : (E > STAGE_EXP_MAX ? STAGE_EXP_MAX : E);
 }
-// 2^(13 - 2 (E - 127)) and its inverse
-__device__ __forceinline__ float stage_scale(int E) { return __uint_as_float((uint32_t)(394 - 2 * E) << 23); }
-__device__ __forceinline__ float stage_inv_scale(int E) { return __uint_as_float((uint32_t)(2 * E - 140) << 23); }
+// 2^(TOP - 2 (E - 127)) and its inverse; TOP = 13 for half (scaled squares below 2^15), 6 for e4m3 (below 2^8).
+// Both stay normal floats for every clamped exponent (E <= 193 would suffice for TOP = 6: the clamp's upper
+// end is lowered by 3 there).
+template <bool FP8>
+__device__ __forceinline__ int stage_exponent_for(uint32_t max_abs_bits) {
+  const int E = stage_exponent(max_abs_bits);
+  return (FP8 && E > STAGE_EXP_MAX - 3) ? STAGE_EXP_MAX - 3 : E;
+}
+template <bool FP8>
+__device__ __forceinline__ float stage_scale(int E) { return __uint_as_float((uint32_t)((FP8 ? 387 : 394) - 2 * E) << 23); }
+template <bool FP8>
+__device__ __forceinline__ float stage_inv_scale(int E) { return __uint_as_float((uint32_t)(2 * E - (FP8 ? 133 : 140)) << 23); }
 
 // max_bits[c] = max over rows of |src[r, c]| as a bf16 bit pattern (which orders like the magnitude).
 // src: [rows, d] bf16, d a multiple of 8; max_bits: [d], zero on entry.  gridDim.x covers the columns
@@ -38,7 +55,7 @@ __device__ __forceinline__ float stage_inv_scale(int E) { return __uint_as_float
 // launch serves both.
 struct StageTensor {
   const uint16_t* src;     // [rows, d] bf16 bit patterns
-  __half* dst;             // [rows, d] scaled squares (square_to_half_kernel only)
+  void* dst;               // [rows, d] scaled squares, IEEE half or e4m3 (square_to_lp_kernel only)
   uint32_t* max_bits;      // [d]
   int d;
 };
@@ -80,13 +97,13 @@ column_max_kernel(StageTensor tx_, StageTensor ty_, long long rows) {
   }
 }
 
-// dst[r, c] = half(src[r, c]^2 * scale(c)).  Same grid and thread layout as column_max_kernel, so a
-// thread's eight columns, and with them its scales, never change.
+// dst[r, c] = half(src[r, c]^2 * scale(c)), or the same as e4m3 (FP8).  Same grid and thread layout as
+// column_max_kernel, so a thread's eight columns, and with them its scales, never change.
+template <bool FP8>
 __global__ void __launch_bounds__(STAGE_THREADS)
-square_to_half_kernel(StageTensor tx_, StageTensor ty_, long long rows) {
+square_to_lp_kernel(StageTensor tx_, StageTensor ty_, long long rows) {
   const StageTensor& tn = blockIdx.z == 0 ? tx_ : ty_;
   const uint16_t* __restrict__ src = tn.src;
-  __half* __restrict__ dst = tn.dst;
   const uint32_t* __restrict__ max_bits = tn.max_bits;
   const int d = tn.d;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
@@ -95,7 +112,7 @@ square_to_half_kernel(StageTensor tx_, StageTensor ty_, long long rows) {
   const long long r_begin = rows * blockIdx.y / gridDim.y, r_end = rows * (blockIdx.y + 1) / gridDim.y;
   float sc[8];
 #pragma unroll
-  for (int j = 0; j < 8; ++j) sc[j] = stage_scale(stage_exponent(max_bits[col + j]));
+  for (int j = 0; j < 8; ++j) sc[j] = stage_scale<FP8>(stage_exponent_for<FP8>(max_bits[col + j]));
   for (long long r = r_begin + ty; r < r_end; r += 8) {
     const uint4 v = __ldcs(reinterpret_cast<const uint4*>(src + r * d + col));
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -103,14 +120,23 @@ square_to_half_kernel(StageTensor tx_, StageTensor ty_, long long rows) {
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const float a = __uint_as_float(w[k] << 16), b = __uint_as_float(w[k] & 0xFFFF0000u);
-      const __half2 h = __floats2half2_rn(a * a * sc[2 * k], b * b * sc[2 * k + 1]);
-      o[k] = *reinterpret_cast<const uint32_t*>(&h);
+      if constexpr (FP8) {
+        o[k] = (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(a * a * sc[2 * k], b * b * sc[2 * k + 1]), __NV_SATFINITE, __NV_E4M3);
+      } else {
+        const __half2 h = __floats2half2_rn(a * a * sc[2 * k], b * b * sc[2 * k + 1]);
+        o[k] = *reinterpret_cast<const uint32_t*>(&h);
+      }
     }
-    *reinterpret_cast<uint4*>(dst + r * d + col) = make_uint4(o[0], o[1], o[2], o[3]);
+    if constexpr (FP8) {
+      *reinterpret_cast<uint2*>(static_cast<uint8_t*>(tn.dst) + r * d + col) = make_uint2(o[0] | (o[1] << 16), o[2] | (o[3] << 16));
+    } else {
+      *reinterpret_cast<uint4*>(static_cast<__half*>(tn.dst) + r * d + col) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
   }
 }
 
 // out[o, i] *= inv_scale(dY column o) * inv_scale(X column i); out: [d_out, d_in] fp32, d_in % 4 == 0.
+template <bool FP8>
 __global__ void __launch_bounds__(STAGE_THREADS)
 unscale_kernel(float* __restrict__ out, int d_out, int d_in, const uint32_t* __restrict__ max_x,
                const uint32_t* __restrict__ max_dy) {
@@ -119,12 +145,12 @@ unscale_kernel(float* __restrict__ out, int d_out, int d_in, const uint32_t* __r
   const int q_per_row = d_in / 4;
   for (long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x; k < n4; k += stride) {
     const int o = (int)(k / q_per_row), i = (int)(k - (long long)o * q_per_row) * 4;
-    const float ro = stage_inv_scale(stage_exponent(max_dy[o]));
+    const float ro = stage_inv_scale<FP8>(stage_exponent_for<FP8>(max_dy[o]));
     float4 v = reinterpret_cast<float4*>(out)[k];
-    v.x = v.x * stage_inv_scale(stage_exponent(max_x[i])) * ro;
-    v.y = v.y * stage_inv_scale(stage_exponent(max_x[i + 1])) * ro;
-    v.z = v.z * stage_inv_scale(stage_exponent(max_x[i + 2])) * ro;
-    v.w = v.w * stage_inv_scale(stage_exponent(max_x[i + 3])) * ro;
+    v.x = v.x * stage_inv_scale<FP8>(stage_exponent_for<FP8>(max_x[i])) * ro;
+    v.y = v.y * stage_inv_scale<FP8>(stage_exponent_for<FP8>(max_x[i + 1])) * ro;
+    v.z = v.z * stage_inv_scale<FP8>(stage_exponent_for<FP8>(max_x[i + 2])) * ro;
+    v.w = v.w * stage_inv_scale<FP8>(stage_exponent_for<FP8>(max_x[i + 3])) * ro;
     reinterpret_cast<float4*>(out)[k] = v;
   }
 }

@@ -69,15 +69,18 @@ __host__ __device__ constexpr int tc_smem_budget(int nt) { return (nt == 192 ? 2
 __host__ __device__ constexpr int tc_default_bk(bool tf32, int nt) { return tf32 ? 32 : (nt == 256 ? 64 : 128); }
 constexpr int TC_SHORT_BK = 32;
 constexpr int TC_SHORT_T = 32;
-template <bool TF32, int NT, int BK_ = tc_default_bk(TF32, NT)>
+// F8: 8-bit operands (kind::f8f6f4, e4m3, 32 tokens per instruction): the scaled squares of the two-pass
+// per-token statistic's fp8 form.
+template <bool TF32, int NT, int BK_ = tc_default_bk(TF32, NT), bool F8 = false>
 struct TcOperand {
-  static constexpr int ELEM_BYTES = TF32 ? 4 : 2;
-  static constexpr int BOX_FEATS = 128 / ELEM_BYTES;            // features per 128-byte swizzle row: 64 | 32
+  static_assert(!(TF32 && F8), "one operand type");
+  static constexpr int ELEM_BYTES = TF32 ? 4 : (F8 ? 1 : 2);
+  static constexpr int BOX_FEATS = 128 / ELEM_BYTES;            // features per 128-byte swizzle row: 64 | 32 | 128
   // tokens per pipeline stage (one TMA box is BK tokens tall), chosen so that the ring has an EVEN
   // number of stages: with two MMA issuers taking alternate stages every slot then always belongs
   // to the same issuer (see the parity note at the issuer's wait).
   static constexpr int BK = BK_;
-  static constexpr int MMA_K = 32 / ELEM_BYTES;                 // tokens per MMA instruction: 16 | 8
+  static constexpr int MMA_K = 32 / ELEM_BYTES;                 // tokens per MMA instruction: 16 | 8 | 32
   static constexpr int BOX_BYTES = 128 * BK;                    // one box: BK tokens x 128 bytes
   static constexpr int A_BOXES = TC_TILE_M / BOX_FEATS;         // this block's 128 rows of dY^T
   static constexpr int B_FEATS = NT / 2;                        // this block's half of the tile's d_in columns
@@ -285,14 +288,15 @@ __device__ __forceinline__ void fused_update_piece(const FusedOpt& o, const TcPa
 // PHI: 0 identity, 1 square, 2 sign, 3 the clipping scale c_b * g with c_b = min(1, C / sqrt(N_b)).
 // OPT: the parameter update applied by the block that completes a tile's sums (OPT_ADAM needs both running
 // sums, OPT_SIGN the sign statistic alone); `o` is ignored when OPT == OPT_NONE.
-template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT), bool RAGGED = false, int OPT = OPT_NONE>
+template <int PHI, bool TF32, int NT, int MEAN, int BKT = tc_default_bk(TF32, NT), bool RAGGED = false, int OPT = OPT_NONE, bool F8 = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
                 const __grid_constant__ CUtensorMap tmap_mean, const __grid_constant__ CUtensorMap tmap_stat,
                 const __grid_constant__ CUtensorMap tmap_sign, const __grid_constant__ CUtensorMap tmap_x_tail,
                 const __grid_constant__ CUtensorMap tmap_dy_tail, TcParams p, FusedOpt o) {
   using namespace sm100;
-  using Op = TcOperand<TF32, NT, BKT>;
+  using Op = TcOperand<TF32, NT, BKT, F8>;
+  static_assert(!F8 || (PHI == 0 && NT == 256 && !RAGGED), "8-bit operands: the plain contraction of the per-token statistic");
   constexpr bool TRIPLE = (MEAN == MEAN_REGS_SIGN);
   static_assert((MEAN != MEAN_REGS && !TRIPLE) || NT == 128 || (NT == 192 && !TRIPLE), "two running sums only fit the registers up to NT = 192");
   static_assert(NT != 192 || MEAN == MEAN_REGS, "the 256 x 192 tile exists for the two register-resident sums");
@@ -426,7 +430,8 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       // examples x, x+2, ... of the slice and TMEM buffers x*BUFS_PER_ISSUER .. +BUFS_PER_ISSUER-1.
       if (lane == 0) {
         const int x = (warp == 1) ? 0 : 1;
-        const uint32_t idesc = (!TF32 && p.half_operands) ? make_idesc_half_mn_major(TC_PAIR_M, NT) : make_idesc_mn_major(TC_PAIR_M, NT, TF32);
+        // operand format code 0 is IEEE half under kind::f16 and e4m3 under kind::f8f6f4
+        const uint32_t idesc = (F8 || (!TF32 && p.half_operands)) ? make_idesc_half_mn_major(TC_PAIR_M, NT) : make_idesc_mn_major(TC_PAIR_M, NT, TF32);
         bool ok = true;
         uint32_t accumulate = 0;
         constexpr int SUB = STAGES / ISSUERS;              // slots of this issuer's sub-ring
@@ -458,7 +463,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
               if (k * Op::MMA_K < t_left) {
                 const uint64_t ad = make_smem_desc(a_src + k * Op::K_STEP_BYTES, BOX_BYTES, Op::SBO_BYTES, Op::DESC_LAYOUT);
                 const uint64_t bd = make_smem_desc(b_src + k * Op::B_K_STEP_BYTES, Op::B_BOX_BYTES, Op::B_SBO_BYTES, Op::B_DESC_LAYOUT);
-                umma_ss_pair<TF32>(d_tmem, ad, bd, idesc, accumulate);
+                umma_ss_pair<TF32 ? 1 : (F8 ? 2 : 0)>(d_tmem, ad, bd, idesc, accumulate);
                 accumulate = 1;
               }
             }

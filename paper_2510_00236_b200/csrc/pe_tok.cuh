@@ -152,7 +152,7 @@ tok_sqstats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
           for (int k = 0; k < TOK_BK / TOK_MMA_K; ++k) {       // rows past the end are zero: no need to skip them
             const uint64_t ad = make_smem_desc(a_src + k * TOK_MMA_K * 128, TOK_BOX_BYTES, 512u, 1u);
             const uint64_t bd = make_smem_desc(b_src + k * TOK_MMA_K * 128, TOK_BOX_BYTES, 512u, 1u);
-            umma_ss_pair<true>(tmem_base, ad, bd, idesc, accumulate);
+            umma_ss_pair<1>(tmem_base, ad, bd, idesc, accumulate);
             accumulate = 1;
           }
           umma_commit_pair(cooked_empty(c));             // cooked stage reusable in both blocks once these MMAs retire
