@@ -237,7 +237,14 @@ size_t pe_token_sqstats_fp8_workspace_bytes(int B, int T, int d_in, int d_out);
  * workspace for those.
  * First call on a device: looks up the array's device address (a host-side query, done once per
  * device with that device current) before enqueuing; make that first call outside any stream
- * capture.
+ * capture.  The array belongs to the one device module that holds all of this library's kernels, and
+ * CUDA loads a module when its first kernel or symbol is used: a process that is going to hand the
+ * whole GPU to a memory pool must make its first call into this library on each device (any entry
+ * point) BEFORE doing so, or the module load itself fails for want of 32 MiB and every pestats call
+ * on that device returns PE_ERR_CUDA.
+ * Speed: every shape that fits the array is small enough that the one-kernel pe_token_sqstats, which
+ * needs no workspace either, is the faster route; this entry point is for callers that want the two-pass
+ * route's arithmetic (IEEE-half squares at the full 16-bit tensor rate) without owning memory.
  * Sharing: all calls on a device use the same array and it keeps whatever the previous call left
  * there.  Each call overwrites the part it reads before reading it, so stale contents never reach
  * a result; but two calls whose kernels can overlap on the GPU (different streams, no dependency
@@ -340,6 +347,14 @@ const char* pe_status_string(pe_status_t status);
  * (a kernel gave up on a bounded wait; its outputs are invalid), or PE_ERR_CUDA.  If `detail` is not
  * NULL it receives a host int identifying the wait that expired (0 if none). */
 pe_status_t pe_get_async_status(pe_stream_t stream, int* detail);
+
+/* Cycle budget of every wait inside the tensor-core kernels on the CURRENT device (each wait of a thread
+ * on an on-chip barrier is bounded; a wait that exhausts the budget makes its kernel give up cleanly,
+ * skip its outputs and latch PE_ERR_TIMEOUT for pe_get_async_status).  The default, restored by
+ * cycles <= 0, is 2^32 cycles (about two seconds), far beyond any wait of a healthy launch; tests lower it
+ * to a few cycles to drive the give-up path, which makes ordinary launches time out.  Synchronous (a
+ * small host-to-device copy); set it while no library kernel is running on the device. */
+pe_status_t pe_set_wait_limit_cycles(long long cycles);
 
 /* Process-wide override of the kernel family (for tests and benchmarks). Returns the previous value. */
 int pe_set_path(int path /* pe_path_t */);

@@ -20,7 +20,7 @@ __all__ = [
     "microadam_family_step", "ADAM_VARIANTS", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms",
     "pe_linear_stats_ragged", "pe_linear_stats_ragged_workspace_bytes", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
     "pe_linear_microadam_step", "pe_linear_microadam_step_f32", "pe_linear_microsignsgd_step", "pe_linear_fused_workspace_bytes",
-    "pe_token_sqstats_fp8", "pe_token_sqstats_fp8_workspace_bytes",
+    "pe_token_sqstats_fp8", "pe_token_sqstats_fp8_workspace_bytes", "pe_set_wait_limit_cycles",
 ]
 
 PHI_IDENTITY, PHI_SQUARE, PHI_SIGN = 0, 1, 2
@@ -35,7 +35,7 @@ EXPORTED_SYMBOLS = [
     "pe_token_sqstats_static", "microadam_family_step", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms",
     "pe_linear_stats_ragged", "pe_linear_stats_ragged_workspace_bytes", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
     "pe_linear_microadam_step", "pe_linear_microadam_step_f32", "pe_linear_microsignsgd_step", "pe_linear_fused_workspace_bytes",
-    "pe_token_sqstats_fp8", "pe_token_sqstats_fp8_workspace_bytes",
+    "pe_token_sqstats_fp8", "pe_token_sqstats_fp8_workspace_bytes", "pe_set_wait_limit_cycles",
 ]
 ADAM_VARIANTS = {"adam": 0, "microadam": 1, "microadam_var": 2, "microadam_msq": 3}      # pe_adam_variant_t
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024      # PE_STATIC_SCRATCH_BYTES of pestats.h
@@ -97,6 +97,8 @@ def load_library() -> ctypes.CDLL:
     lib.pe_status_string.restype = ctypes.c_char_p
     lib.pe_get_async_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
     lib.pe_set_path.argtypes = [i]
+    lib.pe_set_wait_limit_cycles.argtypes = [ll]
+    lib.pe_set_wait_limit_cycles.restype = i
     lib.pe_last_path.argtypes = []
     lib.pe_launch_count.argtypes = []
     lib.pe_launch_count.restype = ll
@@ -387,6 +389,15 @@ def pe_token_sqstats_staged(X, dY, out_stat=None, workspace=None):
         _check("pe_token_sqstats_staged", load_library().pe_token_sqstats_staged(
             X.data_ptr(), dY.data_ptr(), B, T, d_in, d_out, out_stat.data_ptr(), _ptr(workspace), ws_bytes, _stream(X)))
     return out_stat
+
+
+def pe_set_wait_limit_cycles(cycles: int, device=None) -> None:
+    """Cycle budget of the waits inside the tensor-core kernels on `device` (default: the current one);
+    cycles <= 0 restores the default.  For tests of the PE_ERR_TIMEOUT path."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    with torch.cuda.device(dev):
+        torch.cuda.synchronize()
+        _check("pe_set_wait_limit_cycles", load_library().pe_set_wait_limit_cycles(int(cycles)))
 
 
 def pe_token_sqstats_fp8_workspace_bytes(B, T, d_in, d_out) -> int:

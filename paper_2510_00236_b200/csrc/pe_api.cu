@@ -1140,6 +1140,15 @@ pe_status_t pe_get_async_status(pe_stream_t stream, int* detail) {
   return PE_ERR_TIMEOUT;
 }
 
+pe_status_t pe_set_wait_limit_cycles(long long cycles) {
+  DeviceInfo* di = nullptr;
+  pe_status_t rc = device_info(&di);
+  if (rc != PE_OK) return rc;
+  const long long v = cycles > 0 ? cycles : sm100::WAIT_CYCLE_LIMIT_DEFAULT;
+  if (cudaMemcpyToSymbol(sm100::g_wait_cycle_limit, &v, sizeof v) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
+  return PE_OK;
+}
+
 int pe_set_path(int path) {
   if (path < PE_PATH_AUTO || path > PE_PATH_TENSOR_WIDE) return -1;
   return g_path.exchange(path);

@@ -92,10 +92,13 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   unsigned int spins = 0;
+  // the budget and the abort flag are looked at every 256 polls; with a budget below 2^20 cycles (only a
+  // test sets one) at every poll, so that such a budget is honoured to within one poll
+  const unsigned int check_mask = wait_cycle_limit() < (1ll << 20) ? 0u : 0xffu;
   while (true) {
     if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
     if (mbar_try_wait(bar, parity)) return true;
-    if ((++spins & 0xff) == 0) {
+    if ((++spins & check_mask) == 0) {
       if (*abort_flag) return false;
       if (clock64() - t0 > wait_cycle_limit()) {
         *abort_flag = 1;

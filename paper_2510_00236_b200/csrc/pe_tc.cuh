@@ -410,7 +410,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
           bool progressed = try_fill(ca, 0);
           if (ISSUERS == 2 && try_fill(cb, 1)) progressed = true;
           if (progressed) { t0 = -1; spins = 0; continue; }
-          if ((++spins & 0xffu) == 0) {                  // bounded like every other wait
+          if ((++spins & (wait_cycle_limit() < (1ll << 20) ? 0u : 0xffu)) == 0) {      // bounded like every other wait
             if (*abort_flag) break;
             if (t0 < 0) t0 = clock64();
             else if (clock64() - t0 > wait_cycle_limit()) {

@@ -175,8 +175,9 @@ tok_sqstats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
       for (long long n = grp; n < c_end - c_begin; n += 2) {
         const int s = (int)(n % TOK_RAW_STAGES);          // raw and cooked rings advance together (same depth)
         const uint32_t ph = (uint32_t)(n / TOK_RAW_STAGES) & 1u;
-        if (!mbar_wait_bounded(raw_full(s), ph, abort_flag, p.dev_status, TOK_WAIT_RAW_FULL)) { ok = false; break; }
-        if (!mbar_wait_bounded(cooked_empty(s), ph ^ 1u, abort_flag, p.dev_status, TOK_WAIT_COOKED_EMPTY)) { ok = false; break; }
+        // every lane polls, the warp acts on one answer (what follows contains warp-wide instructions)
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(raw_full(s), ph, abort_flag, p.dev_status, TOK_WAIT_RAW_FULL))) { ok = false; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(cooked_empty(s), ph ^ 1u, abort_flag, p.dev_status, TOK_WAIT_COOKED_EMPTY))) { ok = false; break; }
         const uint8_t* raw = smem_gen + s * TOK_RAW_STAGE;
         uint8_t* cooked = smem_gen + TOK_RAW_STAGES * TOK_RAW_STAGE + s * TOK_COOKED_STAGE;
         // A stage is 1024 16-byte chunks (4 boxes x 32 rows x 8 chunks of 8 features); chunk g of the
@@ -214,7 +215,8 @@ tok_sqstats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
       }
     }
     static_assert(TOK_RAW_STAGES == TOK_COOKED_STAGES && TOK_RAW_STAGES % 2 == 0, "the two rings advance together; each slot belongs to one converter group");
-    if (ok) ok = mbar_wait_bounded(acc_full, 0, abort_flag, p.dev_status, TOK_WAIT_ACC);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(acc_full, 0, abort_flag, p.dev_status, TOK_WAIT_ACC));
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       // Write-out as in the statistics kernel: 32 rows x 128 columns per warp, staged in the idle ring

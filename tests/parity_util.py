@@ -23,6 +23,24 @@ def rel_frob(a: np.ndarray, ref: np.ndarray) -> float:
     return float(num / den) if den > 0 else float(num)
 
 
+def assert_entries_close(a, ref, what, rel_rms=1e-3):
+    """Per-entry bound beside the Frobenius one: no single entry may be off by more than rel_rms times the
+    reference's rms (observed deviations are around 1e-7 of it; one wrong entry among millions is of order 1)."""
+    a = np.asarray(a, np.float64)
+    ref = np.asarray(ref, np.float64)
+    scale = float(np.sqrt(np.mean(ref ** 2)))
+    worst = float(np.max(np.abs(a - ref))) if a.size else 0.0
+    assert worst <= rel_rms * scale + 1e-30, f"{what}: an entry is off by {worst:.3e} (rms of the reference {scale:.3e})"
+
+
+def assert_token_entries_close(a, ref, what):
+    """Per-token statistic: all terms are non-negative and each squared operand is rounded to 11 bits, so every
+    entry must be within 2e-3 of its own exact value."""
+    a = np.asarray(a, np.float64)
+    ref = np.asarray(ref, np.float64)
+    assert np.all(np.abs(a - ref) <= 2e-3 * np.abs(ref) + 1e-30), f"{what}: an entry is off by more than 2e-3 of its value"
+
+
 def boundary_and_random(n: int, k: int, seed: int, tile: int = 128) -> list[int]:
     """Sample of indices in [0, n): tile edges (first/last element of the first, second and last tile)
     plus seeded random ones."""
@@ -85,21 +103,25 @@ def check_all(li_full: inputs.LayerInputs, rows=None, cols=None, phis=("square",
         assert np.isfinite(mean).all() and np.isfinite(stat).all(), "unwritten or non-finite outputs"
         e = rel_frob(mean, st.sum_g)
         assert e <= tol, f"sum_b G_b: rel. Frobenius error {e:.3e} > {tol}"
+        assert_entries_close(mean, st.sum_g, f"sum_b G_b ({phi})")
         report[f"mean_err_{phi}"] = e
         if phi == "square":
             e = rel_frob(stat, st.sum_g2)
             assert e <= tol, f"sum_b G_b^2: rel. Frobenius error {e:.3e} > {tol}"
+            assert_entries_close(stat, st.sum_g2, "sum_b G_b^2")
             report["square_err"] = e
         elif phi == "sign":
             report["sign_disagreements"] = check_sign(stat, st)
         else:
             e = rel_frob(stat, st.sum_g)
             assert e <= tol
+            assert_entries_close(stat, st.sum_g, "sum_b G_b (identity)")
     if token:
         t = pick(gpu_token(li_full))
         assert np.isfinite(t).all()
         e = rel_frob(t, tok)
         assert e <= tol, f"per-token statistic: rel. Frobenius error {e:.3e} > {tol}"
+        assert_token_entries_close(t, tok, "per-token statistic")
         report["token_err"] = e
     if bench_calls:
         # the calls the benchmark step makes: all three statistics in one pass, the two-pass per-token statistic
@@ -113,11 +135,15 @@ def check_all(li_full: inputs.LayerInputs, rows=None, cols=None, phis=("square",
         assert np.isfinite(mean).all() and np.isfinite(sq).all() and np.isfinite(sgn).all()
         report["one_pass_mean_err"], report["one_pass_square_err"] = rel_frob(mean, st.sum_g), rel_frob(sq, st.sum_g2)
         assert report["one_pass_mean_err"] <= tol and report["one_pass_square_err"] <= tol
+        assert_entries_close(mean, st.sum_g, "one-pass sum_b G_b")
+        assert_entries_close(sq, st.sum_g2, "one-pass sum_b G_b^2")
         report["one_pass_sign_disagreements"] = check_sign(sgn, st)
         t = pick(pe.pe_token_sqstats_staged(li_full.X, li_full.dY).cpu().numpy())
         assert np.isfinite(t).all()
         report["token_two_pass_err"] = rel_frob(t, tok)
         assert report["token_two_pass_err"] <= tol
+        assert_token_entries_close(t, tok, "two-pass per-token statistic")
+        report["oracle_stats"] = st
     status, detail = pe.pe_get_async_status(li_full.X.device)
     assert status == 0, f"device status {status} detail {detail}"
     return report

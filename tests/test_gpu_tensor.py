@@ -7,7 +7,7 @@ import torch
 import oracle
 import paper_2510_00236_b200 as pe
 from paper_2510_00236_b200 import inputs
-from parity_util import boundary_and_random, check_all, gpu_stats
+from parity_util import boundary_and_random, check_all, gpu_stats, rel_frob
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -306,6 +306,7 @@ def test_config2_full_size_sampled_outputs():
     rows = boundary_and_random(2048, 40, 1)
     cols = boundary_and_random(512, 32, 2)
     rep = check_all(li, rows, cols, bench_calls=True)
+    rep.pop("oracle_stats", None)
     assert pe.pe_last_path() == pe.PATH_TENSOR
     print("config2", rep)
 
@@ -315,12 +316,42 @@ def test_config4_full_size_sampled_outputs():
     rows = boundary_and_random(8192, 24, 3)
     cols = boundary_and_random(2048, 24, 4)
     rep = check_all(li, rows, cols, bench_calls=True)
+    st = rep.pop("oracle_stats")
     print("config4", rep)
-    del li
+    # ... followed by the MicroSignSGD step on the fp32 master weights (beta = 0.9, lr = 3.47e-3, m_0 = 0), with the
+    # bf16 copy: once as the separate update kernel on the sign statistic, once fused into the statistics kernel
+    B, d_out, d_in = li.shape[0], 8192, 2048
+    kw = dict(lr=3.47e-3, beta=0.9)
+    pick = lambda t: t.float().cpu().numpy().astype(np.float64)[np.ix_(rows, cols)]
+    W0 = pick(li.W)
+    th_ref, m_ref = oracle.microsignsgd_step(W0, np.zeros_like(W0), st.sum_sign, B, **kw)
+    slack = 2.0 * st.n_small / B * (1.0 - kw["beta"])            # what the examples below the sign threshold may move m by
+    sgn = torch.empty((d_out, d_in), device=DEV)
+    pe.pe_linear_stats(li.X, li.dY, "sign", None, sgn)
+    for fused in (False, True):
+        th, m = li.W.clone(), torch.zeros((d_out, d_in), device=DEV)
+        lp = torch.empty((d_out, d_in), dtype=torch.bfloat16, device=DEV)
+        if fused:
+            ws = torch.empty(pe.pe_linear_fused_workspace_bytes(d_in, d_out), dtype=torch.uint8, device=DEV)
+            pe.pe_linear_microsignsgd_step(li.X, li.dY, th, m, theta_lp=lp, out_sign=sgn, workspace=ws, **kw)
+        else:
+            pe.microsignsgd_step(th, m, sgn, B, theta_lp=lp, **kw)
+        torch.cuda.synchronize()
+        assert np.all(np.abs(pick(m) - m_ref) <= slack + 1e-7), fused
+        assert np.all(np.abs(pick(th) - th_ref) <= kw["lr"] * slack + 1e-7), fused
+        exact = st.n_small == 0
+        # the update itself (fp32 master weights hold it to about 1e-4 of its size), at the tolerance for updated parameters
+        from parity_util import FROB_TOL
+        assert rel_frob((pick(th) - W0)[exact], (th_ref - W0)[exact]) <= FROB_TOL
+        assert torch.equal(lp, th.to(torch.bfloat16))
+        del th, m, lp
+    assert pe.pe_get_async_status(DEV) == (0, 0)
+    del li, sgn
     torch.cuda.empty_cache()
 
 
-@pytest.mark.parametrize("B,T,d", [(16, 32, 1024), (16, 4096, 1024), (1024, 32, 1024), (128, 512, 4096), (1024, 512, 1024)])
+@pytest.mark.parametrize("d", inputs.SWEEP_D)
+@pytest.mark.parametrize("B,T", inputs.SWEEP_BT)
 def test_config5_points_sampled_outputs(B, T, d):
     li = inputs.config5_point(B, T, d, DEV)
     rows = boundary_and_random(d, 16, 5)
@@ -328,6 +359,22 @@ def test_config5_points_sampled_outputs(B, T, d):
     check_all(li, rows, cols)
     del li
     torch.cuda.empty_cache()
+
+
+def test_sign_counters_force_a_batch_split_beyond_32767_examples_per_block():
+    """The one-pass kernel counts sign(G_b) + 1 in 16-bit halves of a register, good for 32767 examples per
+    block; with more examples than 16 x 32767 the host must split the batch further than it otherwise would."""
+    B, T, d = 16 * 32767 + 40, 33, 8
+    li = inputs.gaussian_layer(B, T, d, d, seed=123, device=DEV)
+    outs = [torch.full((d, d), float("nan"), device=DEV) for _ in range(3)]
+    pe.pe_linear_stats_all(li.X, li.dY, *outs)
+    torch.cuda.synchronize()
+    assert pe.pe_last_path() == pe.PATH_TENSOR and pe.pe_get_async_status(DEV) == (0, 0)
+    from parity_util import check_sign, oracle_on, rel_frob, FROB_TOL
+    st, _ = oracle_on(li)
+    assert rel_frob(outs[0].cpu().numpy(), st.sum_g) <= FROB_TOL and rel_frob(outs[1].cpu().numpy(), st.sum_g2) <= FROB_TOL
+    check_sign(outs[2].cpu().numpy(), st)
+    assert float(outs[2].abs().max()) <= B
 
 
 def test_staged_token_stat_requires_workspace():

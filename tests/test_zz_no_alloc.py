@@ -13,9 +13,10 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2510_00236_b200 as pe
 from paper_2510_00236_b200 import inputs
-from parity_util import FROB_TOL, rel_frob
+from parity_util import FROB_TOL, assert_token_entries_close, rel_frob
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -37,10 +38,17 @@ def _both_ways(li):
     got = torch.full((d_out, d_in), float("nan"), device=DEV)
     lib = pe.load_library()
     stream = torch.cuda.current_stream().cuda_stream
+    torch.cuda.synchronize()
+    # the call must neither allocate nor free: the device's free memory and torch's own books stay as they are,
+    # and it launches exactly the kernels of the two-pass route (two staging passes, the zeroing kernel of a
+    # split row range if any, the contraction, the unscaling)
+    free_before, torch_before, launches_before = torch.cuda.mem_get_info(0)[0], torch.cuda.memory_allocated(), pe.pe_launch_count()
     status = lib.pe_token_sqstats_static(li.X.data_ptr(), li.dY.data_ptr(), B, T, d_in, d_out, got.data_ptr(), stream)
     assert status == 0, pe.pe_status_string(status)
     assert pe.pe_last_path() == pe.PATH_TENSOR
     torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info(0)[0] == free_before and torch.cuda.memory_allocated() == torch_before
+    assert pe.pe_launch_count() - launches_before in (4, 5)
     assert pe.pe_get_async_status(DEV) == (0, 0)
     return got.cpu().numpy(), want.cpu().numpy()
 
@@ -48,11 +56,16 @@ def _both_ways(li):
 def test_static_scratch_matches_workspace_version_twice_in_a_row():
     first = inputs.gaussian_layer(12, 128, 264, 392, seed=901, device=DEV)        # 2 MB of staging, ragged tiles
     second = inputs.heavy_tailed_layer(5, 64, 136, 128, seed=902, device=DEV)     # smaller: reuses the array's front
+    _both_ways(first)          # warm-up: the first call on a device looks the array's address up
     for li in (first, second):
         got, want = _both_ways(li)
         assert np.isfinite(got).all()
         assert rel_frob(got, want) <= FROB_TOL
         assert np.all(got >= 0)
+        # and against the oracle, not only against the library's other entry point
+        ref = oracle.token_sqstats(inputs.to_numpy_bits(li.X), inputs.to_numpy_bits(li.dY))
+        assert rel_frob(got, ref) <= FROB_TOL
+        assert_token_entries_close(got, ref, "static-scratch per-token statistic")
     # and the first shape again, now over the second call's leftovers
     got, want = _both_ways(first)
     assert rel_frob(got, want) <= FROB_TOL
