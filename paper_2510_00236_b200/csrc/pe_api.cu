@@ -34,6 +34,10 @@ constexpr int TC_MEAN_TMEM_MIN_T = 4096;
 // tile's padding (columns up to the next multiple of 192) eats the gain.
 constexpr int TC_WIDE_MIN_T = 64;
 constexpr int TC_WIDE_MAX_PAD_PERCENT = 13;
+// The three-statistic pass on the 256 x 192 tile keeps two thirds of sum_b G_b in tensor memory (a read, an add
+// and a write per example): it needs longer sequences than the two-sum kernel to hide that epilogue (measured: 6-8 % faster
+// than the 256 x 128 one-pass kernel at T = 512 and 1024, 10 % slower at T = 256).
+constexpr int TC_WIDE_TRIPLE_MIN_T = 512;
 constexpr int PHI_CLIP_SCALE = 3;   // internal phi of the clipped sum: c_b * G_b (not part of pe_phi_t)
 constexpr int TC_BAND = 8;          // pair rows per band of the tile order (8 x 256 rows of d_out)
 
@@ -237,8 +241,9 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   const int forced = g_path.load();
   // 256 x 192 tile: 22 % less operand traffic per flop than 256 x 128
   const long long pad192 = (long long)((d_in + 191) / 192) * 192, pad128 = (long long)((d_in + 127) / 128) * 128;
-  const bool wide = both && !triple && forced != PE_PATH_TENSOR_NARROW &&
-                    (forced == PE_PATH_TENSOR_WIDE || (T >= TC_WIDE_MIN_T && pad192 * 100 <= pad128 * (100 + TC_WIDE_MAX_PAD_PERCENT)));
+  const bool wide = both && forced != PE_PATH_TENSOR_NARROW &&
+                    (forced == PE_PATH_TENSOR_WIDE || (T >= (triple ? TC_WIDE_TRIPLE_MIN_T : TC_WIDE_MIN_T) &&
+                                                       pad192 * 100 <= pad128 * (100 + TC_WIDE_MAX_PAD_PERCENT)));
   const bool mean_regs = both && (triple || wide || T < TC_MEAN_TMEM_MIN_T || forced == PE_PATH_TENSOR_NARROW);
   const int nt = mean_regs ? (wide ? 192 : 128) : 256;
   const int box_feats = TcOperand<false, 256>::BOX_FEATS;
@@ -273,6 +278,7 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   p.seq_offsets = nullptr; p.sq_norms = sq_norms; p.clip_norm = clip_norm;
   dim3 grid(2 * pairs_m * tiles_n, 1, ns);
   if (phi == PHI_CLIP_SCALE) return launch_tc_inst<3, false, 256, MEAN_NONE>(di, 14, mx, my, mm, ms, msgn, p, grid, st);
+  if (triple && wide) return launch_tc_inst<1, false, 192, MEAN_HYBRID_SIGN>(di, 26, mx, my, mm, ms, msgn, p, grid, st);
   if (triple) return launch_tc_inst<1, false, 128, MEAN_REGS_SIGN>(di, 10, mx, my, mm, ms, msgn, p, grid, st);
   if (!per_example) return launch_tc_inst<0, false, 256, MEAN_NONE>(di, 4, mx, my, mm, ms, msgn, p, grid, st);
   if (short_seq) {

@@ -15,6 +15,9 @@
 //                        warps shrink to 48 registers so that the epilogue warps can take 232) -- both outputs
 //   MEAN_REGS_SIGN, NT = 128: the same plus sum_b sign(G_b), counted in 16-bit halves
 //                        of 32 more registers                                      -- mean, square and sign in one pass
+//   MEAN_HYBRID_SIGN, NT = 192: mean, square and sign on the wider tile: sum_b G_b^2 (96 registers), the sign
+//                        counts (48) and a third of sum_b G_b (32) in registers, the other two thirds of
+//                        sum_b G_b in the 128 tensor-memory columns the two accumulators leave free
 //   MEAN_TMEM, NT = 256: sum_b phi(G_b) in 128 registers per thread, sum_b G_b in
 //                        tensor memory beside ONE per-example accumulator, one issuer -- both outputs
 //   MEAN_NONE, NT = 256: one running sum per thread (128 registers)               -- only sum_b phi(G_b) wanted
@@ -223,7 +226,7 @@ __global__ void __launch_bounds__(256) zero_outputs_kernel(float4* __restrict__ 
 
 // where sum_b G_b is kept in per-example mode; MEAN_REGS_SIGN = MEAN_REGS with phi = square plus the sign statistic
 // MEAN_NORMS keeps no [d_out, d_in] sums at all: it reduces each G_b tile to its sum of squares
-enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2, MEAN_REGS_SIGN = 3, MEAN_NORMS = 4 };
+enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2, MEAN_REGS_SIGN = 3, MEAN_NORMS = 4, MEAN_HYBRID_SIGN = 5 };
 constexpr int TC_SIGN_COUNT_MAX = 32767;   // examples per block in MEAN_REGS_SIGN mode: 2 * count must fit 16 bits
 
 // gridDim = (2 * pairs_m * tiles_n, 1, nsplit); blockIdx.x = 2 * (pair index in the tile order) + rank in pair.
@@ -297,9 +300,11 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   using namespace sm100;
   using Op = TcOperand<TF32, NT, BKT, F8>;
   static_assert(!F8 || (PHI == 0 && NT == 256 && !RAGGED), "8-bit operands: the plain contraction of the per-token statistic");
-  constexpr bool TRIPLE = (MEAN == MEAN_REGS_SIGN);
-  static_assert((MEAN != MEAN_REGS && !TRIPLE) || NT == 128 || (NT == 192 && !TRIPLE), "two running sums only fit the registers up to NT = 192");
-  static_assert(NT != 192 || MEAN == MEAN_REGS, "the 256 x 192 tile exists for the two register-resident sums");
+  constexpr bool HYBRID = (MEAN == MEAN_HYBRID_SIGN);
+  constexpr bool TRIPLE = (MEAN == MEAN_REGS_SIGN) || HYBRID;
+  static_assert((MEAN != MEAN_REGS && MEAN != MEAN_REGS_SIGN) || NT == 128 || (NT == 192 && MEAN == MEAN_REGS), "two running sums only fit the registers up to NT = 192");
+  static_assert(NT != 192 || MEAN == MEAN_REGS || HYBRID, "the 256 x 192 tile exists for both running sums");
+  static_assert(!HYBRID || (NT == 192 && !RAGGED && OPT == OPT_NONE), "the hybrid mean fills the tensor-memory columns two 192-column accumulators leave free");
   static_assert(!TRIPLE || PHI == 1, "the three-statistic mode is mean + square + sign");
   constexpr bool NORMS = (MEAN == MEAN_NORMS);
   static_assert(!NORMS || (PHI == 1 && NT == 256), "per-example norms: squares on the 256 x 256 tile");
@@ -480,9 +485,12 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     setmaxnreg_inc<Op::REGS_EPILOGUE>();
     const int q = warp & 3;                 // TMEM lane quadrant this warp may access
     const int h = (warp - 4) >> 2;          // column half of the tile
-    constexpr bool KEEP_MEAN = MEAN == MEAN_REGS || TRIPLE || PHI == 0;     // running sum of G_b in registers
+    constexpr bool KEEP_MEAN = MEAN == MEAN_REGS || MEAN == MEAN_REGS_SIGN || PHI == 0;     // running sum of G_b in registers
     constexpr int N_STAT = (PHI != 0 && !NORMS) ? COLS : 1;
-    constexpr int N_MEAN = KEEP_MEAN ? COLS : 1;
+    // HYBRID: of a thread's 96 columns the first 64 have their running sum of G_b in tensor memory (columns
+    // HYB_COL0 + 64 h ..), the last 32 in registers
+    constexpr int HYB_TMEM_COLS = 64, HYB_COL0 = 2 * 192;
+    constexpr int N_MEAN = KEEP_MEAN ? COLS : (HYBRID ? COLS - HYB_TMEM_COLS : 1);
     float acc_stat[N_STAT], acc_mean[N_MEAN];
     // TRIPLE: sum_b (sign(G_b) + 1) of two neighbouring columns in one register, as unsigned 16-bit
     // halves (each at most 2 nb <= 65534, so a plain 32-bit add never carries from one half into the
@@ -539,6 +547,45 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             if (a != 0) r[j] = __float_as_uint(g + __uint_as_float(m[j]));
           }
           tmem_st_32x32b_x16(maddr + c * 16, r);
+        }
+        tmem_st_wait();
+      } else if constexpr (HYBRID) {
+        const uint32_t maddr = lane_base + (uint32_t)(HYB_COL0 + h * HYB_TMEM_COLS);
+#pragma unroll
+        for (int c = 0; c < COLS / 16; ++c) {
+          constexpr int LAST = COLS / 16 - 1;
+          const bool in_tmem = c * 16 < HYB_TMEM_COLS;           // compile-time after unrolling
+          uint32_t r[16], m[16];
+          if (in_tmem && a != 0) tmem_ld_32x32b_x16_pair_wait(taddr + c * 16, r, maddr + c * 16, m);
+          else tmem_ld_32x32b_x16_wait(taddr + c * 16, r);
+          if (c == LAST) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));   // G_b read: the issuer may start its next example
+          }
+#pragma unroll
+          for (int j = 0; j < 16; j += 2) {
+            const uint64_t g2 = f32x2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+            const uint64_t s2 = f32x2_fma(g2, g2, f32x2_pack(acc_stat[c * 16 + j], acc_stat[c * 16 + j + 1]));
+            f32x2_unpack(s2, acc_stat[c * 16 + j], acc_stat[c * 16 + j + 1]);
+            const float t0 = phi_apply<2>(__uint_as_float(r[j])) + 12582913.f;
+            const float t1 = phi_apply<2>(__uint_as_float(r[j + 1])) + 12582913.f;
+            acc_cnt[(c * 16 + j) >> 1] += __byte_perm(__float_as_uint(t0), __float_as_uint(t1), 0x5410);
+            if (in_tmem) {
+              if (a != 0) {
+                const uint64_t m2 = f32x2_add(f32x2_pack(__uint_as_float(m[j]), __uint_as_float(m[j + 1])), g2);
+                float lo, hi;
+                f32x2_unpack(m2, lo, hi);
+                r[j] = __float_as_uint(lo);
+                r[j + 1] = __float_as_uint(hi);
+              }
+            } else {
+              const int k = c * 16 + j - HYB_TMEM_COLS;
+              const uint64_t m2 = f32x2_add(f32x2_pack(acc_mean[k], acc_mean[k + 1]), g2);
+              f32x2_unpack(m2, acc_mean[k], acc_mean[k + 1]);
+            }
+          }
+          if (in_tmem) tmem_st_32x32b_x16(maddr + c * 16, r);      // the first example just writes G_b
         }
         tmem_st_wait();
       } else if constexpr (NORMS) {
@@ -660,9 +707,19 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         if (p.out_stat) send(&tmap_stat, stage_base);
       }
       // sum_b G_b
-      if ((p.out_mean || (stage_for_update && OPT == OPT_ADAM)) && (KEEP_MEAN || MEAN == MEAN_TMEM)) {
+      if ((p.out_mean || (stage_for_update && OPT == OPT_ADAM)) && (KEEP_MEAN || MEAN == MEAN_TMEM || HYBRID)) {
         uint32_t first = stage_base + PANELS * 4096;          // MEAN_REGS / PHI == 0: second half of the warp's 16 KiB
-        if constexpr (MEAN == MEAN_TMEM) {
+        if constexpr (HYBRID) {
+          // two panels from tensor memory, the third from registers; staged behind the statistic's three panels
+          const uint32_t maddr = lane_base + (uint32_t)(HYB_COL0 + h * HYB_TMEM_COLS);
+#pragma unroll
+          for (int c = 0; c < HYB_TMEM_COLS / 32; ++c) {
+            uint32_t m[32];
+            tmem_ld_32x32b_x32_wait(maddr + c * 32, m);
+            put_panel(first + c * 4096, reinterpret_cast<const float*>(m));
+          }
+          put_panel(first + (HYB_TMEM_COLS / 32) * 4096, &acc_mean[0]);
+        } else if constexpr (MEAN == MEAN_TMEM) {
           // the panels are needed again: wait until TMA has read the first output out of them
           if (lane == 0) bulk_wait_read_all();
           __syncwarp();

@@ -104,6 +104,29 @@ def test_register_mean_kernel_at_any_sequence_length(B, T, d_in, d_out):
     assert pe.pe_last_path() == pe.PATH_TENSOR
 
 
+@pytest.mark.parametrize("B,T,d_in,d_out", [(5, 200, 136, 264), (40, 96, 384, 256), (3, 2000, 264, 520), (33, 300, 776, 264),
+                                            (9, 48, 320, 192), (1, 1000, 200, 128), (70, 64, 8, 8)])
+def test_three_statistics_on_the_wide_tile(B, T, d_in, d_out):
+    """The one-pass mean + square + sign kernel on the 256 x 192 tile (two thirds of sum_b G_b in tensor memory,
+    a third in registers), forced on shapes with ragged tiles, one and many examples per block, split batches."""
+    from parity_util import FROB_TOL, assert_entries_close, check_sign, oracle_on, rel_frob
+    pe.pe_set_path(pe.PATH_TENSOR_WIDE)
+    li = inputs.heterogeneous_layer(B, T, d_in, d_out, seed=1700 + B, device=DEV, with_weights=False)
+    outs = [torch.full((d_out, d_in), float("nan"), device=DEV) for _ in range(3)]
+    launches0 = pe.pe_launch_count()
+    pe.pe_linear_stats_all(li.X, li.dY, *outs)
+    torch.cuda.synchronize()
+    assert pe.pe_get_async_status(DEV) == (0, 0) and pe.pe_last_path() == pe.PATH_TENSOR
+    assert pe.pe_launch_count() - launches0 <= 2
+    mean, sq, sgn = (o.cpu().numpy() for o in outs)
+    assert np.isfinite(mean).all() and np.isfinite(sq).all() and np.isfinite(sgn).all()
+    st, _ = oracle_on(li)
+    assert rel_frob(mean, st.sum_g) <= FROB_TOL and rel_frob(sq, st.sum_g2) <= FROB_TOL
+    assert_entries_close(mean, st.sum_g, "sum_b G_b")
+    assert_entries_close(sq, st.sum_g2, "sum_b G_b^2")
+    check_sign(sgn, st)
+
+
 def test_wide_tile_structured_inputs_catch_layout_mistakes():
     """The 256 x 192 tile loads X in 64-byte rows with the 64-byte swizzle.  Distinct small integers per
     (token, feature), exactly representable in bf16: a wrong swizzle, stride or column offset of that
