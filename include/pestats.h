@@ -155,8 +155,8 @@ pe_status_t pe_linear_stats_accumulate(const void* X, const void* dY, int B, int
  * bf16 inputs as for pe_linear_stats; all three outputs [d_out, d_in] fp32, 16-byte aligned, non-NULL,
  * overwritten.  Each G_b tile is formed once and feeds all three running sums (the sign sum is kept
  * as a per-column count), so the call costs about one pe_linear_stats(square) instead of that plus a
- * pe_linear_stats(sign).  Shapes the one-pass kernel does not take (sequences of at most 32 tokens,
- * widths that are not multiples of 8, the SIMT path forced) are served by those two calls.
+ * pe_linear_stats(sign).  Shapes the one-pass kernel does not take (widths that are not multiples of 8,
+ * the SIMT path forced) are served by those two calls.
  */
 pe_status_t pe_linear_stats_all(const void* X, const void* dY, int B, int T, int d_in, int d_out,
                                 float* out_mean, float* out_square, float* out_sign, pe_stream_t stream);

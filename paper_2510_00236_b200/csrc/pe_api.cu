@@ -112,13 +112,13 @@ static pe_status_t check_launch() {
 // chunks for fp32: the MN-major tf32 MMA accepts no other layout).  rows64: 64 bytes of features per box row with
 // the 64-byte swizzle (X of the 256 x 192 tile).  Tokens past T and features past d read as zero.
 static pe_status_t make_operand_map(CUtensorMap* m, const void* base, int B, int T, int d, bool f32, int box_feats, int box_tokens,
-                                    bool rows64 = false) {
+                                    bool rows64 = false, int box_examples = 1) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return PE_ERR_CUDA;
   const cuuint64_t es = f32 ? 4ull : 2ull;
   cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)T, (cuuint64_t)B};
   cuuint64_t strides[2] = {(cuuint64_t)d * es, (cuuint64_t)T * (cuuint64_t)d * es};
-  cuuint32_t box[3] = {(cuuint32_t)box_feats, (cuuint32_t)box_tokens, 1u};
+  cuuint32_t box[3] = {(cuuint32_t)box_feats, (cuuint32_t)box_tokens, (cuuint32_t)box_examples};
   cuuint32_t estr[3] = {1u, 1u, 1u};
   CUresult r = enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -247,13 +247,15 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   const bool mean_regs = both && (triple || wide || T < TC_MEAN_TMEM_MIN_T || forced == PE_PATH_TENSOR_NARROW);
   const int nt = mean_regs ? (wide ? 192 : 128) : 256;
   const int box_feats = TcOperand<false, 256>::BOX_FEATS;
-  const bool short_seq = mean_regs && !wide && !triple && T <= TC_SHORT_T;      // many short examples, both outputs: small stages
+  const bool short_seq = mean_regs && !wide && T <= TC_SHORT_T;      // many short examples, both sums in registers: small stages
   const int box_tokens = short_seq ? TC_SHORT_BK : tc_default_bk(false, nt);
   CUtensorMap mx, my;
+  // short sequences: a box is two examples deep (a stage holds two examples of 32 tokens each)
+  const int box_examples = short_seq ? TcOperand<false, 128, TC_SHORT_BK>::GROUP : 1;
   pe_status_t rc = wide ? make_operand_map(&mx, X, B, T, d_in, false, TcOperand<false, 192>::B_BOX_FEATS, box_tokens, true)
-                        : make_operand_map(&mx, X, B, T, d_in, false, box_feats, box_tokens);
+                        : make_operand_map(&mx, X, B, T, d_in, false, box_feats, box_tokens, false, box_examples);
   if (rc != PE_OK) return rc;
-  rc = make_operand_map(&my, dY, B, T, d_out, false, box_feats, box_tokens);
+  rc = make_operand_map(&my, dY, B, T, d_out, false, box_feats, box_tokens, false, box_examples);
   if (rc != PE_OK) return rc;
   CUtensorMap mm, ms;       // an output that is not wanted gets the other one's map and is never used
   rc = make_output_map(&mm, out_mean ? out_mean : out_stat, d_in, d_out);
@@ -279,6 +281,7 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   dim3 grid(2 * pairs_m * tiles_n, 1, ns);
   if (phi == PHI_CLIP_SCALE) return launch_tc_inst<3, false, 256, MEAN_NONE>(di, 14, mx, my, mm, ms, msgn, p, grid, st);
   if (triple && wide) return launch_tc_inst<1, false, 192, MEAN_HYBRID_SIGN>(di, 26, mx, my, mm, ms, msgn, p, grid, st);
+  if (triple && short_seq) return launch_tc_inst<1, false, 128, MEAN_REGS_SIGN, TC_SHORT_BK>(di, 27, mx, my, mm, ms, msgn, p, grid, st);
   if (triple) return launch_tc_inst<1, false, 128, MEAN_REGS_SIGN>(di, 10, mx, my, mm, ms, msgn, p, grid, st);
   if (!per_example) return launch_tc_inst<0, false, 256, MEAN_NONE>(di, 4, mx, my, mm, ms, msgn, p, grid, st);
   if (short_seq) {
@@ -659,9 +662,8 @@ pe_status_t pe_linear_stats_all(const void* X, const void* dY, int B, int T, int
   rc = device_info(&di);
   if (rc != PE_OK) return rc;
   const int forced = g_path.load();
-  // One pass when the tensor-core kernel takes the shape and an example spans more than a short
-  // stage; otherwise the two calls this one stands for.
-  if (B > 0 && T > TC_SHORT_T && forced != PE_PATH_SIMT && tc_shape_ok(B, T, d_in, d_out)) {
+  // One pass when the tensor-core kernel takes the shape; otherwise the two calls this one stands for.
+  if (B > 0 && T > 0 && forced != PE_PATH_SIMT && tc_shape_ok(B, T, d_in, d_out)) {
     g_last_path.store(PE_PATH_TENSOR);
     return launch_tc(di, X, dY, B, T, d_in, d_out, PE_PHI_SQUARE, 1, out_mean, out_square, st, false, out_sign);
   }

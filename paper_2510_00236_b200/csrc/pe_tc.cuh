@@ -84,7 +84,11 @@ struct TcOperand {
   // to the same issuer (see the parity note at the issuer's wait).
   static constexpr int BK = BK_;
   static constexpr int MMA_K = 32 / ELEM_BYTES;                 // tokens per MMA instruction: 16 | 8 | 32
-  static constexpr int BOX_BYTES = 128 * BK;                    // one box: BK tokens x 128 bytes
+  // Short sequences (the 32-token stages of the 256 x 128 tile): a stage holds TWO examples (the TMA box is
+  // two examples deep, 32 tokens each), the issuer fills both of its accumulators from it and the epilogue
+  // drains both behind one barrier: half the barrier hand-offs per example, which is what bounds T <= 32.
+  static constexpr int GROUP = (!TF32 && !F8 && NT == 128 && BK_ == TC_SHORT_BK) ? 2 : 1;
+  static constexpr int BOX_BYTES = 128 * BK * GROUP;            // one box: GROUP x BK tokens x 128 bytes
   static constexpr int A_BOXES = TC_TILE_M / BOX_FEATS;         // this block's 128 rows of dY^T
   static constexpr int B_FEATS = NT / 2;                        // this block's half of the tile's d_in columns
   // NT = 192: 96 columns of X per block are one and a half 128-byte rows.  X is then loaded in
@@ -94,7 +98,7 @@ struct TcOperand {
   static_assert(!B_NARROW || !TF32, "64-byte rows are only set up for 16-bit operands");
   static constexpr int B_ROW_BYTES = B_NARROW ? 64 : 128;
   static constexpr int B_BOX_FEATS = B_ROW_BYTES / ELEM_BYTES;  // 64 | 32
-  static constexpr int B_BOX_BYTES = B_ROW_BYTES * BK;
+  static constexpr int B_BOX_BYTES = B_ROW_BYTES * BK * GROUP;
   static constexpr int B_BOXES = B_FEATS / B_BOX_FEATS;         // 1 | 2 | 3
   static constexpr int A_BYTES = A_BOXES * BOX_BYTES;           // 32 KiB (BK = 128) | 16 KiB
   static constexpr int B_BYTES = B_BOXES * B_BOX_BYTES;         // 16 KiB | 24 KiB (NT = 192)
@@ -318,6 +322,12 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   constexpr int ISSUERS = (MEAN == MEAN_TMEM) ? 1 : 2;
   constexpr int ACC_BUFS = (MEAN == MEAN_TMEM) ? 1 : Op::ACC_BUFS;
   constexpr int BUFS_PER_ISSUER = ACC_BUFS / ISSUERS;     // 2 | 1
+  // GROUP examples share a stage and a pair of accumulator barriers (short sequences): the unit of work of
+  // the producers, issuers and epilogue warps is then a group of GROUP consecutive examples
+  constexpr int GROUP = Op::GROUP;
+  constexpr int UNITS_PER_ISSUER = BUFS_PER_ISSUER / GROUP;      // accumulator units (of GROUP buffers) per issuer
+  static_assert(GROUP == 1 || ((MEAN == MEAN_REGS || MEAN == MEAN_REGS_SIGN) && !RAGGED && OPT == OPT_NONE && UNITS_PER_ISSUER == 1),
+                "grouped examples: the short-sequence variants of the two- and three-sum kernels");
   constexpr int MEAN_COL0 = 256;                    // first tensor-memory column of the MEAN_TMEM running sum
   constexpr int COLS = NT / 2;                      // accumulator columns per epilogue thread
   extern __shared__ uint8_t smem_raw[];
@@ -338,6 +348,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
   const int b_begin = (int)(((long long)p.B * blockIdx.z) / p.nsplit);
   const int b_end = (int)(((long long)p.B * (blockIdx.z + 1)) / p.nsplit);
   const int nb = b_end - b_begin;
+  const int nu = (nb + GROUP - 1) / GROUP;          // units of work: groups of GROUP examples (GROUP = 1: the examples)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -376,13 +387,13 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         constexpr int SUB = STAGES / ISSUERS;            // slots per sub-ring
         auto start = [&](RingCursor& c, int x) {
           c.e = x; c.kc = 0; c.n = 0;
-          if (c.e < nb) c.g = seq_geom<RAGGED>(p, b_begin + c.e, BK);
+          if (c.e < nu) c.g = seq_geom<RAGGED>(p, b_begin + GROUP * c.e, BK);
         };
         // Fills the next stage of sub-ring x if it has one and its slot is free; never blocks, because a
         // sub-ring may stay full for as long as the OTHER one has to be filled (its issuer waits for an
         // accumulator that the epilogue frees only after the other issuer's example).
         auto try_fill = [&](RingCursor& c, int x) -> bool {
-          if (c.e >= nb) return false;
+          if (c.e >= nu) return false;
           const int s = ISSUERS * (c.n % SUB) + x;
           const uint32_t ph = (uint32_t)(c.n / SUB) & 1u;
           if (!mbar_test_wait(empty_bar(s), ph ^ 1u)) return false;
@@ -395,23 +406,24 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
               tma_load_3d_pair(dst + g * box_bytes, tail ? tmap_tail : tmap, leader_full, c0 + g * box_feats,
                                tail ? 0 : c.g.row0 + c.kc * BK, tail ? b_begin + c.e : 0);
           } else {
+            // (grouped examples: the box is GROUP examples deep; past the batch's end it reads zeros)
             for (int g = 0; g < n_boxes; ++g)
-              tma_load_3d_pair(dst + g * box_bytes, tmap, leader_full, c0 + g * box_feats, c.kc * BK, b_begin + c.e);
+              tma_load_3d_pair(dst + g * box_bytes, tmap, leader_full, c0 + g * box_feats, c.kc * BK, b_begin + GROUP * c.e);
           }
           ++c.n;
           if (++c.kc == c.g.nk) {
             c.kc = 0;
             c.e += ISSUERS;
-            if (c.e < nb) c.g = seq_geom<RAGGED>(p, b_begin + c.e, BK);
+            if (c.e < nu) c.g = seq_geom<RAGGED>(p, b_begin + GROUP * c.e, BK);
           }
           return true;
         };
         RingCursor ca, cb;
         start(ca, 0);
-        start(cb, ISSUERS == 2 ? 1 : nb);
+        start(cb, ISSUERS == 2 ? 1 : nu);
         long long t0 = -1;
         unsigned int spins = 0;
-        while (ca.e < nb || cb.e < nb) {
+        while (ca.e < nu || cb.e < nu) {
           bool progressed = try_fill(ca, 0);
           if (ISSUERS == 2 && try_fill(cb, 1)) progressed = true;
           if (progressed) { t0 = -1; spins = 0; continue; }
@@ -442,17 +454,17 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         constexpr int SUB = STAGES / ISSUERS;              // slots of this issuer's sub-ring
         int i_local = 0;                                   // examples this issuer has started
         int n_local = 0;                                   // stages this issuer has consumed
-        for (int e = x; e < nb && ok; e += ISSUERS, ++i_local) {
-          const SeqGeom sg = seq_geom<RAGGED>(p, b_begin + e, BK);
+        for (int e = x; e < nu && ok; e += ISSUERS, ++i_local) {
+          const SeqGeom sg = seq_geom<RAGGED>(p, b_begin + GROUP * e, BK);
           const int grp = p.per_example ? i_local : 0;
-          const int buf = BUFS_PER_ISSUER * x + (grp % BUFS_PER_ISSUER);
+          const int buf = UNITS_PER_ISSUER * x + (grp % UNITS_PER_ISSUER);      // accumulator unit: GROUP buffers, one barrier pair
           if (p.per_example || i_local == 0) {
-            const uint32_t acc_ph = (uint32_t)(grp / BUFS_PER_ISSUER) & 1u;
+            const uint32_t acc_ph = (uint32_t)(grp / UNITS_PER_ISSUER) & 1u;
             if (!mbar_wait_bounded(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, p.dev_status, TC_WAIT_ACC_EMPTY)) { ok = false; break; }
             tc_fence_after();
             accumulate = 0;
           }
-          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * NT);
+          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * GROUP * NT);
           for (int kc = 0; kc < sg.nk; ++kc, ++n_local) {
             const int s = ISSUERS * (n_local % SUB) + x;
             const uint32_t ph = (uint32_t)(n_local / SUB) & 1u;
@@ -463,18 +475,24 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             // tokens of this example in this stage: the rest of its whole 16-token groups, or the padded tail group
             const int t_left = (RAGGED && kc >= sg.nk_main) ? 16 : sg.main - kc * BK;
 #pragma unroll
-            for (int k = 0; k < BK / Op::MMA_K; ++k) {
-              // rows past T are zero-filled by TMA; whole MMA steps past T are skipped
-              if (k * Op::MMA_K < t_left) {
-                const uint64_t ad = make_smem_desc(a_src + k * Op::K_STEP_BYTES, BOX_BYTES, Op::SBO_BYTES, Op::DESC_LAYOUT);
-                const uint64_t bd = make_smem_desc(b_src + k * Op::B_K_STEP_BYTES, Op::B_BOX_BYTES, Op::B_SBO_BYTES, Op::B_DESC_LAYOUT);
-                umma_ss_pair<TF32 ? 1 : (F8 ? 2 : 0)>(d_tmem, ad, bd, idesc, accumulate);
-                accumulate = 1;
+            for (int j = 0; j < GROUP; ++j) {
+              // grouped examples: example j of the group sits BK tokens further in every box and has its own accumulator
+              if (GROUP > 1) { if (GROUP * e + j >= nb) break; accumulate = 0; }
+#pragma unroll
+              for (int k = 0; k < BK / Op::MMA_K; ++k) {
+                // rows past T are zero-filled by TMA; whole MMA steps past T are skipped
+                if (k * Op::MMA_K < t_left) {
+                  const uint64_t ad = make_smem_desc(a_src + j * (BK * 128) + k * Op::K_STEP_BYTES, BOX_BYTES, Op::SBO_BYTES, Op::DESC_LAYOUT);
+                  const uint64_t bd = make_smem_desc(b_src + j * (BK * Op::B_ROW_BYTES) + k * Op::B_K_STEP_BYTES, Op::B_BOX_BYTES, Op::B_SBO_BYTES,
+                                                     Op::B_DESC_LAYOUT);
+                  umma_ss_pair<TF32 ? 1 : (F8 ? 2 : 0)>(d_tmem + (uint32_t)(j * NT), ad, bd, idesc, accumulate);
+                  accumulate = 1;
+                }
               }
             }
             umma_commit_pair(empty_bar(s));                // stage reusable in both blocks once these MMAs retire
           }
-          const bool last_of_group = p.per_example || (e + ISSUERS >= nb);
+          const bool last_of_group = p.per_example || (e + ISSUERS >= nu);
           if (ok && last_of_group) umma_commit_pair(acc_full_bar(buf));   // accumulator complete, both blocks
         }
       }
@@ -506,12 +524,12 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     bool ok = true;
     // per-example mode: one accumulator per example, in example order (example e -> issuer e&1).
     // plain mode: one accumulator per issuer that had work.
-    const int n_acc = p.per_example ? nb : (nb >= ISSUERS ? ISSUERS : nb);
+    const int n_acc = p.per_example ? nu : (nu >= ISSUERS ? ISSUERS : nu);
     const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
     for (int a = 0; a < n_acc; ++a) {
       const int x = a % ISSUERS, grp = p.per_example ? (a / ISSUERS) : 0;
-      const int buf = BUFS_PER_ISSUER * x + (grp % BUFS_PER_ISSUER);
-      const uint32_t acc_ph = (uint32_t)(grp / BUFS_PER_ISSUER) & 1u;
+      const int buf = UNITS_PER_ISSUER * x + (grp % UNITS_PER_ISSUER);        // accumulator unit (GROUP buffers)
+      const uint32_t acc_ph = (uint32_t)(grp / UNITS_PER_ISSUER) & 1u;
       // PHI == 3: this example's clipping coefficient c_b = min(1, C / sqrt(N_b)); the load is issued before
       // the wait for the accumulator, which hides its latency.  N_b = 0 (a zero gradient) gives 1.
       uint64_t coef2 = 0;
@@ -525,7 +543,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       // instructions, so no lane may leave the loop alone when its own wait is the one that gives up
       if (!__all_sync(0xffffffffu, mbar_wait_bounded(acc_full_bar(buf), acc_ph, abort_flag, p.dev_status, TC_WAIT_ACC_FULL))) { ok = false; break; }
       tc_fence_after();
-      const uint32_t taddr = lane_base + (uint32_t)(buf * NT + h * COLS);
+      const uint32_t taddr = lane_base + (uint32_t)(buf * GROUP * NT + h * COLS);
       if constexpr (MEAN == MEAN_TMEM) {
         // sum_b G_b lives in tensor-memory columns MEAN_COL0.. of the same lanes: read it with G_b,
         // add, write it back (the first example just writes G_b).
@@ -618,16 +636,11 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
       } else {
         // CH columns per tensor-memory read: 32, or 16 where the two running sums leave few registers (NT = 192)
         constexpr int CH = (NT == 192) ? 16 : 32;
-#pragma unroll
-        for (int c = 0; c < COLS / CH; ++c) {
-          uint32_t r[CH];
-          if constexpr (CH == 32) tmem_ld_32x32b_x32_wait(taddr + c * CH, r);
-          else tmem_ld_32x32b_x16_wait(taddr + c * CH, r);
-          if (c == COLS / CH - 1) {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));   // buffer free for the issuer's next example
-          }
+        constexpr int NCH = COLS / CH;                // reads per example
+        // grouped examples: the unit's accumulators one after the other; the unit is released after the last read
+        const int in_unit = (GROUP > 1) ? min(GROUP, nb - GROUP * a) : 1;
+        // phi and the running sums for one read of CH columns (chunk c of this thread's COLS columns)
+        auto fold = [&](const uint32_t (&r)[CH], int c) {
           if constexpr (PHI == 2) {
 #pragma unroll
             for (int j = 0; j < CH; ++j) {
@@ -655,6 +668,48 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 const float t1 = phi_apply<2>(__uint_as_float(r[j + 1])) + 12582913.f;
                 acc_cnt[(c * CH + j) >> 1] += __byte_perm(__float_as_uint(t0), __float_as_uint(t1), 0x5410);
               }
+            }
+          }
+        };
+        auto release_unit = [&]() {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));   // buffer(s) free for the issuer's next example(s)
+        };
+        // Where the registers allow two reads in flight (running sums of at most 128 floats beside two 32-column
+        // reads), the reads are software-pipelined: read k+1 is issued before the arithmetic on read k, so only the
+        // first read of a unit exposes the tensor-memory latency.  That latency, paid twice per example, was a third
+        // of the epilogue's time per example, which is what bounds short sequences.
+        constexpr bool PIPELINED = CH == 32 && !TRIPLE && PHI != 3;
+        if constexpr (PIPELINED) {
+          constexpr int TOTAL = GROUP * NCH;          // reads per unit when every example of the group exists
+          const int n_reads = in_unit * NCH;
+          uint32_t ra[CH], rb[CH];
+          tmem_ld_32x32b_x32_issue(taddr, ra);
+#pragma unroll
+          for (int k = 0; k < TOTAL; ++k) {
+            if (GROUP > 1 && k >= n_reads) break;
+            if (k & 1) tmem_ld_wait_for(rb); else tmem_ld_wait_for(ra);
+            if (k + 1 < n_reads) {
+              const uint32_t next = taddr + (uint32_t)(((k + 1) / NCH) * NT + ((k + 1) % NCH) * CH);
+              if (k & 1) tmem_ld_32x32b_x32_issue(next, ra); else tmem_ld_32x32b_x32_issue(next, rb);
+            } else {
+              release_unit();
+            }
+            if (k & 1) fold(rb, k % NCH); else fold(ra, k % NCH);
+          }
+        } else {
+#pragma unroll
+          for (int ju = 0; ju < GROUP; ++ju) {
+            if (GROUP > 1 && ju >= in_unit) break;
+            const uint32_t taddr_j = taddr + (uint32_t)(ju * NT);
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+              uint32_t r[CH];
+              if constexpr (CH == 32) tmem_ld_32x32b_x32_wait(taddr_j + c * CH, r);
+              else tmem_ld_32x32b_x16_wait(taddr_j + c * CH, r);
+              if (c == NCH - 1 && ju == in_unit - 1) release_unit();
+              fold(r, c);
             }
           }
         }

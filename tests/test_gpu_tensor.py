@@ -203,8 +203,10 @@ def test_staged_token_stat_keeps_every_column_accurate_over_a_wide_range_of_magn
     (1, 1000, 256, 128, True),     # single example
     (2, 4100, 136, 264, True),     # very long sequences stay on the one-pass kernel
     (64, 256, 512, 2048, True),    # the benchmark layer, sampled below
-    (9, 16, 320, 192, False),      # short sequences: served by the two separate calls
-    (21, 32, 136, 520, False),     # exactly one short stage per example: still the two calls
+    (9, 16, 320, 192, True),       # short sequences: the one-pass kernel on 32-token stages
+    (21, 32, 136, 520, True),      # exactly one short stage per example
+    (130, 32, 264, 392, True),     # many short sequences, batch split
+    (2, 1, 64, 72, True),          # rank-one gradients
     (21, 64, 136, 520, True),      # half-filled stages
 ])
 def test_three_statistics_in_one_pass(B, T, d_in, d_out, tensor_one_pass):
