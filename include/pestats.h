@@ -315,7 +315,15 @@ pe_status_t microsignsgd_step(float* theta, void* theta_lp, float* m, const floa
  * block per tile walks all examples: correct, slower on layers with few tiles).  B >= 1, T >= 1; other
  * arguments as for pe_linear_stats and microadam_family_step.  The _f32 form takes fp32 inputs (SIMT
  * kernel, never splits the batch).  After PE_ERR_TIMEOUT the parameters of unfinished tiles are left as
- * they were.
+ * they were (the two-kernel sequence skips its update kernel while the device status word is set, i.e.
+ * until pe_get_async_status has read and cleared it).
+ * What the fusion buys is MEMORY, not time: with out_mean = out_stat = NULL no [d_out, d_in] statistic
+ * buffer exists anywhere (2 x 4 bytes per parameter saved).  In time the update inside the statistics
+ * kernel is a latency-bound tail of every tile during which that block's tensor cores idle (about 25 us
+ * per tile and block, measured), while a separate update kernel streams at the HBM rate.  By default
+ * (PE_FUSED_AUTO) the call therefore fuses only when it was given no statistic buffers and otherwise
+ * runs the statistics kernel and the update kernel back to back on `stream`; pe_set_fused_update
+ * overrides that choice.
  */
 pe_status_t pe_linear_microadam_step(const void* X, const void* dY, int B, int T, int d_in, int d_out,
                                      float* theta, void* theta_lp, float* m, float* v, float* out_mean,
@@ -339,6 +347,12 @@ pe_status_t pe_linear_microsignsgd_step(const void* X, const void* dY, int B, in
                                         size_t workspace_bytes, pe_stream_t stream);
 /* Bytes of workspace the two calls above can use (one 32-bit counter per thread block of the widest grid). */
 size_t pe_linear_fused_workspace_bytes(int d_in, int d_out);
+/* How pe_linear_microadam_step / pe_linear_microsignsgd_step run on the tensor-core path (process-wide;
+ * returns the previous mode, -1 for an unknown one): AUTO = one fused launch when no statistic buffers
+ * were given, the two-kernel sequence otherwise; ALWAYS = the fused launch whenever possible; NEVER =
+ * the two-kernel sequence (the statistic buffers are then required: PE_ERR_NULL without them). */
+typedef enum { PE_FUSED_AUTO = 0, PE_FUSED_ALWAYS = 1, PE_FUSED_NEVER = 2 } pe_fused_mode_t;
+int pe_set_fused_update(int mode /* pe_fused_mode_t */);
 
 /* Human-readable name of a status code (static storage). */
 const char* pe_status_string(pe_status_t status);

@@ -21,10 +21,12 @@ __all__ = [
     "pe_linear_stats_ragged", "pe_linear_stats_ragged_workspace_bytes", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
     "pe_linear_microadam_step", "pe_linear_microadam_step_f32", "pe_linear_microsignsgd_step", "pe_linear_fused_workspace_bytes",
     "pe_token_sqstats_fp8", "pe_token_sqstats_fp8_workspace_bytes", "pe_set_wait_limit_cycles",
+    "pe_set_fused_update", "FUSED_AUTO", "FUSED_ALWAYS", "FUSED_NEVER",
 ]
 
 PHI_IDENTITY, PHI_SQUARE, PHI_SIGN = 0, 1, 2
 PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_NARROW, PATH_TENSOR_WIDE = 0, 1, 2, 3, 4
+FUSED_AUTO, FUSED_ALWAYS, FUSED_NEVER = 0, 1, 2      # pe_fused_mode_t
 _PHI_NAMES = {"identity": PHI_IDENTITY, "square": PHI_SQUARE, "sign": PHI_SIGN}
 
 # every symbol include/pestats.h declares
@@ -36,6 +38,7 @@ EXPORTED_SYMBOLS = [
     "pe_linear_stats_ragged", "pe_linear_stats_ragged_workspace_bytes", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
     "pe_linear_microadam_step", "pe_linear_microadam_step_f32", "pe_linear_microsignsgd_step", "pe_linear_fused_workspace_bytes",
     "pe_token_sqstats_fp8", "pe_token_sqstats_fp8_workspace_bytes", "pe_set_wait_limit_cycles",
+    "pe_set_fused_update",
 ]
 ADAM_VARIANTS = {"adam": 0, "microadam": 1, "microadam_var": 2, "microadam_msq": 3}      # pe_adam_variant_t
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024      # PE_STATIC_SCRATCH_BYTES of pestats.h
@@ -97,6 +100,8 @@ def load_library() -> ctypes.CDLL:
     lib.pe_status_string.restype = ctypes.c_char_p
     lib.pe_get_async_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
     lib.pe_set_path.argtypes = [i]
+    lib.pe_set_fused_update.argtypes = [i]
+    lib.pe_set_fused_update.restype = i
     lib.pe_set_wait_limit_cycles.argtypes = [ll]
     lib.pe_set_wait_limit_cycles.restype = i
     lib.pe_last_path.argtypes = []
@@ -509,6 +514,11 @@ def pe_get_async_status(device=None):
     with torch.cuda.device(dev):
         st = load_library().pe_get_async_status(torch.cuda.current_stream(dev).cuda_stream, ctypes.byref(detail))
     return int(st), int(detail.value)
+
+
+def pe_set_fused_update(mode: int) -> int:
+    """Chooses how the statistics + update calls run (FUSED_AUTO / FUSED_ALWAYS / FUSED_NEVER); returns the previous mode."""
+    return int(load_library().pe_set_fused_update(int(mode)))
 
 
 def pe_set_path(path: int) -> int:

@@ -25,6 +25,7 @@ __device__ unsigned int g_dev_status = 0;   // first device-side wait that gave 
 static std::atomic<int> g_path{PE_PATH_AUTO};
 static std::atomic<int> g_last_path{PE_PATH_AUTO};
 static std::atomic<long long> g_launches{0};
+static std::atomic<int> g_fused_mode{PE_FUSED_AUTO};
 // Both outputs: from this sequence length on the running sum of G_b lives in tensor memory beside a
 // 256-column accumulator (measured: wins or ties at T = 4096, loses 16 % at T = 2048, 17 % at T = 1024).
 constexpr int TC_MEAN_TMEM_MIN_T = 4096;
@@ -789,6 +790,33 @@ pe_status_t fused_impl(const TIn* X, const TIn* dY, int B, int T, int d_in, int 
   if (tc_ok && forced != PE_PATH_SIMT) {
     if constexpr (sizeof(TIn) == 2) {
       g_last_path.store(PE_PATH_TENSOR);
+      // The update inside the statistics kernel is a latency-bound tail during which that block's tensor cores
+      // idle (measured: about 25 us per tile and block, against a separate update kernel that streams at the
+      // HBM rate), so it saves memory (no [d_out, d_in] statistic buffers) rather than time.  PE_FUSED_AUTO
+      // therefore fuses only when the caller gave no buffers for the statistics; with buffers it runs the
+      // statistics kernel and the update kernel back to back.
+      const int mode = g_fused_mode.load();
+      const bool have_stats = out_b && (kind != OPT_ADAM || out_a);
+      if (mode == PE_FUSED_NEVER && !have_stats) return PE_ERR_NULL;
+      if (mode == PE_FUSED_NEVER || (mode == PE_FUSED_AUTO && have_stats)) {
+        rc = launch_tc(di, X, dY, B, T, d_in, d_out, kind == OPT_ADAM ? (int)PE_PHI_SQUARE : (int)PE_PHI_SIGN, 1,
+                       kind == OPT_ADAM ? out_a : nullptr, out_b, st);
+        if (rc != PE_OK) return rc;
+        const long long n = (long long)d_in * d_out;
+        const int grid = grid_for(n / 4 + 4, di->sm_count);
+        __nv_bfloat16* lp = static_cast<__nv_bfloat16*>(theta_lp);
+        if (kind == OPT_ADAM) {
+          switch (opt.variant) {
+            case ADAM_ORIGINAL: microadam_kernel<ADAM_ORIGINAL><<<grid, OPT_THREADS, 0, st>>>(theta, lp, m, v, out_a, out_b, n, opt.adam, di->status_ptr); break;
+            case ADAM_MICRO: microadam_kernel<ADAM_MICRO><<<grid, OPT_THREADS, 0, st>>>(theta, lp, m, v, out_a, out_b, n, opt.adam, di->status_ptr); break;
+            case ADAM_MICRO_VAR: microadam_kernel<ADAM_MICRO_VAR><<<grid, OPT_THREADS, 0, st>>>(theta, lp, m, v, out_a, out_b, n, opt.adam, di->status_ptr); break;
+            default: microadam_kernel<ADAM_MICRO_MSQ><<<grid, OPT_THREADS, 0, st>>>(theta, lp, m, v, out_a, out_b, n, opt.adam, di->status_ptr); break;
+          }
+        } else {
+          microsignsgd_kernel<<<grid, OPT_THREADS, 0, st>>>(theta, lp, m, out_b, n, opt.sign, di->status_ptr);
+        }
+        return check_launch();
+      }
       return launch_tc_fused(di, X, dY, B, T, d_in, d_out, kind, out_a, out_b, opt, static_cast<unsigned int*>(workspace),
                              workspace_bytes / sizeof(unsigned int), st);
     }
@@ -1155,6 +1183,11 @@ pe_status_t pe_set_wait_limit_cycles(long long cycles) {
   const long long v = cycles > 0 ? cycles : sm100::WAIT_CYCLE_LIMIT_DEFAULT;
   if (cudaMemcpyToSymbol(sm100::g_wait_cycle_limit, &v, sizeof v) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
   return PE_OK;
+}
+
+int pe_set_fused_update(int mode) {
+  if (mode < PE_FUSED_AUTO || mode > PE_FUSED_NEVER) return -1;
+  return g_fused_mode.exchange(mode);
 }
 
 int pe_set_path(int path) {

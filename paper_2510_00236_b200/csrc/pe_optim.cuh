@@ -61,7 +61,9 @@ template <int VARIANT>
 __global__ void __launch_bounds__(OPT_THREADS)
 microadam_kernel(float* __restrict__ theta, __nv_bfloat16* __restrict__ theta_lp, float* __restrict__ m,
                  float* __restrict__ v, const float* __restrict__ sum_g, const float* __restrict__ sum_g2,
-                 long long n, AdamParams p) {
+                 long long n, AdamParams p, const unsigned int* __restrict__ skip_if_set = nullptr) {
+  // when this step follows a statistics kernel in the same call: leave the parameters alone if that kernel gave up
+  if (skip_if_set && *reinterpret_cast<const volatile unsigned int*>(skip_if_set) != 0u) return;
   const long long n4 = n >> 2;
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x; k < n4; k += stride) {
@@ -109,7 +111,9 @@ __device__ __forceinline__ void sign_one(float& th, float& m, float ss, const Si
 
 __global__ void __launch_bounds__(OPT_THREADS)
 microsignsgd_kernel(float* __restrict__ theta, __nv_bfloat16* __restrict__ theta_lp, float* __restrict__ m,
-                    const float* __restrict__ sum_sign, long long n, SignParams p) {
+                    const float* __restrict__ sum_sign, long long n, SignParams p,
+                    const unsigned int* __restrict__ skip_if_set = nullptr) {
+  if (skip_if_set && *reinterpret_cast<const volatile unsigned int*>(skip_if_set) != 0u) return;
   const long long n4 = n >> 2;
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x; k < n4; k += stride) {

@@ -234,56 +234,74 @@ enum : int { MEAN_NONE = 0, MEAN_REGS = 1, MEAN_TMEM = 2, MEAN_REGS_SIGN = 3, ME
 constexpr int TC_SIGN_COUNT_MAX = 32767;   // examples per block in MEAN_REGS_SIGN mode: 2 * count must fit 16 bits
 
 // gridDim = (2 * pairs_m * tiles_n, 1, nsplit); blockIdx.x = 2 * (pair index in the tile order) + rank in pair.
-// The fused parameter update of one epilogue warp's 32-row x (PANELS * 32)-column piece of the tile.  Here a
-// lane is a COLUMN (global accesses of a warp are 128 contiguous bytes of one row), whereas the running
-// sums live one ROW per lane: the sums therefore come either from the warp's staged panels in shared
-// memory (the 128-byte-swizzled 32 x 32 panels the write-out also hands to TMA; chunk k of row r sits at
-// chunk position k ^ (r & 7)) or, when the batch was split and this block added the last partial sum,
-// from the outputs in global memory (read past L1).  16 rows are in flight per lane at a time.
+// The fused parameter update of one epilogue warp's 32-row x (PANELS * 32)-column piece of the tile.  The piece
+// is walked as float4 groups, a warp instruction covering 128 float4 in row-major order (global accesses of a
+// warp are whole 16-byte groups of one or two rows), whereas the running sums live one ROW per lane: the sums
+// therefore come either from the warp's staged panels in shared memory (the 128-byte-swizzled 32 x 32 panels the
+// write-out also hands to TMA; chunk k of row r sits at chunk position k ^ (r & 7)) or, when the batch was
+// split and this block added the last partial sum, from the outputs in global memory (read past L1).  Eight
+// float4 per array and lane are in flight at a time (about 100 KiB per SM): the step is a latency-bound tail
+// during which the block's tensor cores idle, so what counts is the number of memory round trips.
 template <int OPT, int PANELS>
 __device__ __forceinline__ void fused_update_piece(const FusedOpt& o, const TcParams& p, int row0, int col0, int lane,
                                                    const uint8_t* stat_panels, const uint8_t* mean_panels) {
-  for (int c = 0; c < PANELS; ++c) {
-    if (col0 + c * 32 >= p.d_in) break;
-    const int col = col0 + c * 32 + lane;
-    const bool col_ok = col < p.d_in;
+  constexpr int C4 = PANELS * 8;             // float4 groups per row of the piece
+  constexpr int ITERS = C4;                  // 32 rows x C4 groups / 32 lanes
+  constexpr int BATCH = 8;
+  static_assert(ITERS % BATCH == 0, "whole batches");
+  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
+  for (int it0 = 0; it0 < ITERS; it0 += BATCH) {
+    float4 th[BATCH], mm[BATCH], vv[BATCH], s1[BATCH], s2[BATCH];
 #pragma unroll
-    for (int rb = 0; rb < 32; rb += 16) {
-      float th[16], mm[16], vv[16], s1[16], s2[16];
-#pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const int r = rb + i;
-        const bool in = col_ok && row0 + r < p.d_out;
-        const long long idx = (long long)(row0 + r) * p.d_in + col;
-        th[i] = in ? o.theta[idx] : 0.f;
-        mm[i] = in ? o.m[idx] : 0.f;
-        vv[i] = (OPT == OPT_ADAM && in) ? o.v[idx] : 0.f;
-        float st, mn = 0.f;
-        if (stat_panels) {
-          const int off = c * 4096 + r * 128 + (((lane >> 2) ^ (r & 7)) << 4) + (lane & 3) * 4;
-          st = *reinterpret_cast<const float*>(stat_panels + off);
-          if (OPT == OPT_ADAM) mn = *reinterpret_cast<const float*>(mean_panels + off);
-        } else {
-          st = in ? __ldcg(p.out_stat + idx) : 0.f;
-          if (OPT == OPT_ADAM) mn = in ? __ldcg(p.out_mean + idx) : 0.f;
-        }
-        s1[i] = (OPT == OPT_ADAM) ? mn : st;
-        s2[i] = st;
+    for (int i = 0; i < BATCH; ++i) {
+      const int k = (it0 + i) * 32 + lane;
+      const int r = k / C4, c4 = k - r * C4;
+      const int row = row0 + r, col = col0 + 4 * c4;
+      const bool in = row < p.d_out && col < p.d_in;           // d_in is a multiple of 8: a group is all in or all out
+      const long long idx = (long long)row * p.d_in + col;
+      th[i] = in ? *reinterpret_cast<const float4*>(o.theta + idx) : zero4;
+      mm[i] = in ? *reinterpret_cast<const float4*>(o.m + idx) : zero4;
+      vv[i] = (OPT == OPT_ADAM && in) ? *reinterpret_cast<const float4*>(o.v + idx) : zero4;
+      float4 st, mn = zero4;
+      if (stat_panels) {
+        const int off = (c4 >> 3) * 4096 + r * 128 + (((c4 & 7) ^ (r & 7)) << 4);
+        st = *reinterpret_cast<const float4*>(stat_panels + off);
+        if (OPT == OPT_ADAM) mn = *reinterpret_cast<const float4*>(mean_panels + off);
+      } else {
+        st = in ? __ldcg(reinterpret_cast<const float4*>(p.out_stat + idx)) : zero4;
+        if (OPT == OPT_ADAM) mn = in ? __ldcg(reinterpret_cast<const float4*>(p.out_mean + idx)) : zero4;
       }
+      s1[i] = (OPT == OPT_ADAM) ? mn : st;
+      s2[i] = st;
+    }
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const int r = rb + i;
-        if (col_ok && row0 + r < p.d_out) {
-          const long long idx = (long long)(row0 + r) * p.d_in + col;
-          if constexpr (OPT == OPT_ADAM) {
-            adam_one_rt(o.variant, th[i], mm[i], vv[i], s1[i], s2[i], o.adam);
-            o.v[idx] = vv[i];
-          } else {
-            sign_one(th[i], mm[i], s1[i], o.sign);
-          }
-          o.theta[idx] = th[i];
-          o.m[idx] = mm[i];
-          if (o.theta_lp) o.theta_lp[idx] = __float2bfloat16_rn(th[i]);
+    for (int i = 0; i < BATCH; ++i) {
+      const int k = (it0 + i) * 32 + lane;
+      const int r = k / C4, c4 = k - r * C4;
+      const int row = row0 + r, col = col0 + 4 * c4;
+      if (row < p.d_out && col < p.d_in) {
+        const long long idx = (long long)row * p.d_in + col;
+        if constexpr (OPT == OPT_ADAM) {
+          adam_one_rt(o.variant, th[i].x, mm[i].x, vv[i].x, s1[i].x, s2[i].x, o.adam);
+          adam_one_rt(o.variant, th[i].y, mm[i].y, vv[i].y, s1[i].y, s2[i].y, o.adam);
+          adam_one_rt(o.variant, th[i].z, mm[i].z, vv[i].z, s1[i].z, s2[i].z, o.adam);
+          adam_one_rt(o.variant, th[i].w, mm[i].w, vv[i].w, s1[i].w, s2[i].w, o.adam);
+          *reinterpret_cast<float4*>(o.v + idx) = vv[i];
+        } else {
+          sign_one(th[i].x, mm[i].x, s1[i].x, o.sign);
+          sign_one(th[i].y, mm[i].y, s1[i].y, o.sign);
+          sign_one(th[i].z, mm[i].z, s1[i].z, o.sign);
+          sign_one(th[i].w, mm[i].w, s1[i].w, o.sign);
+        }
+        *reinterpret_cast<float4*>(o.theta + idx) = th[i];
+        *reinterpret_cast<float4*>(o.m + idx) = mm[i];
+        if (o.theta_lp) {
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(th[i].x, th[i].y), hi = __floats2bfloat162_rn(th[i].z, th[i].w);
+          uint2 pk;
+          pk.x = *reinterpret_cast<const unsigned int*>(&lo);
+          pk.y = *reinterpret_cast<const unsigned int*>(&hi);
+          *reinterpret_cast<uint2*>(o.theta_lp + idx) = pk;
         }
       }
     }
