@@ -353,6 +353,11 @@ def run_sweep(args):
             t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
             t_hbm = (bytes_in + 8.0 * d * d) / (peaks["hbm_gbs"] * 1e9)
             t_alu = 2.0 * B * d * d / (148 * 128 * 1.965e9)
+            # sign costs about 5 fp32 operations per entry instead of 2; and short sequences are bound by how many
+            # per-example tiles tensor memory holds at once: an accumulator entry is occupied for one hand-off chain
+            # (about 1.4 us: load landed -> MMA -> commit -> epilogue read -> release), 65536 entries per SM
+            t_alu_sign = 5.0 * B * d * d / (148 * 128 * 1.965e9)
+            t_occupancy = B * float(d) * d / (148 * 65536) * 1.4e-6
             print(json.dumps({
                 "sweep_point": {"B": B, "T": T, "d_in": d, "d_out": d}, "input_sets": nsets,
                 "both_outputs_us": med_b * 1e3, "both_outputs_tflops": flops / med_b / 1e9,
@@ -361,7 +366,8 @@ def run_sweep(args):
                 "sign_only_us": med_n * 1e3, "all_three_us": med_a * 1e3, "overhead_all_three_vs_gemm": med_a / med_g,
                 "cublas_gemm_us": med_g * 1e3, "cublas_gemm_tflops": flops / med_g / 1e9,
                 "overhead_both_vs_gemm": med_b / med_g, "overhead_stat_vs_gemm": med_s / med_g,
-                "bound_tensor_us": t_tensor * 1e6, "bound_hbm_us": t_hbm * 1e6, "bound_alu_us": t_alu * 1e6, "peak_source": peaks["source"]}), flush=True)
+                "bound_tensor_us": t_tensor * 1e6, "bound_hbm_us": t_hbm * 1e6, "bound_alu_us": t_alu * 1e6, "bound_alu_sign_us": t_alu_sign * 1e6,
+                "bound_tmem_occupancy_us": t_occupancy * 1e6, "peak_source": peaks["source"]}), flush=True)
             del sets, mean, stat, sgn
             torch.cuda.empty_cache()
 
