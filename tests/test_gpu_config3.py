@@ -116,6 +116,13 @@ def test_config3_every_linear_layer_and_microadam_step():
         e_upd = rel_frob(pick(theta) - pick(theta0), th_ref - pick(theta0).astype(np.float64))
         assert e_upd <= FROB_TOL, (name, e_upd)
         assert rel_frob(pick(v), v_ref) <= FROB_TOL and rel_frob(pick(m), m_ref) <= FROB_TOL
-        worst = max(worst, e_mean, e_sq, e_upd)
+        # the same step with the update inside the statistics kernel and no statistic buffers at all
+        theta_f, m_f, v_f = theta0.clone(), torch.zeros_like(theta), torch.zeros_like(theta)
+        pe.pe_linear_microadam_step(X, dY, theta_f, m_f, v_f, **kw)
+        torch.cuda.synchronize()
+        e_fused = rel_frob(pick(theta_f) - pick(theta0), th_ref - pick(theta0).astype(np.float64))
+        assert e_fused <= FROB_TOL, (name, e_fused)
+        assert rel_frob(pick(v_f), v_ref) <= FROB_TOL and rel_frob(pick(m_f), m_ref) <= FROB_TOL
+        worst = max(worst, e_mean, e_sq, e_upd, e_fused)
     assert pe.pe_get_async_status(DEV) == (0, 0)
     print("config3: 25 linear layers, worst relative Frobenius error", worst)
