@@ -318,9 +318,11 @@ pe_status_t microsignsgd_step(float* theta, void* theta_lp, float* m, const floa
  * they were (the two-kernel sequence skips its update kernel while the device status word is set, i.e.
  * until pe_get_async_status has read and cleared it).
  * What the fusion buys is MEMORY, not time: with out_mean = out_stat = NULL no [d_out, d_in] statistic
- * buffer exists anywhere (2 x 4 bytes per parameter saved).  In time the update inside the statistics
- * kernel is a latency-bound tail of every tile during which that block's tensor cores idle (about 25 us
- * per tile and block, measured), while a separate update kernel streams at the HBM rate.  By default
+ * buffer exists anywhere (2 x 4 bytes per parameter saved).  In time there is little to gain (the update
+ * moves 34 bytes per parameter whoever performs it; fusing saves the 8 bytes of re-reading the sums) and
+ * something to lose: the blocks of a wave finish their tiles together, so the update's traffic reaches
+ * memory in bursts during which the tensor cores idle (about 25 us per wave, measured), while a separate
+ * update kernel streams at the HBM rate after the statistics kernel.  By default
  * (PE_FUSED_AUTO) the call therefore fuses only when it was given no statistic buffers and otherwise
  * runs the statistics kernel and the update kernel back to back on `stream`; pe_set_fused_update
  * overrides that choice.

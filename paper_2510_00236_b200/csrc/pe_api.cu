@@ -790,9 +790,10 @@ pe_status_t fused_impl(const TIn* X, const TIn* dY, int B, int T, int d_in, int 
   if (tc_ok && forced != PE_PATH_SIMT) {
     if constexpr (sizeof(TIn) == 2) {
       g_last_path.store(PE_PATH_TENSOR);
-      // The update inside the statistics kernel is a latency-bound tail during which that block's tensor cores
-      // idle (measured: about 25 us per tile and block, against a separate update kernel that streams at the
-      // HBM rate), so it saves memory (no [d_out, d_in] statistic buffers) rather than time.  PE_FUSED_AUTO
+      // The update inside the statistics kernel cannot overlap the contraction: the blocks of a wave finish
+      // together, so a wave's update traffic reaches memory at once while the tensor cores idle (measured: about
+      // 25 us per wave, against a separate update kernel that streams at the HBM rate).  Fusing saves memory (no
+      // [d_out, d_in] statistic buffers) rather than time.  PE_FUSED_AUTO
       // therefore fuses only when the caller gave no buffers for the statistics; with buffers it runs the
       // statistics kernel and the update kernel back to back.
       const int mode = g_fused_mode.load();
