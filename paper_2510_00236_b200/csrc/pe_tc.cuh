@@ -1,18 +1,19 @@
 // Tensor-core kernel for the sequence-level per-example statistics (Section 2.3; Eq. (2)).
 //
 // Work unit: a CTA PAIR (a cluster of two thread blocks on two SMs) owns a 256 x NT tile of the
-// [d_out, d_in] output (NT = 128 or 256) and a contiguous slice of the batch.  For every example of
+// [d_out, d_in] output (NT = 128, 192 or 256) and a contiguous slice of the batch.  For every example of
 // the slice the tile of G_b = dY_b^T X_b is formed by pair-wide tcgen05 MMAs (cta_group::2,
 // M = 256: each block supplies 128 rows of dY_b^T and half of the NT rows of X_b^T from its own
 // shared memory and receives its 128 accumulator rows in its own tensor memory), read back by the
 // epilogue warps, passed through phi and added to register-resident running sums (sum_b phi(G_b)
 // and, when asked for, sum_b G_b).  The per-example tile never leaves the SM.  Pairing cuts the
 // operand bytes each SM pulls from L2 per flop; an SM sustains about 70 B/clk from L2, a lone
-// 128 x 128 tile would need 128 B/clk at full tensor rate, a 256 x 128 pair 96, a 256 x 256 pair 64.
+// 128 x 128 tile would need 128 B/clk at full tensor rate, a 256 x 128 pair 96, a 256 x 192 pair 75, a
+// 256 x 256 pair 64.
 //
 //   MEAN_REGS, NT = 128: two running sums per thread (64 + 64 registers)         -- both outputs, short sequences
 //   MEAN_REGS, NT = 192: two running sums per thread (96 + 96 registers; the control
-//                        warps shrink to 48 registers so that the epilogue warps can take 232) -- both outputs
+//                        warps shrink to 40 registers so that the epilogue warps can take 232) -- both outputs
 //   MEAN_REGS_SIGN, NT = 128: the same plus sum_b sign(G_b), counted in 16-bit halves
 //                        of 32 more registers                                      -- mean, square and sign in one pass
 //   MEAN_HYBRID_SIGN, NT = 192: mean, square and sign on the wider tile: sum_b G_b^2 (96 registers), the sign
@@ -24,6 +25,8 @@
 //   MEAN_NORMS, NT = 256: no running sums; every example's sum of squares over the
 //                        tile is reduced and added to out_norms[b]                 -- per-example squared norms
 //   PHI = 0,   NT = 256: no per-example reset (accumulate in tensor memory)        -- plain contraction over all rows
+// Further template arguments: RAGGED (packed batches with per-example token ranges), OPT (the parameter
+// update applied by the block that completes a tile's sums), F8 (e4m3 operands for the plain contraction).
 //
 // Warp roles per block (12 warps): 0 = TMA producer of the dY boxes, 2 = TMEM allocator, then TMA
 // producer of the X boxes, 1 and 3 = MMA issuers (leader block only), 4..11 = epilogue (warp w reads
@@ -45,7 +48,7 @@
 // "MN-major".  A TMA box is 128 bytes of features (64 bf16) x BK tokens; with the 128-byte swizzle that is
 // exactly the canonical MN-major layout of the MMA: 8-token x 64-feature atoms of 1 KiB, the next
 // 8 tokens 1 KiB further (stride byte offset), the next 64 features one box further (leading byte
-// offset).
+// offset).  (X at NT = 192: 64 bytes of features per box row and the 64-byte swizzle, 512-byte atoms.)
 #pragma once
 #include "pe_optim.cuh"
 #include "pe_sm100.cuh"
