@@ -197,15 +197,19 @@ static pe_status_t zero_for_split(DeviceInfo* di, float* a, float* b, size_t n, 
 
 // Launches `kernel`; as a programmatic dependent of the zeroing kernel when the batch is split.
 template <typename Kernel, typename... Args>
-static pe_status_t launch_pair_kernel(Kernel kernel, dim3 grid, int smem, cudaStream_t st, bool after_zeroing, Args... args) {
+static pe_status_t launch_pair_kernel_t(Kernel kernel, dim3 grid, int threads, int smem, cudaStream_t st, bool after_zeroing, Args... args) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid; cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = st;
+  cfg.gridDim = grid; cfg.blockDim = dim3(threads); cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = st;
   cudaLaunchAttribute attr;
   attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr; cfg.numAttrs = after_zeroing ? 1 : 0;
   if (cudaLaunchKernelEx(&cfg, kernel, args...) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
   return check_launch();
+}
+template <typename Kernel, typename... Args>
+static pe_status_t launch_pair_kernel(Kernel kernel, dim3 grid, int smem, cudaStream_t st, bool after_zeroing, Args... args) {
+  return launch_pair_kernel_t(kernel, grid, TC_THREADS, smem, st, after_zeroing, args...);
 }
 
 // mxt, myt: the maps of the zero-padded tail groups of a packed batch (RAGGED); any valid map otherwise.
@@ -605,7 +609,7 @@ static pe_status_t launch_tok(DeviceInfo* di, const void* X, const void* dY, lon
   TokParams p;
   p.rows = rows; p.d_in = d_in; p.d_out = d_out; p.pairs_m = pairs_m; p.tiles_n = tiles_n;
   p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND; p.nsplit = ns; p.dev_status = di->status_ptr;
-  return launch_pair_kernel(tok_sqstats_kernel, dim3(2 * pairs_m * tiles_n, 1, ns), TOK_SMEM_BYTES, st, ns > 1, mx, my, mo, p);
+  return launch_pair_kernel_t(tok_sqstats_kernel, dim3(2 * pairs_m * tiles_n, 1, ns), TOK_THREADS, TOK_SMEM_BYTES, st, ns > 1, mx, my, mo, p);
 }
 
 }  // namespace pe

@@ -18,12 +18,14 @@
 // and 4 "cooked" stages of 32 KiB (fp32 holding tf32 values: eight 32-feature boxes; 128-byte swizzle
 // with 32-byte chunks, the only MN-major form of the tf32 MMA).
 //
-// Warps: 0 = TMA producer of the dY boxes (also posts the stage's byte count), 2 = TMEM allocator,
-// then TMA producer of the X boxes, 1 = MMA issuer (leader block only), 4..11 = converters, then
-// write-out.  Barriers: raw_full[s] / raw_empty[s] are local to each block (its own TMA, its own
-// converters); cooked_full[c] lives in the leader and collects the converter warps of both blocks
-// (four per block and stage: the eight warps work as two groups on alternate stages);
-// cooked_empty[c] and acc_full are signalled in both blocks by one multicast commit.
+// Warps (20 per block): 0 = TMA producer of the dY boxes (also posts the stage's byte count), 2 = TMEM
+// allocator, then TMA producer of the X boxes, 1 = MMA issuer (leader block only), 4..19 = converters
+// (sixteen warps: the conversion is a stream of dependent shared-memory round trips, and eight warps
+// only reached 1.4 instructions per clock of the SM's 4), of which 4..11 then write the result out.
+// Barriers: raw_full[s] / raw_empty[s] are local to each block (its own TMA, its own converters);
+// cooked_full[c] lives in the leader and collects the converter warps of both blocks (four per block
+// and stage: the sixteen warps work as four groups, group g on the stages n = g mod 4, i.e. always
+// on ring slot g); cooked_empty[c] and acc_full are signalled in both blocks by one multicast commit.
 #pragma once
 #include "pe_tc.cuh"
 
@@ -39,6 +41,10 @@ constexpr int TOK_RAW_STAGES = 4, TOK_COOKED_STAGES = 4;
 constexpr int TOK_RING_BYTES = TOK_RAW_STAGES * TOK_RAW_STAGE + TOK_COOKED_STAGES * TOK_COOKED_STAGE;   // 192 KiB
 constexpr int TOK_SMEM_BYTES = TOK_RING_BYTES + TC_BAR_BYTES + 1024;
 constexpr int TOK_MMA_K = 8;                      // rows per tf32 MMA
+constexpr int TOK_CONV_WARPS = 16;                // converter warps per block, in groups of four
+constexpr int TOK_CONV_GROUPS = TOK_CONV_WARPS / 4;
+constexpr int TOK_THREADS = 128 + 32 * TOK_CONV_WARPS;          // 640: 96 registers per thread at one block per SM
+static_assert(TOK_CONV_GROUPS == TOK_RAW_STAGES, "converter group g owns ring slot g");
 enum : int { TOK_WAIT_RAW_EMPTY = 11, TOK_WAIT_RAW_FULL = 12, TOK_WAIT_COOKED_EMPTY = 13, TOK_WAIT_COOKED_FULL = 14, TOK_WAIT_ACC = 15 };
 
 struct TokParams {
@@ -70,7 +76,7 @@ __device__ __forceinline__ uint64_t tok_square_tf32_pair(uint32_t two_bf16) {
 // gridDim = (2 * pairs_m * tiles_n, 1, nsplit); blockIdx.x = 2 * (pair index in the tile order) + rank in pair.
 // tmap_x / tmap_dy: [rows, d] bf16 viewed as (d, rows), box 64 x 32, 128-byte swizzle.
 // tmap_out: [d_out, d_in] fp32 viewed as (d_in, d_out), box 32 x 32, 128-byte swizzle.
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TOK_THREADS, 1)
 tok_sqstats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
                    const __grid_constant__ CUtensorMap tmap_out, TokParams p) {
   using namespace sm100;
@@ -117,7 +123,6 @@ tok_sqstats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp < 4) {
-    setmaxnreg_dec<TC_REGS_CONTROL>();
     if (warp == 0 || warp == 2) {
       // ---------------------------------------------------------- TMA producers (each block for itself)
       if (lane == 0) {
@@ -164,15 +169,14 @@ tok_sqstats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     }
   } else {
     // ------------------------------------------------------------ converters, then write-out (both blocks)
-    setmaxnreg_inc<TC_REGS_EPILOGUE>();
-    const int w = warp - 4;                 // 0..7
+    // (no setmaxnreg here: 640 threads x 96 registers is all a converter needs)
+    const int w = warp - 4;                 // 0..15
     bool ok = true;
     {
-      // The eight warps work as two groups of four on alternate stages (group = parity of the stage,
-      // hence of the ring slot), so that one group's shared-memory round trips and barrier hand-offs
-      // overlap the other's arithmetic.
+      // The sixteen warps work as four groups of four, group g on the stages n = g, g + 4, ... (ring slot g),
+      // so that the groups' shared-memory round trips and barrier hand-offs overlap one another's arithmetic.
       const int grp = w >> 2, wl = w & 3;
-      for (long long n = grp; n < c_end - c_begin; n += 2) {
+      for (long long n = grp; n < c_end - c_begin; n += TOK_CONV_GROUPS) {
         const int s = (int)(n % TOK_RAW_STAGES);          // raw and cooked rings advance together (same depth)
         const uint32_t ph = (uint32_t)(n / TOK_RAW_STAGES) & 1u;
         // every lane polls, the warp acts on one answer (what follows contains warp-wide instructions)
@@ -216,9 +220,9 @@ tok_sqstats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     }
     static_assert(TOK_RAW_STAGES == TOK_COOKED_STAGES && TOK_RAW_STAGES % 2 == 0, "the two rings advance together; each slot belongs to one converter group");
     ok = __all_sync(0xffffffffu, ok);
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(acc_full, 0, abort_flag, p.dev_status, TOK_WAIT_ACC));
+    if (ok && w < 8) ok = __all_sync(0xffffffffu, mbar_wait_bounded(acc_full, 0, abort_flag, p.dev_status, TOK_WAIT_ACC));
     ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
+    if (ok && w < 8) {
       // Write-out as in the statistics kernel: 32 rows x 128 columns per warp, staged in the idle ring
       // as four 128-byte-swizzled 4 KiB panels, stored (or added, with a split row range) by TMA.
       tc_fence_after();
