@@ -75,6 +75,51 @@ def test_workspace_size_formula(lib):
         pe.pe_set_path(prev)
 
 
+def test_other_workspace_sizes_and_mode_switches(lib):
+    prev = pe.pe_set_path(pe.PATH_AUTO)
+    try:
+        # packed batches: the zero-padded last partial 16-token group of every sequence, X's then dY's, bf16
+        assert pe.pe_linear_stats_ragged_workspace_bytes(10, 64, 128) == 10 * 16 * 64 * 2 + 10 * 16 * 128 * 2
+        assert pe.pe_linear_stats_ragged_workspace_bytes(3, 8, 8) == 768 + 768          # 3 * 16 * 8 * 2 = 768, already a multiple of 256
+        assert pe.pe_linear_stats_ragged_workspace_bytes(3, 7, 8) == 0                  # SIMT shape: no workspace
+        assert pe.pe_linear_stats_ragged_workspace_bytes(0, 8, 8) == 0
+        # fused update: one counter per thread block of the widest grid (256 x 128 tiles, two blocks per pair)
+        assert pe.pe_linear_fused_workspace_bytes(2048, 8192) == 2 * 32 * 16 * 4
+        assert pe.pe_linear_fused_workspace_bytes(8, 8) == 256
+        # fp8 staging: one byte per element when both widths are multiples of 16, the half layout otherwise
+        assert pe.pe_token_sqstats_fp8_workspace_bytes(64, 256, 512, 2048) == (512 + 2048) * 4 + 64 * 256 * (512 + 2048)
+        assert pe.pe_token_sqstats_fp8_workspace_bytes(64, 256, 520, 2048) == pe.pe_token_sqstats_staged_workspace_bytes(64, 256, 520, 2048)
+    finally:
+        pe.pe_set_path(prev)
+    prev = pe.pe_set_fused_update(pe.FUSED_ALWAYS)
+    assert pe.pe_set_fused_update(prev) == pe.FUSED_ALWAYS
+    assert pe.pe_set_fused_update(9) == -1
+    assert pe.pe_set_path(pe.PATH_TENSOR_WIDE) == pe.PATH_AUTO and pe.pe_set_path(pe.PATH_AUTO) == pe.PATH_TENSOR_WIDE
+
+
+def test_new_entry_points_validate_on_the_host(lib):
+    buf = ctypes.create_string_buffer(8192)
+    p16 = (ctypes.addressof(buf) + 255) & ~255
+    vp, ll, f = ctypes.c_void_p, ctypes.c_longlong, ctypes.c_float
+    # packed batches: offsets required, sizes checked, outputs required
+    assert lib.pe_linear_stats_ragged(p16, p16, None, 2, ll(32), 8, 8, 1, p16, p16, p16, 4096, None) == 1
+    assert lib.pe_linear_stats_ragged(p16, p16, p16, -1, ll(32), 8, 8, 1, p16, p16, p16, 4096, None) == 2
+    assert lib.pe_linear_stats_ragged(p16, p16, p16, 2, ll(1 << 31), 8, 8, 1, p16, p16, p16, 4096, None) == 2
+    assert lib.pe_linear_stats_ragged(p16, p16, p16, 2, ll(32), 8, 8, 1, None, None, p16, 4096, None) == 1
+    assert lib.pe_linear_stats_ragged(p16, p16, p16, 2, ll(32), 8, 8, 9, p16, p16, p16, 4096, None) == 5
+    # clipped sum: negative or NaN threshold, missing norms buffer
+    assert lib.pe_linear_clipped_sum(p16, p16, 2, 4, 8, 8, f(-1.0), p16, 0, p16, None) == 2
+    assert lib.pe_linear_clipped_sum(p16, p16, 2, 4, 8, 8, f(float("nan")), p16, 0, p16, None) == 2
+    assert lib.pe_linear_clipped_sum(p16, p16, 2, 4, 8, 8, f(1.0), None, 0, p16, None) == 1
+    # statistics + update: parameters required, step and variant checked, a variance needs two examples
+    adam = (1, f(1.0), f(1e-3), f(0.9), f(0.99), f(1e-8), 0, f(0.0))
+    assert lib.pe_linear_microadam_step(p16, p16, 2, 4, 8, 8, None, None, p16, p16, None, None, *adam, 1, None, 0, None) == 1
+    assert lib.pe_linear_microadam_step(p16, p16, 2, 4, 8, 8, p16, None, p16, p16, None, None, *adam, 0, None, 0, None) == 2
+    assert lib.pe_linear_microadam_step(p16, p16, 2, 4, 8, 8, p16, None, p16, p16, None, None, 7, *adam[1:], 1, None, 0, None) == 5
+    assert lib.pe_linear_microadam_step(p16, p16, 1, 4, 8, 8, p16, None, p16, p16, None, None, 2, *adam[1:], 1, None, 0, None) == 2
+    assert lib.pe_linear_microsignsgd_step(p16, p16, 0, 4, 8, 8, p16, None, p16, None, f(1e-3), f(0.9), f(0.0), None, 0, None) == 2
+
+
 def test_cpu_tensors_are_rejected_loudly():
     import torch
     X = torch.zeros(1, 2, 8, dtype=torch.bfloat16)
