@@ -355,9 +355,9 @@ def run_sweep(args):
             t_alu = 2.0 * B * d * d / (148 * 128 * 1.965e9)
             # sign costs about 5 fp32 operations per entry instead of 2; and short sequences are bound by how many
             # per-example tiles tensor memory holds at once: an accumulator entry is occupied for one hand-off chain
-            # (about 1.4 us: load landed -> MMA -> commit -> epilogue read -> release), 65536 entries per SM
+            # (about 1.25 us, measured: stage full seen -> MMAs and commits issued -> epilogue read -> release), 65536 entries per SM
             t_alu_sign = 5.0 * B * d * d / (148 * 128 * 1.965e9)
-            t_occupancy = B * float(d) * d / (148 * 65536) * 1.4e-6
+            t_occupancy = B * float(d) * d / (148 * 65536) * 1.25e-6
             print(json.dumps({
                 "sweep_point": {"B": B, "T": T, "d_in": d, "d_out": d}, "input_sets": nsets,
                 "both_outputs_us": med_b * 1e3, "both_outputs_tflops": flops / med_b / 1e9,
