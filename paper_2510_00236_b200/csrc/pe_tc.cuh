@@ -189,6 +189,31 @@ __device__ __forceinline__ void tc_tile_of_block(const TcParams& p, uint32_t ran
   tile_m = 2 * (band * p.band + (r - tile_n * rows)) + (int)rank;
 }
 
+// (sign(g) + 1) / 2, i.e. 0, 0.5 or 1, with sign(+-0) = 0, in two instructions: g is scaled by 2^64 (exact, or to
+// infinity; the callers do it two columns at a time), then 2^127 * g + 0.5 is rounded and saturated to [0, 1].  The
+// smallest nonzero |g|, the denormal 2^-149, arrives as 2^42, so every nonzero g saturates and zero alone gives 0.5.
+// Summed over nb examples this is (sum_b sign(G_b) + nb) / 2, exact in fp32 (multiples of 0.5 below 2^23).
+constexpr float SIGN_PRESCALE = 18446744073709551616.f;     // 2^64
+__device__ __forceinline__ float sign_half_of_scaled(float g_scaled) {
+  float u;
+  asm("fma.rn.sat.f32 %0, %1, 0f7F000000, 0f3F000000;" : "=f"(u) : "f"(g_scaled));
+  return u;
+}
+__device__ __forceinline__ float sign_half(float g) { return sign_half_of_scaled(g * SIGN_PRESCALE); }
+// The same for two columns: {u(lo), u(hi)} packed for the two-wide fp32 instructions.
+__device__ __forceinline__ uint64_t sign_half2(uint64_t g2) {
+  float a0, a1;
+  sm100::f32x2_unpack(sm100::f32x2_mul(g2, sm100::f32x2_pack(SIGN_PRESCALE, SIGN_PRESCALE)), a0, a1);
+  return sm100::f32x2_pack(sign_half_of_scaled(a0), sign_half_of_scaled(a1));
+}
+// Two columns' sign(g) + 1 in {0, 1, 2} as the low and high 16 bits of one word: 2 u + 1.5 * 2^23 has the integer in
+// the low bits of its pattern, and one byte permute packs the two low halves.
+__device__ __forceinline__ uint32_t sign_plus_one_packed(uint64_t g2) {
+  float t0, t1;
+  sm100::f32x2_unpack(sm100::f32x2_fma(sign_half2(g2), sm100::f32x2_pack(2.f, 2.f), sm100::f32x2_pack(12582912.f, 12582912.f)), t0, t1);
+  return __byte_perm(__float_as_uint(t0), __float_as_uint(t1), 0x5410);
+}
+
 template <int PHI>
 __device__ __forceinline__ float phi_apply(float g) {
   if (PHI == 1) return g * g;
@@ -582,7 +607,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const float g = __uint_as_float(r[j]);
-            acc_stat[c * 16 + j] += phi_apply<PHI>(g);
+            acc_stat[c * 16 + j] += (PHI == 2) ? sign_half(g) : phi_apply<PHI>(g);
             if (a != 0) r[j] = __float_as_uint(g + __uint_as_float(m[j]));
           }
           tmem_st_32x32b_x16(maddr + c * 16, r);
@@ -607,9 +632,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             const uint64_t g2 = f32x2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
             const uint64_t s2 = f32x2_fma(g2, g2, f32x2_pack(acc_stat[c * 16 + j], acc_stat[c * 16 + j + 1]));
             f32x2_unpack(s2, acc_stat[c * 16 + j], acc_stat[c * 16 + j + 1]);
-            const float t0 = phi_apply<2>(__uint_as_float(r[j])) + 12582913.f;
-            const float t1 = phi_apply<2>(__uint_as_float(r[j + 1])) + 12582913.f;
-            acc_cnt[(c * 16 + j) >> 1] += __byte_perm(__float_as_uint(t0), __float_as_uint(t1), 0x5410);
+            acc_cnt[(c * 16 + j) >> 1] += sign_plus_one_packed(g2);
             if (in_tmem) {
               if (a != 0) {
                 const uint64_t m2 = f32x2_add(f32x2_pack(__uint_as_float(m[j]), __uint_as_float(m[j + 1])), g2);
@@ -663,11 +686,16 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         // phi and the running sums for one read of CH columns (chunk c of this thread's COLS columns)
         auto fold = [&](const uint32_t (&r)[CH], int c) {
           if constexpr (PHI == 2) {
+            // the running sum holds sum_b (sign(G_b) + 1) / 2 until the write-out turns it into sum_b sign(G_b)
 #pragma unroll
-            for (int j = 0; j < CH; ++j) {
-              const float g = __uint_as_float(r[j]);
-              if (KEEP_MEAN) acc_mean[c * CH + j] += g;
-              acc_stat[c * CH + j] += phi_apply<PHI>(g);
+            for (int j = 0; j < CH; j += 2) {
+              const uint64_t g2 = f32x2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+              if (KEEP_MEAN) {
+                const uint64_t m2 = f32x2_add(f32x2_pack(acc_mean[c * CH + j], acc_mean[c * CH + j + 1]), g2);
+                f32x2_unpack(m2, acc_mean[c * CH + j], acc_mean[c * CH + j + 1]);
+              }
+              const uint64_t s2 = f32x2_add(f32x2_pack(acc_stat[c * CH + j], acc_stat[c * CH + j + 1]), sign_half2(g2));
+              f32x2_unpack(s2, acc_stat[c * CH + j], acc_stat[c * CH + j + 1]);
             }
           } else {
             // two columns per instruction: packed fp32 add for sum_b G_b, packed fma for sum_b G_b^2
@@ -683,11 +711,7 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 f32x2_unpack(s2, acc_stat[c * CH + j], acc_stat[c * CH + j + 1]);
               }
               if (TRIPLE) {
-                // sign(g) as a float, plus 2^23 * 1.5 + 1: the low 16 bits of the sum's bit pattern are
-                // sign(g) + 1 in {0, 1, 2}; one byte permute packs the two columns' low halves
-                const float t0 = phi_apply<2>(__uint_as_float(r[j])) + 12582913.f;
-                const float t1 = phi_apply<2>(__uint_as_float(r[j + 1])) + 12582913.f;
-                acc_cnt[(c * CH + j) >> 1] += __byte_perm(__float_as_uint(t0), __float_as_uint(t1), 0x5410);
+                acc_cnt[(c * CH + j) >> 1] += sign_plus_one_packed(g2);
               }
             }
           }
@@ -743,6 +767,12 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     // whatever lies outside the matrix.  The tensor-memory loads are warp-wide instructions: the
     // condition around them is made uniform over the warp.
     ok = __all_sync(0xffffffffu, ok);
+    if constexpr (PHI == 2) {
+      // sum_b (sign(G_b) + 1) / 2  ->  sum_b sign(G_b)
+      const float nbf = (float)nb;
+#pragma unroll
+      for (int j = 0; j < N_STAT; ++j) acc_stat[j] = fmaf(2.f, acc_stat[j], -nbf);
+    }
     constexpr int PANELS = COLS / 32;
     int tile_m, tile_n;
     tc_tile_of_block(p, rank, tile_m, tile_n);
