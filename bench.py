@@ -353,10 +353,11 @@ def run_sweep(args):
             t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
             t_hbm = (bytes_in + 8.0 * d * d) / (peaks["hbm_gbs"] * 1e9)
             t_alu = 2.0 * B * d * d / (148 * 128 * 1.965e9)
-            # sign costs about 5 fp32 operations per entry instead of 2; and short sequences are bound by how many
+            # the sign statistic alone costs 2 fp32 instructions per entry (packed scale, saturating fma, packed add), 4 beside
+            # the other two sums; and short sequences are bound by how many
             # per-example tiles tensor memory holds at once: an accumulator entry is occupied for one hand-off chain
             # (about 1.25 us, measured: stage full seen -> MMAs and commits issued -> epilogue read -> release), 65536 entries per SM
-            t_alu_sign = 5.0 * B * d * d / (148 * 128 * 1.965e9)
+            t_alu_sign = 4.0 * B * d * d / (148 * 128 * 1.965e9)
             t_occupancy = B * float(d) * d / (148 * 65536) * 1.25e-6
             print(json.dumps({
                 "sweep_point": {"B": B, "T": T, "d_in": d, "d_out": d}, "input_sets": nsets,

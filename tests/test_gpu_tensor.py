@@ -314,6 +314,34 @@ def test_three_statistics_need_all_three_outputs():
     assert lib.pe_linear_stats_all(li.X.data_ptr(), li.dY.data_ptr(), 2, 128, 64, 64, out.data_ptr(), out.data_ptr(), None, None) == 1
 
 
+@pytest.mark.parametrize("exponent", [-10, -60, -68, -72])
+def test_sign_statistic_of_tiny_denormal_and_zero_gradients(exponent):
+    """Gradients as small as fp32 denormals keep their sign, and exact zeros of either sign count as zero: every
+    example repeats one token of entries +-2^e (bf16 holds them exactly), so G_b = +-T 2^(2e), down to 2^-139; a block
+    of zero columns in dY with negative X next to it gives -0 products and +0 sums."""
+    B, T, d_in, d_out = 5, 32, 264, 136
+    g = torch.Generator().manual_seed(17 - exponent)
+    sx = (torch.randint(0, 2, (B, 1, d_in), generator=g) * 2 - 1).float()
+    sy = (torch.randint(0, 2, (B, 1, d_out), generator=g) * 2 - 1).float()
+    sy[:, :, 40:56] = 0.0                              # zero gradient columns: G_b[40:56, :] = +-0
+    X = (sx * 2.0 ** exponent).expand(B, T, d_in).to(torch.bfloat16).contiguous().to(DEV)
+    dY = (sy * 2.0 ** exponent).expand(B, T, d_out).to(torch.bfloat16).contiguous().to(DEV)
+    li = inputs.LayerInputs("tiny", X, dY)
+    st = oracle.linear_stats(inputs.to_numpy_bits(X), inputs.to_numpy_bits(dY))
+    want = np.einsum("bo,bi->oi", sy[:, 0, :].numpy(), sx[:, 0, :].numpy())
+    assert np.array_equal(st.sum_sign, want)           # the oracle keeps every sign, whatever the magnitude
+    for path in (pe.PATH_TENSOR, pe.PATH_SIMT):
+        pe.pe_set_path(path)
+        _, stat = gpu_stats(li, "sign")
+        assert pe.pe_last_path() == path
+        assert np.array_equal(stat, want), f"path {path}: {int((stat != want).sum())} entries differ"
+        outs = [torch.full((d_out, d_in), float("nan"), device=DEV) for _ in range(3)]
+        pe.pe_linear_stats_all(X, dY, *outs)
+        torch.cuda.synchronize()
+        assert np.array_equal(outs[2].cpu().numpy(), want)
+        assert np.all(outs[2].cpu().numpy()[40:56] == 0)
+
+
 def test_heavy_tailed_and_heterogeneous_small():
     check_all(inputs.heavy_tailed_layer(12, 128, 256, 384, seed=41, device=DEV))
     check_all(inputs.heterogeneous_layer(20, 64, 128, 256, seed=42, device=DEV))
