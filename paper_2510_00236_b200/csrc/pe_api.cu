@@ -1,11 +1,13 @@
 // C-ABI entry points of libpestats: argument validation, path selection, tensor-map creation and
 // kernel launches.  Everything that computes runs in the CUDA kernels included below.
+#include <algorithm>
 #include <atomic>
 #include <cstdint>
 #include <cstdlib>
 #include <cstring>
 #include <cmath>
 #include <mutex>
+#include <vector>
 
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -175,6 +177,55 @@ static int choose_nsplit(long long tiles, int B, int T, int slots, int max_split
   return best;
 }
 
+// Pair rows per band of the tile order (tc_tile_of_block).  Thread blocks start in the order of their index, `slots`
+// CTA pairs at a time, the batch slices one after the other; such a wave streams, for every example of its slice, the dY
+// panels of the pair rows and the X panels of the column tiles it touches, and between two waves the batch has passed
+// through L2.  So the bytes a launch reads from HBM follow the sum over waves of (pair rows x 256 + column tiles x nt):
+// measured on the 8192 x 2048 layer with 256 sequences of 1024 tokens, 18.5 GB with bands of 8 pair rows, which the
+// waves cut unevenly there, against 13.0 GB with bands of 1 (the model gives 2.54 and 1.88 times the operands' size).
+// The candidates are walked on the host; the previous default is kept unless another band saves more than 3 %.
+static int choose_band(int pairs_m, int tiles_n, int nt, int nsplit, int slots) {
+  const int fallback = pairs_m < TC_BAND ? pairs_m : TC_BAND;
+  const long long total = (long long)pairs_m * tiles_n;
+  if (slots < 1 || pairs_m <= 1 || total * nsplit <= slots) return fallback;       // one wave: the order does not matter
+  struct Key { int pairs_m, tiles_n, nt, nsplit, slots, band; };
+  thread_local Key cache[4] = {};
+  thread_local int cache_next = 0;
+  for (const Key& k : cache)
+    if (k.band > 0 && k.pairs_m == pairs_m && k.tiles_n == tiles_n && k.nt == nt && k.nsplit == nsplit && k.slots == slots) return k.band;
+  // units walked per candidate: the whole launch, or its first 64 Ki thread-block pairs (the pattern repeats)
+  const long long units = total * nsplit < (1ll << 16) ? total * nsplit : (1ll << 16);
+  thread_local std::vector<int> row_seen, col_seen;
+  row_seen.assign((size_t)pairs_m, -1);
+  col_seen.assign((size_t)tiles_n, -1);
+  static const int candidates[] = {TC_BAND, 1, 2, 3, 4, 6, 12, 16};
+  double best_cost = 0.0, fallback_cost = 0.0;
+  int best = fallback;
+  for (int band : candidates) {
+    if (band > pairs_m) band = pairs_m;
+    std::fill(row_seen.begin(), row_seen.end(), -1);
+    std::fill(col_seen.begin(), col_seen.end(), -1);
+    const long long per_band = (long long)band * tiles_n;
+    double cost = 0.0;
+    for (long long u = 0; u < units; ++u) {
+      const int wave = (int)(u / slots);
+      const long long pair_id = u % total;
+      const int b = (int)(pair_id / per_band);
+      const int r = (int)(pair_id - (long long)b * per_band);
+      const int rows = band < pairs_m - b * band ? band : pairs_m - b * band;
+      const int tile_n = r / rows, pair_row = b * band + (r - tile_n * rows);
+      if (row_seen[pair_row] != wave) { row_seen[pair_row] = wave; cost += TC_PAIR_M; }
+      if (col_seen[tile_n] != wave) { col_seen[tile_n] = wave; cost += nt; }
+    }
+    if (band == fallback) fallback_cost = cost;
+    if (best_cost == 0.0 || cost < best_cost) { best_cost = cost; best = band; }
+  }
+  if (fallback_cost > 0.0 && best_cost > 0.97 * fallback_cost) best = fallback;
+  cache[cache_next] = Key{pairs_m, tiles_n, nt, nsplit, slots, best};
+  cache_next = (cache_next + 1) % 4;
+  return best;
+}
+
 static pe_status_t zero_outputs(float* a, float* b, size_t bytes, cudaStream_t st) {
   if (a && cudaMemsetAsync(a, 0, bytes, st) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
   if (b && cudaMemsetAsync(b, 0, bytes, st) != cudaSuccess) { cudaGetLastError(); return PE_ERR_CUDA; }
@@ -280,7 +331,7 @@ static pe_status_t launch_tc(DeviceInfo* di, const void* X, const void* dY, int 
   TcParams p;
   p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = per_example; p.half_operands = half_ops ? 1 : 0;
   p.accumulate = accumulate ? 1 : 0;
-  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
+  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = choose_band(pairs_m, tiles_n, nt, ns, di->sm_count / 2);
   p.out_mean = out_mean; p.out_stat = out_stat; p.out_sign = out_sign; p.out_norms = nullptr; p.dev_status = di->status_ptr;
   p.seq_offsets = nullptr; p.sq_norms = sq_norms; p.clip_norm = clip_norm;
   dim3 grid(2 * pairs_m * tiles_n, 1, ns);
@@ -325,7 +376,7 @@ static pe_status_t launch_tc_norms(DeviceInfo* di, const void* X, const void* dY
   TcParams p;
   p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = 1; p.half_operands = 0;
   p.accumulate = 1;       // nothing is zeroed by a preceding kernel and no matrix is written
-  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
+  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = choose_band(pairs_m, tiles_n, 256, ns, di->sm_count / 2);
   p.out_mean = nullptr; p.out_stat = nullptr; p.out_sign = nullptr; p.out_norms = norms; p.dev_status = di->status_ptr;
   p.seq_offsets = nullptr; p.sq_norms = nullptr; p.clip_norm = 0.f;
   // the three output maps are never used by this variant: any valid map will do
@@ -410,7 +461,7 @@ static pe_status_t launch_tc_ragged(DeviceInfo* di, const void* X, const void* d
   TcParams p;
   p.B = B; p.T = 0; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = 1; p.half_operands = 0;
   p.accumulate = norms ? 1 : 0;
-  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
+  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = choose_band(pairs_m, tiles_n, nt, ns, di->sm_count / 2);
   p.out_mean = both ? out_mean : nullptr; p.out_stat = norms ? nullptr : first; p.out_sign = nullptr; p.out_norms = norms;
   p.seq_offsets = offsets; p.sq_norms = nullptr; p.clip_norm = 0.f; p.dev_status = di->status_ptr;
   const dim3 grid(2 * pairs_m * tiles_n, 1, ns);
@@ -552,7 +603,7 @@ static pe_status_t launch_tc_fused(DeviceInfo* di, const void* X, const void* dY
   }
   TcParams p;
   p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = 1; p.half_operands = 0; p.accumulate = 0;
-  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
+  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = choose_band(pairs_m, tiles_n, nt, ns, di->sm_count / 2);
   p.out_mean = adam ? out_a : nullptr; p.out_stat = out_b; p.out_sign = nullptr; p.out_norms = nullptr; p.dev_status = di->status_ptr;
   p.seq_offsets = nullptr; p.sq_norms = nullptr; p.clip_norm = 0.f;
   opt.kind = kind;
@@ -608,7 +659,7 @@ static pe_status_t launch_tok(DeviceInfo* di, const void* X, const void* dY, lon
   }
   TokParams p;
   p.rows = rows; p.d_in = d_in; p.d_out = d_out; p.pairs_m = pairs_m; p.tiles_n = tiles_n;
-  p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND; p.nsplit = ns; p.dev_status = di->status_ptr;
+  p.band = choose_band(pairs_m, tiles_n, TOK_NT, ns, di->sm_count / 2); p.nsplit = ns; p.dev_status = di->status_ptr;
   return launch_pair_kernel_t(tok_sqstats_kernel, dim3(2 * pairs_m * tiles_n, 1, ns), TOK_THREADS, TOK_SMEM_BYTES, st, ns > 1, mx, my, mo, p);
 }
 
@@ -969,7 +1020,7 @@ static pe_status_t launch_tc_fp8(DeviceInfo* di, const void* x8, const void* y8,
   }
   TcParams p;
   p.B = B; p.T = T; p.d_in = d_in; p.d_out = d_out; p.nsplit = ns; p.per_example = 0; p.half_operands = 0; p.accumulate = 0;
-  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = pairs_m < TC_BAND ? pairs_m : TC_BAND;
+  p.pairs_m = pairs_m; p.tiles_n = tiles_n; p.band = choose_band(pairs_m, tiles_n, 256, ns, di->sm_count / 2);
   p.out_mean = nullptr; p.out_stat = out; p.out_sign = nullptr; p.out_norms = nullptr; p.dev_status = di->status_ptr;
   p.seq_offsets = nullptr; p.sq_norms = nullptr; p.clip_norm = 0.f;
   return launch_tc_inst<0, false, 256, MEAN_NONE, 128, false, OPT_NONE, true>(di, 25, mx, my, mo, mo, mo, p, dim3(2 * pairs_m * tiles_n, 1, ns), st);
