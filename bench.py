@@ -61,8 +61,8 @@ def measured_peaks():
 
 def profile_traffic(workload: str, kernel: str):
     """DRAM bytes per launch of one kernel from the committed ncu summaries, if present (a line
-    "dram_bytes_per_launch <kernel>: <bytes>").  The full large layer is too big to capture; its figures are
-    the 16-sequence slice's, scaled by the examples processed (lines "dram_bytes_per_launch_c4 ...")."""
+    "dram_bytes_per_launch <kernel>: <bytes>").  The large layer's figures (lines "dram_bytes_per_launch_c4 ...")
+    come from a capture of full-size launches with the two DRAM byte counters alone, which take a single pass."""
     fname, tag = {"c2": ("c2", "dram_bytes_per_launch"), "c4s": ("c4_slice", "dram_bytes_per_launch"),
                   "c4": ("c4_slice", "dram_bytes_per_launch_c4")}.get(workload, (workload, "dram_bytes_per_launch"))
     path = os.path.join(ROOT, "profiles", f"tc_stats_kernel_{fname}.txt")
