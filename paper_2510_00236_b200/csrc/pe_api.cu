@@ -189,12 +189,12 @@ static int choose_band(int pairs_m, int tiles_n, int nt, int nsplit, int slots) 
   const long long total = (long long)pairs_m * tiles_n;
   if (slots < 1 || pairs_m <= 1 || total * nsplit <= slots) return fallback;       // one wave: the order does not matter
   struct Key { int pairs_m, tiles_n, nt, nsplit, slots, band; };
-  thread_local Key cache[4] = {};
+  thread_local Key cache[16] = {};
   thread_local int cache_next = 0;
   for (const Key& k : cache)
     if (k.band > 0 && k.pairs_m == pairs_m && k.tiles_n == tiles_n && k.nt == nt && k.nsplit == nsplit && k.slots == slots) return k.band;
-  // units walked per candidate: the whole launch, or its first 64 Ki thread-block pairs (the pattern repeats)
-  const long long units = total * nsplit < (1ll << 16) ? total * nsplit : (1ll << 16);
+  // units walked per candidate: the whole launch, or its first 16 Ki thread-block pairs (over 200 waves; the pattern repeats)
+  const long long units = total * nsplit < (1ll << 14) ? total * nsplit : (1ll << 14);
   thread_local std::vector<int> row_seen, col_seen;
   row_seen.assign((size_t)pairs_m, -1);
   col_seen.assign((size_t)tiles_n, -1);
@@ -222,7 +222,7 @@ static int choose_band(int pairs_m, int tiles_n, int nt, int nsplit, int slots) 
   }
   if (fallback_cost > 0.0 && best_cost > 0.97 * fallback_cost) best = fallback;
   cache[cache_next] = Key{pairs_m, tiles_n, nt, nsplit, slots, best};
-  cache_next = (cache_next + 1) % 4;
+  cache_next = (cache_next + 1) % 16;
   return best;
 }
 

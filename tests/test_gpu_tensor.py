@@ -7,7 +7,7 @@ import torch
 import oracle
 import paper_2510_00236_b200 as pe
 from paper_2510_00236_b200 import inputs
-from parity_util import boundary_and_random, check_all, gpu_stats, rel_frob
+from parity_util import SIGN_REL, boundary_and_random, check_all, check_sign, gpu_stats, rel_frob
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -312,6 +312,28 @@ def test_three_statistics_need_all_three_outputs():
     out = torch.empty((64, 64), device=DEV)
     lib = pe.load_library()
     assert lib.pe_linear_stats_all(li.X.data_ptr(), li.dY.data_ptr(), 2, 128, 64, 64, out.data_ptr(), out.data_ptr(), None, None) == 1
+
+
+@pytest.mark.parametrize("B,T", [(2, 64), (3, 16), (5, 80)])
+def test_launches_of_several_waves_full_comparison(B, T):
+    """10 pair rows x 9-17 column tiles: more thread-block pairs than the GPU holds at once, so the order in which
+    tiles are handed out matters, and the host picks it per launch (bands of 1, 6 or 8 pair rows here, depending on
+    the tile width and the batch split); every output entry is compared."""
+    d_in, d_out = 2112, 2560
+    li = inputs.gaussian_layer(B, T, d_in, d_out, seed=77 + B, device=DEV)
+    check_all(li, phis=("identity", "square", "sign"), token=False)
+    assert pe.pe_last_path() == pe.PATH_TENSOR
+    st = oracle.linear_stats(inputs.to_numpy_bits(li.X), inputs.to_numpy_bits(li.dY), small_rel=SIGN_REL)
+    outs = [torch.full((d_out, d_in), float("nan"), device=DEV) for _ in range(3)]
+    pe.pe_linear_stats_all(li.X, li.dY, *outs)
+    stat_only = torch.full((d_out, d_in), float("nan"), device=DEV)
+    pe.pe_linear_stats(li.X, li.dY, "square", None, stat_only)
+    torch.cuda.synchronize()
+    mean, sq, sg = (o.cpu().numpy() for o in outs)
+    assert np.isfinite(mean).all() and np.isfinite(sq).all() and np.isfinite(sg).all()
+    assert rel_frob(mean, st.sum_g) <= 1e-5 and rel_frob(sq, st.sum_g2) <= 1e-5
+    assert rel_frob(stat_only.cpu().numpy(), st.sum_g2) <= 1e-5
+    check_sign(sg, st)
 
 
 @pytest.mark.parametrize("exponent", [-10, -60, -68, -72])
