@@ -340,12 +340,21 @@ def run_sweep(args):
             mean = torch.empty((d, d), device=dev)
             stat = torch.empty((d, d), device=dev)
             flops = 2.0 * B * T * d * d
-            med_b, best_b = time_each(torch, lambda i: pe.pe_linear_stats(sets[i % nsets].X, sets[i % nsets].dY, pe.PHI_SQUARE, mean, stat), iters=12)
-            med_s, best_s = time_each(torch, lambda i: pe.pe_linear_stats(sets[i % nsets].X, sets[i % nsets].dY, pe.PHI_SQUARE, None, stat), iters=12)
+
+            def rested(fn):
+                # every timed group starts one second after the device went idle: the clock the power limit left behind
+                # a heavy group otherwise carries over into the next one (short sequences ran 1.5x slower right after a
+                # 17 ms point), and the GEMM, timed last, would always meet the hottest chip
+                torch.cuda.synchronize()
+                time.sleep(1.0)
+                return time_each(torch, fn, iters=12)
+
+            med_b, best_b = rested(lambda i: pe.pe_linear_stats(sets[i % nsets].X, sets[i % nsets].dY, pe.PHI_SQUARE, mean, stat))
+            med_s, best_s = rested(lambda i: pe.pe_linear_stats(sets[i % nsets].X, sets[i % nsets].dY, pe.PHI_SQUARE, None, stat))
             sgn = torch.empty((d, d), device=dev)
-            med_n, _ = time_each(torch, lambda i: pe.pe_linear_stats(sets[i % nsets].X, sets[i % nsets].dY, pe.PHI_SIGN, None, stat), iters=12)
-            med_a, _ = time_each(torch, lambda i: pe.pe_linear_stats_all(sets[i % nsets].X, sets[i % nsets].dY, mean, stat, sgn), iters=12)
-            med_g, best_g = time_each(torch, lambda i: torch.matmul(sets[i % nsets].dY.view(B * T, d).t(), sets[i % nsets].X.view(B * T, d)), iters=12)
+            med_n, _ = rested(lambda i: pe.pe_linear_stats(sets[i % nsets].X, sets[i % nsets].dY, pe.PHI_SIGN, None, stat))
+            med_a, _ = rested(lambda i: pe.pe_linear_stats_all(sets[i % nsets].X, sets[i % nsets].dY, mean, stat, sgn))
+            med_g, best_g = rested(lambda i: torch.matmul(sets[i % nsets].dY.view(B * T, d).t(), sets[i % nsets].X.view(B * T, d)))
             status, detail = pe.pe_get_async_status(dev)
             assert status == 0, (status, detail)
             # bounds per point: tensor pipe, the fp32 epilogue (2 ops per example and output entry on
