@@ -377,6 +377,13 @@ int pe_set_path(int path /* pe_path_t */);
 /* The family the most recent pe_linear_stats / pe_token_sqstats call on this thread's process used
  * (PE_PATH_SIMT or PE_PATH_TENSOR; PE_PATH_AUTO if none yet). */
 int pe_last_path(void);
+/* The tile order a tensor-core launch would use, as a host-side query (no GPU is touched): the number of 256-row pair
+ * rows of d_out that consecutive thread-block pairs walk before they move to the next column tile of d_in.  tile_cols is
+ * the tile's width in d_in (128, 192 or 256), batch_slices the number of slices the batch is split into (>= 1),
+ * sm_count the device's SM count (two SMs hold one pair).  The library picks, per launch, the band that minimises the
+ * operand columns its waves of sm_count / 2 pairs stream from memory, sum over waves of (pair rows x 256 + column tiles x
+ * tile_cols); the paper has no counterpart (it leaves scheduling to XLA).  Returns 0 for arguments out of range. */
+int pe_tile_order_band(int d_in, int d_out, int tile_cols, int batch_slices, int sm_count);
 /* Number of kernels the library has launched since load (or since the last reset to 0 via
  * pe_reset_launch_count). */
 long long pe_launch_count(void);

@@ -20,7 +20,7 @@ __all__ = [
     "microadam_family_step", "ADAM_VARIANTS", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms",
     "pe_linear_stats_ragged", "pe_linear_stats_ragged_workspace_bytes", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
     "pe_linear_microadam_step", "pe_linear_microadam_step_f32", "pe_linear_microsignsgd_step", "pe_linear_fused_workspace_bytes",
-    "pe_token_sqstats_fp8", "pe_token_sqstats_fp8_workspace_bytes", "pe_set_wait_limit_cycles",
+    "pe_token_sqstats_fp8", "pe_token_sqstats_fp8_workspace_bytes", "pe_set_wait_limit_cycles", "pe_tile_order_band",
     "pe_set_fused_update", "FUSED_AUTO", "FUSED_ALWAYS", "FUSED_NEVER",
 ]
 
@@ -37,7 +37,7 @@ EXPORTED_SYMBOLS = [
     "pe_token_sqstats_static", "microadam_family_step", "pe_linear_stats_all", "pe_linear_stats_accumulate", "pe_example_sqnorms",
     "pe_linear_stats_ragged", "pe_linear_stats_ragged_workspace_bytes", "pe_example_sqnorms_ragged", "pe_linear_clipped_sum",
     "pe_linear_microadam_step", "pe_linear_microadam_step_f32", "pe_linear_microsignsgd_step", "pe_linear_fused_workspace_bytes",
-    "pe_token_sqstats_fp8", "pe_token_sqstats_fp8_workspace_bytes", "pe_set_wait_limit_cycles",
+    "pe_token_sqstats_fp8", "pe_token_sqstats_fp8_workspace_bytes", "pe_set_wait_limit_cycles", "pe_tile_order_band",
     "pe_set_fused_update",
 ]
 ADAM_VARIANTS = {"adam": 0, "microadam": 1, "microadam_var": 2, "microadam_msq": 3}      # pe_adam_variant_t
@@ -105,6 +105,8 @@ def load_library() -> ctypes.CDLL:
     lib.pe_set_wait_limit_cycles.argtypes = [ll]
     lib.pe_set_wait_limit_cycles.restype = i
     lib.pe_last_path.argtypes = []
+    lib.pe_tile_order_band.argtypes = [ctypes.c_int] * 5
+    lib.pe_tile_order_band.restype = ctypes.c_int
     lib.pe_launch_count.argtypes = []
     lib.pe_launch_count.restype = ll
     lib.pe_reset_launch_count.argtypes = []
@@ -523,6 +525,11 @@ def pe_set_fused_update(mode: int) -> int:
 
 def pe_set_path(path: int) -> int:
     return int(load_library().pe_set_path(int(path)))
+
+
+def pe_tile_order_band(d_in: int, d_out: int, tile_cols: int, batch_slices: int, sm_count: int) -> int:
+    """Pair rows per band of the tile order a tensor-core launch of this shape would use (host-side query)."""
+    return int(load_library().pe_tile_order_band(int(d_in), int(d_out), int(tile_cols), int(batch_slices), int(sm_count)))
 
 
 def pe_last_path() -> int:

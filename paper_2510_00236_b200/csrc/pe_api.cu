@@ -1250,6 +1250,13 @@ int pe_set_path(int path) {
   if (path < PE_PATH_AUTO || path > PE_PATH_TENSOR_WIDE) return -1;
   return g_path.exchange(path);
 }
+int pe_tile_order_band(int d_in, int d_out, int tile_cols, int batch_slices, int sm_count) {
+  if (d_in < 1 || d_out < 1 || batch_slices < 1 || sm_count < 2) return 0;
+  if (tile_cols != 128 && tile_cols != 192 && tile_cols != 256) return 0;
+  const long long tiles_n = ((long long)d_in + tile_cols - 1) / tile_cols, pairs_m = ((long long)d_out + pe::TC_PAIR_M - 1) / pe::TC_PAIR_M;
+  if (tiles_n * pairs_m > (1ll << 29)) return 0;
+  return pe::choose_band((int)pairs_m, (int)tiles_n, tile_cols, batch_slices, sm_count / 2);
+}
 int pe_last_path(void) { return g_last_path.load(); }
 long long pe_launch_count(void) { return g_launches.load(); }
 void pe_reset_launch_count(void) { g_launches.store(0); }

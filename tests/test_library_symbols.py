@@ -125,3 +125,40 @@ def test_cpu_tensors_are_rejected_loudly():
     X = torch.zeros(1, 2, 8, dtype=torch.bfloat16)
     with pytest.raises(pe.PestatsError):
         pe.pe_linear_stats(X, X, "square")
+
+
+def _wave_columns(pairs_m, tiles_n, tile_cols, band, slices, slots):
+    """Operand columns the waves of a launch stream: thread-block pairs start in index order, `slots` at a time, one
+    batch slice after the other; within a slice consecutive pairs walk `band` pair rows, then the next column tile."""
+    order = []
+    for first in range(0, pairs_m, band):
+        rows = min(band, pairs_m - first)
+        order += [(first + r, n) for n in range(tiles_n) for r in range(rows)]
+    units = (order * slices)[: 1 << 14]
+    total = 0
+    for w in range(0, len(units), slots):
+        wave = units[w:w + slots]
+        total += 256 * len({m for m, _ in wave}) + tile_cols * len({n for _, n in wave})
+    return total
+
+
+def test_tile_order_band_follows_the_wave_model(lib):
+    band = pe.pe_tile_order_band
+    # out-of-range arguments
+    assert band(0, 256, 192, 1, 148) == 0 and band(256, 256, 100, 1, 148) == 0 and band(256, 256, 192, 0, 148) == 0
+    # launches of a single wave keep the default: 8 pair rows, or all of them
+    assert band(512, 2048, 192, 3, 148) == 8 and band(1024, 1024, 256, 1, 148) == 4
+    # the large layer (32 pair rows x 11 column tiles of 192, five batch slices): bands of one pair row
+    assert band(2048, 8192, 192, 5, 148) == 1
+    # 16 x 22 tiles: the default is the cheapest
+    assert band(4096, 4096, 192, 1, 148) == 8
+    # whatever it returns costs, by the model, no more than the default, and is within 3 % of the best candidate
+    for (d_in, d_out, cols, slices) in [(2048, 8192, 192, 5), (2048, 8192, 256, 2), (2112, 2560, 192, 1), (2112, 2560, 256, 1),
+                                        (512, 32768, 192, 1), (8192, 2048, 192, 1), (4096, 4096, 256, 2), (1152, 4096, 128, 1)]:
+        pairs_m, tiles_n = -(-d_out // 256), -(-d_in // cols)
+        got = band(d_in, d_out, cols, slices, 148)
+        assert 1 <= got <= pairs_m
+        cost = {b: _wave_columns(pairs_m, tiles_n, cols, min(b, pairs_m), slices, 74) for b in (1, 2, 3, 4, 6, 8, 12, 16)}
+        mine = _wave_columns(pairs_m, tiles_n, cols, got, slices, 74)
+        assert mine <= cost[8]
+        assert mine <= min(cost.values()) / 0.97 + 1
