@@ -678,8 +678,9 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
         if (lane == 0) atomicAdd(p.out_norms + b_begin + a, s);
       } else {
-        // CH columns per tensor-memory read: 32, or 16 where the two running sums leave few registers (NT = 192)
-        constexpr int CH = (NT == 192) ? 16 : 32;
+        // CH columns per tensor-memory read: 32, or 16 where the running sums leave few registers (NT = 192; the three
+        // statistics on the 256 x 128 tile, whose 160 registers of sums leave room for two reads of 16 in flight, not 32)
+        constexpr int CH = (NT == 192 || TRIPLE) ? 16 : 32;
         constexpr int NCH = COLS / CH;                // reads per example
         // grouped examples: the unit's accumulators one after the other; the unit is released after the last read
         const int in_unit = (GROUP > 1) ? min(GROUP, nb - GROUP * a) : 1;
@@ -722,22 +723,24 @@ tc_stats_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
           if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));   // buffer(s) free for the issuer's next example(s)
         };
         // Where the registers allow two reads in flight (running sums of at most 128 floats beside two 32-column
-        // reads), the reads are software-pipelined: read k+1 is issued before the arithmetic on read k, so only the
-        // first read of a unit exposes the tensor-memory latency.  That latency, paid twice per example, was a third
-        // of the epilogue's time per example, which is what bounds short sequences.
-        constexpr bool PIPELINED = CH == 32 && !TRIPLE && PHI != 3;
+        // reads; the three statistics' 160 registers beside two 16-column reads), the reads are software-pipelined:
+        // read k+1 is issued before the arithmetic on read k, so only the first read of a unit exposes the
+        // tensor-memory latency.  That latency, paid twice per example, was a third of the two-sum epilogue's time
+        // per example, which is what bounds short sequences (the three-statistic epilogue, bound by its instruction
+        // count, gains 2-3 %).
+        constexpr bool PIPELINED = (CH == 32 && PHI != 3) || (TRIPLE && NT == 128);
         if constexpr (PIPELINED) {
           constexpr int TOTAL = GROUP * NCH;          // reads per unit when every example of the group exists
           const int n_reads = in_unit * NCH;
           uint32_t ra[CH], rb[CH];
-          tmem_ld_32x32b_x32_issue(taddr, ra);
+          tmem_ld_issue(taddr, ra);
 #pragma unroll
           for (int k = 0; k < TOTAL; ++k) {
             if (GROUP > 1 && k >= n_reads) break;
             if (k & 1) tmem_ld_wait_for(rb); else tmem_ld_wait_for(ra);
             if (k + 1 < n_reads) {
               const uint32_t next = taddr + (uint32_t)(((k + 1) / NCH) * NT + ((k + 1) % NCH) * CH);
-              if (k & 1) tmem_ld_32x32b_x32_issue(next, ra); else tmem_ld_32x32b_x32_issue(next, rb);
+              if (k & 1) tmem_ld_issue(next, ra); else tmem_ld_issue(next, rb);
             } else {
               release_unit();
             }
