@@ -44,7 +44,8 @@ typedef enum {
 
 /* The elementwise function applied to each per-example gradient before the sum over examples
  * (Eq. (2): the nonlinear statistic (1/B) sum_i phi(grad f(theta; x_i)); square gives Eq. (3)'s
- * nu_micro, sign gives the MicroSignSGD statistic of Section 3.1).  sign(0) = 0. */
+ * nu_micro, sign gives the MicroSignSGD statistic of Section 3.1).  sign(+0) = sign(-0) = 0; every other fp32 value of
+ * G_b, denormals included, counts with its sign. */
 typedef enum { PE_PHI_IDENTITY = 0, PE_PHI_SQUARE = 1, PE_PHI_SIGN = 2 } pe_phi_t;
 
 /* Which kernel family a call may use.  AUTO picks the tensor-core kernel whenever the shape allows
